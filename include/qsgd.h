@@ -1,0 +1,148 @@
+/*
+ * qsgd.h -- C ABI of the QSGD gradient codec for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the data-parallel hot path of QSGD (Alistarh et al., arXiv
+ * 1610.02132): Encode = stochastic quantizer Q_s (Section 3.1, Eq. 2; bucketing and max-norm
+ * scaling of Section 4) followed by a lossless code -- either fixed-width bit fields (the
+ * "2/4/8-bit QSGD" of Section 5) or the Elias-coded string S of Section 3.1 / Appendix A.2 --
+ * and Decode of K peers' messages summed into the step of Algorithm 1,
+ * x <- x - (eta / K) * sum_k Decode(M^k).
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless its comment says "host".
+ *     The library allocates no device memory and never synchronises the host: each call
+ *     validates its arguments, enqueues kernels on `stream` and returns.
+ *   - Return value: 0 = launched; < 0 = invalid argument (nothing was launched), see
+ *     QSGD_ERR_*; > 0 = a cudaError_t reported by a launch.
+ *   - Faults found by kernels (message capacity exceeded, malformed Elias stream) are OR-ed
+ *     into status_dev[0] (QSGD_DEV_*). The caller zeroes that word and reads it back when it
+ *     synchronises. A kernel that finds a fault skips the offending write; it never traps.
+ *   - Messages carry no header: n, bucket, s and the code kind are call arguments on both
+ *     sides, as in the paper where sender and receiver agree on s and n.
+ *   - All fp32 arithmetic is round-to-nearest-even without FMA contraction, in the order
+ *     stated below, so a message and a decoded update are bit-reproducible.
+ *   - Inputs must be finite with s * max|g| representable in fp32; otherwise values are
+ *     unspecified but all memory accesses stay in bounds.
+ *
+ * Notation: n coordinates; bucket size d; B = ceil(n / d) buckets, the last one possibly
+ * shorter, each with its own scale; s quantization levels; lb = 1, 2, 4, 8 level bits for
+ * s <= 1, 3, 15, 255.
+ *
+ * Fixed-width message (QSGD_CODE_FIXED): three regions, each zero-padded to a multiple of 16
+ * bytes: fp32 scale A[B] | sign bitmap, coordinate i at bit (i % 32) of u32 word i / 32, set
+ * when the value is negative and its level is nonzero | level fields, coordinate i at bits
+ * [(i * lb) % 32, +lb) of u32 word (i * lb) / 32.
+ *
+ * Elias message (QSGD_CODE_ELIAS): the per-bucket strings S of Section 3.1 (32 bits of the
+ * IEEE-754 pattern of A, then for every nonzero level, in index order: Elias(distance to the
+ * previous nonzero; for the first one its 1-based position), one sign bit, Elias(level))
+ * concatenated without padding. Stream bit t is bit 31 - (t % 32) of u32 word t / 32. The
+ * payload is zero-padded to a multiple of 16 bytes and followed by a table of B + 1 u64 bit
+ * offsets (offset of each bucket's string; last entry = payload bits). The table is an
+ * addition of this format (the paper codes one vector and needs none); sizes are reported
+ * with and without it. QSGD_CODE_ELIAS_DENSE is the variant Code'_s of Appendix A.3: after
+ * the 32 bits of A, every coordinate sends one sign bit and Elias(level + 1).
+ */
+#ifndef QSGD_H_
+#define QSGD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QSGD_NORM_L2 0  /* A = ||v||_2 of the bucket (Eq. 2)              */
+#define QSGD_NORM_MAX 1 /* A = max |v_i| of the bucket (Section 4)        */
+
+#define QSGD_CODE_FIXED 0
+#define QSGD_CODE_ELIAS 1
+#define QSGD_CODE_ELIAS_DENSE 2
+
+#define QSGD_MAX_BUCKET 4096
+#define QSGD_MAX_LEVELS 255
+#define QSGD_MAX_PEERS 64
+
+#define QSGD_OK 0
+#define QSGD_ERR_NULL (-1)      /* a required pointer is null                         */
+#define QSGD_ERR_SIZE (-2)      /* n == 0                                             */
+#define QSGD_ERR_BUCKET (-3)    /* bucket not a multiple of 32 in [32, 4096]          */
+#define QSGD_ERR_LEVELS (-4)    /* s outside [1, 255]                                 */
+#define QSGD_ERR_ALIGN (-5)     /* a pointer is not 16-byte aligned                   */
+#define QSGD_ERR_CAPACITY (-6)  /* out_capacity below the minimum for this call       */
+#define QSGD_ERR_PEERS (-7)     /* K outside [1, 64]                                  */
+#define QSGD_ERR_KIND (-8)      /* unknown norm_kind or code_kind                     */
+#define QSGD_ERR_NO_DEVICE (-9) /* no usable CUDA device / kernel image for this GPU  */
+
+#define QSGD_DEV_CAPACITY 1u  /* encoded message would exceed out_capacity             */
+#define QSGD_DEV_OVERRUN 2u   /* an Elias code runs past the end of its bucket string  */
+#define QSGD_DEV_POSITION 4u  /* a decoded position lies outside its bucket            */
+#define QSGD_DEV_LEVEL 8u     /* a decoded level lies outside [1, s]                   */
+#define QSGD_DEV_TABLE 16u    /* offset table not ascending / bucket shorter than 32   */
+#define QSGD_DEV_TIMEOUT 32u  /* a bounded wait inside a kernel gave up                */
+
+typedef void* qsgd_stream_t; /* a cudaStream_t; NULL is the default stream */
+
+/* Worst-case bytes of one message (Section 3.1 string lengths; fixed-width: exact size). */
+size_t qsgd_message_capacity(uint64_t n, uint32_t bucket, uint32_t s, int code_kind);
+
+/* Bytes of scratch qsgd_encode needs for the Elias kinds (0 for QSGD_CODE_FIXED). */
+size_t qsgd_workspace_bytes(uint64_t n, uint32_t bucket, uint32_t s, int code_kind);
+
+/* Fixed-width layout: layout[0] = byte offset of the sign bitmap, [1] = byte offset of the
+ * level fields, [2] = total bytes, [3] = level bits lb. `layout` is a host pointer. */
+int qsgd_fixed_layout(uint64_t n, uint32_t bucket, uint32_t s, uint64_t* layout);
+
+/*
+ * Encode (Algorithm 1, "M^i <- Encode(g^i)"; Section 3.1, Eq. 2 and the string S).
+ * Per bucket: scale A (fp32; 2-norm accumulated in fp32 per 8 values and fp64 across them,
+ * or the exact maximum); a scale below the smallest normal fp32 makes a zero bucket (A = +0,
+ * all levels 0). Per coordinate i (global index): u = Philox4x32-10(counter = (i / 4 lo,
+ * i / 4 hi, step, worker), key = seed lo, hi) word i % 4, top 24 bits times 2^-24;
+ * level = min(floor((s * |g_i|) * (1 / A) + u), s).
+ *   g            n fp32 values, 16-byte aligned, read once
+ *   out          message buffer of out_capacity bytes, 16-byte aligned, fully overwritten
+ *                up to the message length
+ *   out_bits     4 u64 words written on the stream: [0] payload bits (fixed-width: 8 * bytes),
+ *                [1] byte offset of the offset table in `out` (0 for fixed), [2] message
+ *                bytes, [3] 0
+ *   workspace    qsgd_workspace_bytes() of scratch, 16-byte aligned (may be NULL for fixed)
+ *   status_dev   one u32, OR-ed with QSGD_DEV_CAPACITY when out_capacity is too small
+ */
+int qsgd_encode(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int norm_kind,
+                int code_kind, uint64_t seed, uint32_t step, uint32_t worker, void* out,
+                size_t out_capacity, uint64_t* out_bits, void* workspace, uint32_t* status_dev,
+                qsgd_stream_t stream);
+
+/*
+ * Decode K messages and sum them (Algorithm 1, "g^l <- Decode(M^l)" and the sum):
+ * acc_i = ((+0 + g^0_i) + g^1_i) + ... in ascending k, where g^k_i = +-(A * (level / s)).
+ *   msgs    host array of K device pointers to messages (16-byte aligned)
+ *   tables  host array of K device pointers to the offset tables (Elias kinds; msgs[k] +
+ *           out_bits[1]); NULL for fixed-width
+ *   acc     n fp32 values, overwritten
+ */
+int qsgd_decode_accumulate(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
+                           uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* acc,
+                           uint32_t* status_dev, qsgd_stream_t stream);
+
+/* SGD step (Algorithm 1, last line): c = eta / K once; x_i <- x_i - c * acc_i. */
+int qsgd_sgd_step(float* x, const float* acc, float eta, uint32_t K, uint64_t n,
+                  qsgd_stream_t stream);
+
+/* Decode, sum and step in one pass over x; bit-identical to the two calls above. */
+int qsgd_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
+                         uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* x,
+                         float eta, uint32_t* status_dev, qsgd_stream_t stream);
+
+/* Text for a negative return code ("ok" for 0). Host pointer to a static string. */
+const char* qsgd_status_string(int status);
+
+/* Number of kernels this library has launched in this process (all calls, all streams). */
+uint64_t qsgd_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QSGD_H_ */

@@ -1,0 +1,159 @@
+"""ctypes binding of libqsgd.so: the same entry points as include/qsgd.h, argument marshalling
+only. PyTorch supplies device memory and the CUDA stream; every step of the path runs in the
+library's kernels. There is no CPU fallback: a missing library or a missing device raises.
+"""
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libqsgd.so")
+
+NORM_L2, NORM_MAX = 0, 1
+CODE_FIXED, CODE_ELIAS, CODE_ELIAS_DENSE = 0, 1, 2
+
+DEV_CAPACITY, DEV_OVERRUN, DEV_POSITION, DEV_LEVEL, DEV_TABLE, DEV_TIMEOUT = 1, 2, 4, 8, 16, 32
+
+EXPORTS = ["qsgd_message_capacity", "qsgd_workspace_bytes", "qsgd_fixed_layout", "qsgd_encode",
+           "qsgd_decode_accumulate", "qsgd_sgd_step", "qsgd_decode_sgd_step",
+           "qsgd_status_string", "qsgd_launch_count"]
+
+_lib = None
+
+
+class QsgdError(RuntimeError):
+    pass
+
+
+def lib():
+    """Loads libqsgd.so (must have been built: `python -m paper_1610_02132_b200.build`)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise QsgdError("libqsgd.so is not built; run paper_1610_02132_b200.build.build()")
+        L = C.CDLL(_LIB_PATH)
+        vp, u64, u32, sz = C.c_void_p, C.c_uint64, C.c_uint32, C.c_size_t
+        L.qsgd_message_capacity.argtypes = [u64, u32, u32, C.c_int]
+        L.qsgd_message_capacity.restype = sz
+        L.qsgd_workspace_bytes.argtypes = [u64, u32, u32, C.c_int]
+        L.qsgd_workspace_bytes.restype = sz
+        L.qsgd_fixed_layout.argtypes = [u64, u32, u32, C.POINTER(u64)]
+        L.qsgd_fixed_layout.restype = C.c_int
+        L.qsgd_encode.argtypes = [vp, u64, u32, u32, C.c_int, C.c_int, u64, u32, u32, vp, sz, vp,
+                                  vp, vp, vp]
+        L.qsgd_encode.restype = C.c_int
+        L.qsgd_decode_accumulate.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, u64, u32, u32,
+                                             C.c_int, vp, vp, vp]
+        L.qsgd_decode_accumulate.restype = C.c_int
+        L.qsgd_sgd_step.argtypes = [vp, vp, C.c_float, u32, u64, vp]
+        L.qsgd_sgd_step.restype = C.c_int
+        L.qsgd_decode_sgd_step.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, u64, u32, u32,
+                                           C.c_int, vp, C.c_float, vp, vp]
+        L.qsgd_decode_sgd_step.restype = C.c_int
+        L.qsgd_status_string.argtypes = [C.c_int]
+        L.qsgd_status_string.restype = C.c_char_p
+        L.qsgd_launch_count.argtypes = []
+        L.qsgd_launch_count.restype = u64
+        _lib = L
+    return _lib
+
+
+def _check(st):
+    if st != 0:
+        raise QsgdError("qsgd status %d: %s" % (st, lib().qsgd_status_string(st).decode()))
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _require_cuda(t, name):
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.is_contiguous()):
+        raise QsgdError("%s must be a contiguous CUDA tensor" % name)
+
+
+def qsgd_message_capacity(n, bucket, s, code_kind):
+    return int(lib().qsgd_message_capacity(n, bucket, s, code_kind))
+
+
+def qsgd_workspace_bytes(n, bucket, s, code_kind):
+    return int(lib().qsgd_workspace_bytes(n, bucket, s, code_kind))
+
+
+def qsgd_fixed_layout(n, bucket, s):
+    lay = (C.c_uint64 * 4)()
+    _check(lib().qsgd_fixed_layout(n, bucket, s, lay))
+    return [int(v) for v in lay]
+
+
+def qsgd_launch_count():
+    return int(lib().qsgd_launch_count())
+
+
+def qsgd_encode(g, bucket, s, norm_kind, code_kind, seed, step, worker, out, out_bits,
+                workspace=None, status_dev=None, stream=None, n=None):
+    """Encode g (fp32 CUDA tensor) into `out` (uint8 CUDA tensor); see include/qsgd.h."""
+    _require_cuda(g, "g")
+    _require_cuda(out, "out")
+    _require_cuda(out_bits, "out_bits")
+    _require_cuda(status_dev, "status_dev")
+    n = g.numel() if n is None else n
+    ws = None if workspace is None else C.c_void_p(workspace.data_ptr())
+    _check(lib().qsgd_encode(g.data_ptr(), n, bucket, s, norm_kind, code_kind, seed, step, worker,
+                             out.data_ptr(), out.numel() * out.element_size(),
+                             out_bits.data_ptr(), ws, status_dev.data_ptr(), _stream(stream)))
+
+
+def _ptr_array(tensors):
+    arr = (C.c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = t if isinstance(t, int) else t.data_ptr()
+    return arr
+
+
+def qsgd_decode_accumulate(msgs, tables, n, bucket, s, code_kind, acc, status_dev, stream=None):
+    """acc <- ascending-k sum of the decoded messages; msgs / tables: lists of CUDA tensors
+    (or raw device addresses)."""
+    _require_cuda(acc, "acc")
+    mp = _ptr_array(msgs)
+    tp = None if tables is None else _ptr_array(tables)
+    _check(lib().qsgd_decode_accumulate(mp, tp, len(msgs), n, bucket, s, code_kind,
+                                        acc.data_ptr(), status_dev.data_ptr(), _stream(stream)))
+
+
+def qsgd_sgd_step(x, acc, eta, K, stream=None):
+    _require_cuda(x, "x")
+    _require_cuda(acc, "acc")
+    _check(lib().qsgd_sgd_step(x.data_ptr(), acc.data_ptr(), eta, K, x.numel(), _stream(stream)))
+
+
+def qsgd_decode_sgd_step(msgs, tables, n, bucket, s, code_kind, x, eta, status_dev, stream=None):
+    _require_cuda(x, "x")
+    mp = _ptr_array(msgs)
+    tp = None if tables is None else _ptr_array(tables)
+    _check(lib().qsgd_decode_sgd_step(mp, tp, len(msgs), n, bucket, s, code_kind, x.data_ptr(),
+                                      eta, status_dev.data_ptr(), _stream(stream)))
+
+
+# ------------------------------- conveniences (allocation only) -----------------------------
+def new_status(device="cuda"):
+    return torch.zeros(1, dtype=torch.int32, device=device)
+
+
+def encode_alloc(g, bucket, s, norm_kind, code_kind, seed, step, worker, capacity=None,
+                 stream=None):
+    """Allocates the message, info words, workspace and status, then calls qsgd_encode.
+    Returns (out, out_bits, status_dev); synchronise before reading them on the host."""
+    n = g.numel()
+    cap = qsgd_message_capacity(n, bucket, s, code_kind) if capacity is None else capacity
+    out = torch.empty(cap, dtype=torch.uint8, device=g.device)
+    out_bits = torch.zeros(4, dtype=torch.int64, device=g.device)
+    wsb = qsgd_workspace_bytes(n, bucket, s, code_kind)
+    ws = torch.empty(max(wsb, 16), dtype=torch.uint8, device=g.device)
+    status = new_status(g.device)
+    qsgd_encode(g, bucket, s, norm_kind, code_kind, seed, step, worker, out, out_bits, ws, status,
+                stream)
+    return out, out_bits, status

@@ -1,0 +1,187 @@
+// C ABI of the QSGD codec: argument validation and dispatch to the kernels. See include/qsgd.h
+// for the contract of every entry point.
+#include <atomic>
+
+#include "qsgd_common.cuh"
+
+namespace qsgd {
+
+static std::atomic<uint64_t> g_launches{0};
+void count_launch(int k) { g_launches.fetch_add((uint64_t)k, std::memory_order_relaxed); }
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_shape(uint64_t n, uint32_t bucket, uint32_t s, int code_kind) {
+  if (n == 0) return QSGD_ERR_SIZE;
+  if (bucket < 32 || bucket > QSGD_MAX_BUCKET || (bucket & 31u)) return QSGD_ERR_BUCKET;
+  if (s < 1 || s > QSGD_MAX_LEVELS) return QSGD_ERR_LEVELS;
+  if (code_kind != QSGD_CODE_FIXED && code_kind != QSGD_CODE_ELIAS && code_kind != QSGD_CODE_ELIAS_DENSE)
+    return QSGD_ERR_KIND;
+  return QSGD_OK;
+}
+
+// |Elias(k)| on the host, from the recursive definition (Appendix A.2).
+uint32_t host_elias_len(uint32_t k) {
+  uint32_t len = 1;
+  while (k > 1) {
+    uint32_t m = 0;
+    for (uint32_t t = k; t; t >>= 1) ++m;
+    len += m;
+    k = m - 1;
+  }
+  return len;
+}
+
+int resolve_peers(const void* const* msgs, const uint64_t* const* tables, uint32_t K, uint64_t n,
+                  uint32_t bucket, uint32_t s, int code_kind, PeerSet* ps) {
+  if (!msgs) return QSGD_ERR_NULL;
+  if (K < 1 || K > QSGD_MAX_PEERS) return QSGD_ERR_PEERS;
+  if (code_kind != QSGD_CODE_FIXED && !tables) return QSGD_ERR_NULL;
+  const FixedLayout L = make_fixed_layout(n, bucket, s);
+  for (uint32_t k = 0; k < K; ++k) {
+    if (!msgs[k]) return QSGD_ERR_NULL;
+    if (!aligned16(msgs[k])) return QSGD_ERR_ALIGN;
+    const uint8_t* m = static_cast<const uint8_t*>(msgs[k]);
+    if (code_kind == QSGD_CODE_FIXED) {
+      ps->A[k] = reinterpret_cast<const float*>(m);
+      ps->sign[k] = reinterpret_cast<const uint32_t*>(m + L.off_sign);
+      ps->level[k] = reinterpret_cast<const uint32_t*>(m + L.off_level);
+      ps->payload[k] = nullptr; ps->table[k] = nullptr;
+    } else {
+      if (!tables[k]) return QSGD_ERR_NULL;
+      if (reinterpret_cast<uintptr_t>(tables[k]) & 7u) return QSGD_ERR_ALIGN;
+      ps->A[k] = nullptr; ps->sign[k] = nullptr; ps->level[k] = nullptr;
+      ps->payload[k] = reinterpret_cast<const uint32_t*>(m);
+      ps->table[k] = tables[k];
+    }
+  }
+  return QSGD_OK;
+}
+
+}  // namespace
+}  // namespace qsgd
+
+using namespace qsgd;
+
+extern "C" {
+
+size_t qsgd_message_capacity(uint64_t n, uint32_t bucket, uint32_t s, int code_kind) {
+  if (check_shape(n, bucket, s, code_kind) != QSGD_OK) return 0;
+  if (code_kind == QSGD_CODE_FIXED) return (size_t)make_fixed_layout(n, bucket, s).total;
+  const uint64_t B = (n + bucket - 1) / bucket;
+  // longest string: every coordinate nonzero at the level with the longest code, every gap 1
+  const uint64_t per = code_kind == QSGD_CODE_ELIAS ? 2ull + host_elias_len(s) : 1ull + host_elias_len(s + 1);
+  const uint64_t bits = 32ull * B + n * per;
+  return (size_t)(align16((bits + 7) / 8) + 8 * (B + 1));
+}
+
+size_t qsgd_workspace_bytes(uint64_t n, uint32_t bucket, uint32_t s, int code_kind) {
+  if (check_shape(n, bucket, s, code_kind) != QSGD_OK) return 0;
+  if (code_kind == QSGD_CODE_FIXED) return 0;
+  return elias_workspace_bytes(n, bucket, s);
+}
+
+int qsgd_fixed_layout(uint64_t n, uint32_t bucket, uint32_t s, uint64_t* layout) {
+  if (!layout) return QSGD_ERR_NULL;
+  const int st = check_shape(n, bucket, s, QSGD_CODE_FIXED);
+  if (st) return st;
+  const FixedLayout L = make_fixed_layout(n, bucket, s);
+  layout[0] = L.off_sign; layout[1] = L.off_level; layout[2] = L.total; layout[3] = L.lb;
+  return QSGD_OK;
+}
+
+__global__ void write_fixed_info_kernel(uint64_t* out_bits, uint64_t total) {
+  out_bits[0] = 8 * total; out_bits[1] = 0; out_bits[2] = total; out_bits[3] = 0;
+}
+
+int qsgd_encode(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int norm_kind,
+                int code_kind, uint64_t seed, uint32_t step, uint32_t worker, void* out,
+                size_t out_capacity, uint64_t* out_bits, void* workspace, uint32_t* status_dev,
+                qsgd_stream_t stream) {
+  if (!g || !out || !out_bits || !status_dev) return QSGD_ERR_NULL;
+  int st = check_shape(n, bucket, s, code_kind);
+  if (st) return st;
+  if (norm_kind != QSGD_NORM_L2 && norm_kind != QSGD_NORM_MAX) return QSGD_ERR_KIND;
+  if (!aligned16(g) || !aligned16(out)) return QSGD_ERR_ALIGN;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (code_kind == QSGD_CODE_FIXED) {
+    const FixedLayout L = make_fixed_layout(n, bucket, s);
+    if (out_capacity < L.total) return QSGD_ERR_CAPACITY;
+    st = launch_quantize_fixed(g, n, bucket, s, norm_kind, seed, step, worker,
+                               static_cast<uint8_t*>(out), cs);
+    if (st) return st;
+    write_fixed_info_kernel<<<1, 1, 0, cs>>>(out_bits, L.total);
+    count_launch();
+    return (int)cudaGetLastError();
+  }
+  if (!workspace) return QSGD_ERR_NULL;
+  if (!aligned16(workspace)) return QSGD_ERR_ALIGN;
+  const uint64_t B = (n + bucket - 1) / bucket;
+  if (out_capacity < align16(4 * B) + 8 * (B + 1)) return QSGD_ERR_CAPACITY;   // scales + table
+  return launch_elias_encode(g, n, bucket, s, norm_kind, code_kind == QSGD_CODE_ELIAS_DENSE, seed,
+                             step, worker, static_cast<uint8_t*>(out), out_capacity, out_bits,
+                             static_cast<uint8_t*>(workspace), status_dev, cs);
+}
+
+int qsgd_decode_accumulate(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
+                           uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* acc,
+                           uint32_t* status_dev, qsgd_stream_t stream) {
+  if (!acc || !status_dev) return QSGD_ERR_NULL;
+  int st = check_shape(n, bucket, s, code_kind);
+  if (st) return st;
+  if (!aligned16(acc)) return QSGD_ERR_ALIGN;
+  PeerSet ps;
+  st = resolve_peers(msgs, tables, K, n, bucket, s, code_kind, &ps);
+  if (st) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (code_kind == QSGD_CODE_FIXED) return launch_decode_fixed(ps, K, n, bucket, s, acc, false, 0.f, cs);
+  return launch_decode_elias(ps, K, n, bucket, s, code_kind == QSGD_CODE_ELIAS_DENSE, acc, false, 0.f,
+                             status_dev, cs);
+}
+
+int qsgd_sgd_step(float* x, const float* acc, float eta, uint32_t K, uint64_t n,
+                  qsgd_stream_t stream) {
+  if (!x || !acc) return QSGD_ERR_NULL;
+  if (n == 0) return QSGD_ERR_SIZE;
+  if (K < 1 || K > QSGD_MAX_PEERS) return QSGD_ERR_PEERS;
+  if (!aligned16(x) || !aligned16(acc)) return QSGD_ERR_ALIGN;
+  return launch_sgd_step(x, acc, eta, K, n, static_cast<cudaStream_t>(stream));
+}
+
+int qsgd_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
+                         uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* x,
+                         float eta, uint32_t* status_dev, qsgd_stream_t stream) {
+  if (!x || !status_dev) return QSGD_ERR_NULL;
+  int st = check_shape(n, bucket, s, code_kind);
+  if (st) return st;
+  if (!aligned16(x)) return QSGD_ERR_ALIGN;
+  PeerSet ps;
+  st = resolve_peers(msgs, tables, K, n, bucket, s, code_kind, &ps);
+  if (st) return st;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  if (code_kind == QSGD_CODE_FIXED) return launch_decode_fixed(ps, K, n, bucket, s, x, true, eta, cs);
+  return launch_decode_elias(ps, K, n, bucket, s, code_kind == QSGD_CODE_ELIAS_DENSE, x, true, eta,
+                             status_dev, cs);
+}
+
+const char* qsgd_status_string(int status) {
+  switch (status) {
+    case QSGD_OK: return "ok";
+    case QSGD_ERR_NULL: return "a required pointer is null";
+    case QSGD_ERR_SIZE: return "n must be positive";
+    case QSGD_ERR_BUCKET: return "bucket must be a multiple of 32 in [32, 4096]";
+    case QSGD_ERR_LEVELS: return "s must lie in [1, 255]";
+    case QSGD_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case QSGD_ERR_CAPACITY: return "output capacity too small";
+    case QSGD_ERR_PEERS: return "K must lie in [1, 64]";
+    case QSGD_ERR_KIND: return "unknown norm or code kind";
+    case QSGD_ERR_NO_DEVICE: return "no usable CUDA device";
+    default: return status > 0 ? cudaGetErrorString((cudaError_t)status) : "unknown status";
+  }
+}
+
+uint64_t qsgd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

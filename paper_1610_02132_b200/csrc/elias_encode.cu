@@ -1,0 +1,367 @@
+// Encode, Elias path (Section 3.1 "Efficient Coding of Gradients", string S; Appendix A.3 for
+// the dense variant). Pipeline on one stream:
+//   1. quantize into the fixed-width layout held in the workspace (quantize_fixed.cu);
+//   2. per-bucket string length L_b, one warp per bucket;
+//   3. device-wide exclusive scan of L_b -> bit offsets (block sums, scan of sums, downsweep
+//      that also writes the offset table into the message);
+//   4. zero the payload, then a warp-cooperative scatter writes every bucket's string at its
+//      bit offset: lanes own consecutive sub-ranges of the bucket, a warp scan gives each lane
+//      its first bit, words shared between lanes or buckets are merged with atomicOr.
+#include "elias_common.cuh"
+
+namespace qsgd {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kScanItems = 4;                         // buckets per thread in the scan kernels
+constexpr int kScanBlock = kThreads * kScanItems;     // 1024 buckets per CTA
+
+struct Ctrl {                 // control block at the end of the workspace
+  uint64_t total_bits;
+  uint64_t payload_bytes;
+  uint32_t ok;                // 1 when the message fits out_capacity
+  uint32_t pad;
+};
+
+struct EliasWs {
+  uint8_t* fixed;             // fixed-width intermediate
+  uint32_t* len;              // L_b
+  uint64_t* off;              // offsets (B + 1)
+  uint64_t* block_sums;       // per scan CTA
+  Ctrl* ctrl;
+  size_t bytes;
+};
+
+EliasWs carve(uint8_t* ws, uint64_t n, uint32_t d, uint32_t s) {
+  const FixedLayout L = make_fixed_layout(n, d, s);
+  EliasWs w;
+  size_t o = 0;
+  w.fixed = ws + o; o += align16(L.total);
+  w.len = reinterpret_cast<uint32_t*>(ws + o); o += align16(4 * L.B);
+  w.off = reinterpret_cast<uint64_t*>(ws + o); o += align16(8 * (L.B + 1));
+  const uint64_t nblk = (L.B + kScanBlock - 1) / kScanBlock;
+  w.block_sums = reinterpret_cast<uint64_t*>(ws + o); o += align16(8 * (nblk + 1));
+  w.ctrl = reinterpret_cast<Ctrl*>(ws + o); o += align16(sizeof(Ctrl));
+  w.bytes = o;
+  return w;
+}
+
+// Level field of global coordinate i.
+template <int LB>
+__device__ __forceinline__ uint32_t level_at(const uint32_t* __restrict__ lw, uint64_t i) {
+  const uint64_t bit = i * LB;
+  return (__ldg(lw + (bit >> 5)) >> (bit & 31)) & ((1u << LB) - 1u);
+}
+
+// Walks the nonzero levels of bucket-relative coordinates [c_lo, c_hi) in index order and
+// calls visit(position, level). Whole zero words are skipped.
+template <int LB, typename F>
+__device__ __forceinline__ void for_each_nonzero(const uint32_t* __restrict__ lw, uint64_t base,
+                                                 uint32_t c_lo, uint32_t c_hi, F&& visit) {
+  constexpr uint32_t kMask = (1u << LB) - 1u;
+  uint32_t c = c_lo;
+  while (c < c_hi) {
+    const uint64_t bit = (base + c) * LB;
+    const uint32_t sh = (uint32_t)(bit & 31);
+    uint32_t w = __ldg(lw + (bit >> 5)) >> sh;
+    const uint32_t fields = (32u - sh) / LB;
+    const uint32_t cnt = min(fields, c_hi - c);
+    if (cnt * LB < 32u) w &= (1u << (cnt * LB)) - 1u;
+    while (w) {
+      const uint32_t f = (uint32_t)(__ffs((int)w) - 1) / LB;
+      const uint32_t level = (w >> (f * LB)) & kMask;
+      visit(c + f, level);
+      w &= ~(kMask << (f * LB));
+    }
+    c += cnt;
+  }
+}
+
+struct LaneSummary {
+  uint32_t bits;      // bits of this lane's codes, excluding the gap code of its first nonzero
+  int32_t first;      // first nonzero position in the lane's range, -1 if none
+  int32_t last;       // last nonzero position, -1 if none
+};
+
+template <int LB>
+__device__ __forceinline__ LaneSummary summarize_sparse(const uint32_t* __restrict__ lw,
+                                                        uint64_t base, uint32_t c_lo,
+                                                        uint32_t c_hi) {
+  LaneSummary s{0u, -1, -1};
+  for_each_nonzero<LB>(lw, base, c_lo, c_hi, [&](uint32_t pos, uint32_t level) {
+    if (s.first < 0) s.first = (int32_t)pos;
+    else s.bits += elias_len(pos - (uint32_t)s.last);
+    s.bits += 1u + elias_len(level);
+    s.last = (int32_t)pos;
+  });
+  return s;
+}
+
+template <int LB>
+__device__ __forceinline__ uint32_t summarize_dense(const uint32_t* __restrict__ lw, uint64_t base,
+                                                    uint32_t c_lo, uint32_t c_hi) {
+  uint32_t bits = 0;
+  for (uint32_t c = c_lo; c < c_hi; ++c) bits += 1u + elias_len(level_at<LB>(lw, base + c) + 1u);
+  return bits;
+}
+
+// Position of the last nonzero in the lanes before this one (-1 if none).
+__device__ __forceinline__ int32_t prev_nonzero_before_lane(int32_t last, uint32_t lane) {
+  int32_t run = last;                           // inclusive max-scan of `last`
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int32_t t = __shfl_up_sync(0xffffffffu, run, o);
+    if (lane >= (uint32_t)o) run = max(run, t);
+  }
+  const int32_t excl = __shfl_up_sync(0xffffffffu, run, 1);
+  return lane == 0 ? -1 : excl;
+}
+
+struct BucketParams {
+  const float* A;
+  const uint32_t* sign;
+  const uint32_t* level;
+  uint64_t n;
+  uint32_t d;
+  uint64_t B;
+};
+
+// ---- 2. string length per bucket -------------------------------------------------------------
+template <int LB, bool DENSE>
+__global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketParams p,
+                                                                uint32_t* __restrict__ len) {
+  const uint32_t lane = threadIdx.x & 31;
+  const uint64_t b = (uint64_t)blockIdx.x * kWarps + (threadIdx.x >> 5);
+  if (b >= p.B) return;
+  const uint64_t base = b * p.d;
+  const uint32_t db = (uint32_t)min((uint64_t)p.d, p.n - base);
+  const uint32_t seg = p.d >> 5;
+  const uint32_t c_lo = min(lane * seg, db), c_hi = min(c_lo + seg, db);
+  uint32_t bits;
+  if (DENSE) {
+    bits = summarize_dense<LB>(p.level, base, c_lo, c_hi);
+  } else {
+    const LaneSummary s = summarize_sparse<LB>(p.level, base, c_lo, c_hi);
+    const int32_t prev = prev_nonzero_before_lane(s.last, lane);
+    bits = s.bits + (s.first >= 0 ? elias_len((uint32_t)(s.first - prev)) : 0u);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) bits += __shfl_xor_sync(0xffffffffu, bits, o);
+  if (lane == 0) len[b] = 32u + bits;
+}
+
+// ---- 3. exclusive scan of the lengths --------------------------------------------------------
+__device__ __forceinline__ uint64_t block_exclusive_scan(uint64_t v, uint64_t* total) {
+  __shared__ uint64_t warp_sums[kWarps];
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint64_t inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint64_t t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= (uint32_t)o) inc += t;
+  }
+  if (lane == 31) warp_sums[warp] = inc;
+  __syncthreads();
+  uint64_t before = 0, all = 0;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) {
+    const uint64_t t = warp_sums[w];
+    if ((uint32_t)w < warp) before += t;
+    all += t;
+  }
+  __syncthreads();
+  *total = all;
+  return before + inc - v;
+}
+
+__global__ void __launch_bounds__(kThreads) scan_block_sums_kernel(const uint32_t* __restrict__ len,
+                                                                   uint64_t B,
+                                                                   uint64_t* __restrict__ sums) {
+  const uint64_t i0 = (uint64_t)blockIdx.x * kScanBlock + threadIdx.x * kScanItems;
+  uint64_t v = 0;
+#pragma unroll
+  for (int j = 0; j < kScanItems; ++j) if (i0 + j < B) v += len[i0 + j];
+  uint64_t total;
+  block_exclusive_scan(v, &total);
+  if (threadIdx.x == 0) sums[blockIdx.x] = total;
+}
+
+// One CTA: exclusive scan of the block sums in place; total, message size and capacity check.
+__global__ void __launch_bounds__(kThreads) scan_sums_kernel(uint64_t* __restrict__ sums,
+                                                             uint64_t nblk, uint64_t B,
+                                                             size_t out_capacity, Ctrl* ctrl,
+                                                             uint64_t* __restrict__ out_bits,
+                                                             uint32_t* __restrict__ status_dev) {
+  __shared__ uint64_t carry_s;
+  if (threadIdx.x == 0) carry_s = 0;
+  __syncthreads();
+  for (uint64_t base = 0; base < nblk; base += kThreads) {
+    const uint64_t i = base + threadIdx.x;
+    const uint64_t v = i < nblk ? sums[i] : 0;
+    uint64_t total;
+    const uint64_t ex = block_exclusive_scan(v, &total);
+    const uint64_t carry = carry_s;
+    if (i < nblk) sums[i] = carry + ex;
+    __syncthreads();
+    if (threadIdx.x == 0) carry_s = carry + total;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const uint64_t bits = carry_s;
+    const uint64_t pay = align16((bits + 7) / 8);
+    const uint64_t total_bytes = pay + 8 * (B + 1);
+    const bool ok = total_bytes <= out_capacity;
+    ctrl->total_bits = bits;
+    ctrl->payload_bytes = pay;
+    ctrl->ok = ok ? 1u : 0u;
+    out_bits[0] = bits; out_bits[1] = pay; out_bits[2] = total_bytes; out_bits[3] = 0;
+    if (!ok) atomicOr(status_dev, QSGD_DEV_CAPACITY);
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) scan_downsweep_kernel(const uint32_t* __restrict__ len,
+                                                                  uint64_t B,
+                                                                  const uint64_t* __restrict__ sums,
+                                                                  const Ctrl* __restrict__ ctrl,
+                                                                  uint64_t* __restrict__ off,
+                                                                  uint8_t* __restrict__ out) {
+  const uint64_t i0 = (uint64_t)blockIdx.x * kScanBlock + threadIdx.x * kScanItems;
+  uint32_t l[kScanItems];
+  uint64_t v = 0;
+#pragma unroll
+  for (int j = 0; j < kScanItems; ++j) { l[j] = (i0 + j < B) ? len[i0 + j] : 0u; v += l[j]; }
+  uint64_t total;
+  uint64_t run = sums[blockIdx.x] + block_exclusive_scan(v, &total);
+  const bool ok = ctrl->ok != 0;
+  uint64_t* table = reinterpret_cast<uint64_t*>(out + ctrl->payload_bytes);
+#pragma unroll
+  for (int j = 0; j < kScanItems; ++j) {
+    if (i0 + j < B) {
+      off[i0 + j] = run;
+      if (ok) table[i0 + j] = run;
+      run += l[j];
+      if (i0 + j == B - 1) { off[B] = run; if (ok) table[B] = run; }
+    }
+  }
+}
+
+// ---- 4a. zero the payload ----------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) zero_payload_kernel(uint8_t* __restrict__ out,
+                                                                const Ctrl* __restrict__ ctrl) {
+  if (!ctrl->ok) return;
+  const uint64_t quads = ctrl->payload_bytes / 16;
+  uint4* o = reinterpret_cast<uint4*>(out);
+  for (uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x; i < quads;
+       i += (uint64_t)gridDim.x * kThreads)
+    o[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+// ---- 4b. scatter ---------------------------------------------------------------------------------
+template <int LB, bool DENSE>
+__global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketParams p,
+                                                                 const uint64_t* __restrict__ off,
+                                                                 const Ctrl* __restrict__ ctrl,
+                                                                 uint8_t* __restrict__ out) {
+  if (!ctrl->ok) return;
+  const uint32_t lane = threadIdx.x & 31;
+  const uint64_t b = (uint64_t)blockIdx.x * kWarps + (threadIdx.x >> 5);
+  if (b >= p.B) return;
+  const uint64_t base = b * p.d;
+  const uint32_t db = (uint32_t)min((uint64_t)p.d, p.n - base);
+  const uint32_t seg = p.d >> 5;
+  const uint32_t c_lo = min(lane * seg, db), c_hi = min(c_lo + seg, db);
+
+  uint32_t bits;
+  int32_t prev = -1;
+  if (DENSE) {
+    bits = summarize_dense<LB>(p.level, base, c_lo, c_hi);
+  } else {
+    const LaneSummary s = summarize_sparse<LB>(p.level, base, c_lo, c_hi);
+    prev = prev_nonzero_before_lane(s.last, lane);
+    bits = s.bits + (s.first >= 0 ? elias_len((uint32_t)(s.first - prev)) : 0u);
+  }
+  if (lane == 0) bits += 32u;                       // the scale travels with lane 0
+  uint32_t inc = bits;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= (uint32_t)o) inc += t;
+  }
+  if (bits == 0) return;
+  BitWriter bw;
+  bw.begin(reinterpret_cast<uint32_t*>(out), off[b] + (inc - bits));
+  if (lane == 0) bw.put(__float_as_uint(__ldg(p.A + b)), 32);
+  if (DENSE) {
+    for (uint32_t c = c_lo; c < c_hi; ++c) {
+      const uint64_t i = base + c;
+      const uint32_t sg = (__ldg(p.sign + (i >> 5)) >> (i & 31)) & 1u;
+      uint32_t ln;
+      const uint32_t code = elias_code(level_at<LB>(p.level, i) + 1u, &ln);
+      bw.put((sg << ln) | code, ln + 1);
+    }
+  } else {
+    for_each_nonzero<LB>(p.level, base, c_lo, c_hi, [&](uint32_t pos, uint32_t level) {
+      uint32_t ln;
+      uint32_t code = elias_code(pos - (uint32_t)prev, &ln);
+      bw.put(code, ln);
+      const uint64_t i = base + pos;
+      const uint32_t sg = (__ldg(p.sign + (i >> 5)) >> (i & 31)) & 1u;
+      code = elias_code(level, &ln);
+      bw.put((sg << ln) | code, ln + 1);
+      prev = (int32_t)pos;
+    });
+  }
+  bw.finish();
+}
+
+template <int LB, bool DENSE>
+int run_pipeline(const BucketParams& bp, const EliasWs& w, uint8_t* out, size_t out_capacity,
+                 uint64_t* out_bits, uint32_t* status_dev, cudaStream_t stream) {
+  const uint32_t bucket_grid = (uint32_t)((bp.B + kWarps - 1) / kWarps);
+  const uint64_t nblk = (bp.B + kScanBlock - 1) / kScanBlock;
+  elias_length_kernel<LB, DENSE><<<bucket_grid, kThreads, 0, stream>>>(bp, w.len);
+  scan_block_sums_kernel<<<(uint32_t)nblk, kThreads, 0, stream>>>(w.len, bp.B, w.block_sums);
+  scan_sums_kernel<<<1, kThreads, 0, stream>>>(w.block_sums, nblk, bp.B, out_capacity, w.ctrl,
+                                               out_bits, status_dev);
+  scan_downsweep_kernel<<<(uint32_t)nblk, kThreads, 0, stream>>>(w.len, bp.B, w.block_sums, w.ctrl,
+                                                                 w.off, out);
+  zero_payload_kernel<<<148 * 8, kThreads, 0, stream>>>(out, w.ctrl);
+  elias_scatter_kernel<LB, DENSE><<<bucket_grid, kThreads, 0, stream>>>(bp, w.off, w.ctrl, out);
+  count_launch(6);
+  return (int)cudaGetLastError();
+}
+
+}  // namespace
+
+size_t elias_workspace_bytes(uint64_t n, uint32_t d, uint32_t s) {
+  return carve(nullptr, n, d, s).bytes;
+}
+
+int launch_elias_encode(const float* g, uint64_t n, uint32_t d, uint32_t s, int norm_kind,
+                        bool dense, uint64_t seed, uint32_t step, uint32_t worker, uint8_t* out,
+                        size_t out_capacity, uint64_t* out_bits, uint8_t* workspace,
+                        uint32_t* status_dev, cudaStream_t stream) {
+  const EliasWs w = carve(workspace, n, d, s);
+  int st = launch_quantize_fixed(g, n, d, s, norm_kind, seed, step, worker, w.fixed, stream);
+  if (st) return st;
+  const FixedLayout L = make_fixed_layout(n, d, s);
+  BucketParams bp;
+  bp.A = reinterpret_cast<const float*>(w.fixed);
+  bp.sign = reinterpret_cast<const uint32_t*>(w.fixed + L.off_sign);
+  bp.level = reinterpret_cast<const uint32_t*>(w.fixed + L.off_level);
+  bp.n = n; bp.d = d; bp.B = L.B;
+#define QSGD_RUN(LBV)                                                                            \
+  (dense ? run_pipeline<LBV, true>(bp, w, out, out_capacity, out_bits, status_dev, stream)       \
+         : run_pipeline<LBV, false>(bp, w, out, out_capacity, out_bits, status_dev, stream))
+  switch (L.lb) {
+    case 1: return QSGD_RUN(1);
+    case 2: return QSGD_RUN(2);
+    case 4: return QSGD_RUN(4);
+    default: return QSGD_RUN(8);
+  }
+#undef QSGD_RUN
+}
+
+}  // namespace qsgd

@@ -1,0 +1,118 @@
+// Shared device helpers of the QSGD kernels (sm_100a): Philox4x32-10, message layout,
+// bit-field helpers and the internal launch interface between the C ABI and the kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/qsgd.h"
+
+namespace qsgd {
+
+// ------------------------------------------------------------------------------------------
+// Layout of the fixed-width message (also the intermediate of the Elias encoder).
+// ------------------------------------------------------------------------------------------
+struct FixedLayout {
+  uint64_t n;          // coordinates
+  uint32_t d;          // bucket size
+  uint32_t lb;         // level bits per coordinate: 1, 2, 4, 8
+  uint64_t B;          // buckets
+  uint64_t sign_words; // logical u32 words of the sign bitmap
+  uint64_t level_words;
+  uint64_t off_sign;   // byte offsets of the regions (each 16-byte aligned)
+  uint64_t off_level;
+  uint64_t total;      // message bytes
+};
+
+__host__ __device__ inline uint64_t align16(uint64_t x) { return (x + 15ull) & ~15ull; }
+
+__host__ __device__ inline uint32_t level_bits_for(uint32_t s) {
+  return s <= 1 ? 1u : s <= 3 ? 2u : s <= 15 ? 4u : 8u;
+}
+
+__host__ __device__ inline FixedLayout make_fixed_layout(uint64_t n, uint32_t d, uint32_t s) {
+  FixedLayout L;
+  L.n = n; L.d = d; L.lb = level_bits_for(s);
+  L.B = (n + d - 1) / d;
+  L.sign_words = (n + 31) / 32;
+  L.level_words = (n * L.lb + 31) / 32;
+  L.off_sign = align16(4 * L.B);
+  L.off_level = L.off_sign + align16(4 * L.sign_words);
+  L.total = L.off_level + align16(4 * L.level_words);
+  return L;
+}
+
+// ------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11). One call yields the uniforms of four consecutive
+// coordinates: counter = (q lo, q hi, step, worker) with q = i / 4, key = (seed lo, seed hi).
+// ------------------------------------------------------------------------------------------
+struct PhiloxKey { uint32_t k0, k1; };
+
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               uint32_t k0, uint32_t k1) {
+  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+  constexpr uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+    const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+    c0 = hi1 ^ c1 ^ k0;
+    c1 = lo1;
+    c2 = hi0 ^ c3 ^ k1;
+    c3 = lo0;
+    k0 += W0;
+    k1 += W1;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+// Uniform in [0, 1 - 2^-24]: top 24 bits of a Philox word times 2^-24 (exact in fp32).
+__device__ __forceinline__ float u01_from_bits(uint32_t x) {
+  return __fmul_rn(__uint2float_rn(x >> 8), 5.9604644775390625e-08f);
+}
+
+// Level of one coordinate: min(floor((s * |v|) * r + u), s) with r = 1 / A (0 for a zero
+// bucket). Two multiplies and one add, each rounded to nearest, no contraction.
+__device__ __forceinline__ uint32_t quantize_level(float v, float r, float sf, uint32_t s,
+                                                   uint32_t rnd) {
+  const float t = __fmul_rn(__fmul_rn(sf, fabsf(v)), r);
+  const float c = __fadd_rn(t, u01_from_bits(rnd));
+  const uint32_t l = (uint32_t)__float2int_rz(c);
+  return min(l, s);
+}
+
+// ------------------------------------------------------------------------------------------
+// Internal launch interface (host). Each returns a cudaError_t-compatible int.
+// ------------------------------------------------------------------------------------------
+struct PeerSet {                 // K messages, resolved to region pointers on the host
+  const float* A[QSGD_MAX_PEERS];          // fixed: scale arrays
+  const uint32_t* sign[QSGD_MAX_PEERS];    // fixed: sign bitmaps
+  const uint32_t* level[QSGD_MAX_PEERS];   // fixed: level fields
+  const uint32_t* payload[QSGD_MAX_PEERS]; // Elias: payload words
+  const uint64_t* table[QSGD_MAX_PEERS];   // Elias: offset tables
+};
+
+int launch_quantize_fixed(const float* g, uint64_t n, uint32_t d, uint32_t s, int norm_kind,
+                          uint64_t seed, uint32_t step, uint32_t worker, uint8_t* out,
+                          cudaStream_t stream);
+
+int launch_decode_fixed(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s,
+                        float* acc_or_x, bool fused, float eta, cudaStream_t stream);
+
+int launch_sgd_step(float* x, const float* acc, float eta, uint32_t K, uint64_t n,
+                    cudaStream_t stream);
+
+size_t elias_workspace_bytes(uint64_t n, uint32_t d, uint32_t s);
+
+int launch_elias_encode(const float* g, uint64_t n, uint32_t d, uint32_t s, int norm_kind,
+                        bool dense, uint64_t seed, uint32_t step, uint32_t worker, uint8_t* out,
+                        size_t out_capacity, uint64_t* out_bits, uint8_t* workspace,
+                        uint32_t* status_dev, cudaStream_t stream);
+
+int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s,
+                        bool dense, float* acc_or_x, bool fused, float eta, uint32_t* status_dev,
+                        cudaStream_t stream);
+
+void count_launch(int k = 1);
+
+}  // namespace qsgd

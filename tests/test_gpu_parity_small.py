@@ -1,0 +1,87 @@
+"""GPU parity, whole-message compare at sizes the oracle finishes in seconds: several tiles, a
+ragged tail, every code kind, both norms, all field widths."""
+import numpy as np
+import pytest
+import torch
+
+import paper_1610_02132_b200 as Q
+from oracle import oracle as O
+from paper_1610_02132_b200 import inputs as I
+
+from parity_util import decode_parity, encode_parity
+
+pytestmark = pytest.mark.gpu
+
+CODES = [O.CODE_FIXED, O.CODE_ELIAS, O.CODE_ELIAS_DENSE]
+
+
+def make(n, kind, seed):
+    if kind == "gauss":
+        return I.gaussian(n, 0.01, seed=seed)
+    if kind == "sparse":
+        return I.sparse_laplace(n, 1e-3, 0.3, seed=seed)
+    return I.gaussian_mixture(n, seed=seed)
+
+
+@pytest.mark.parametrize("n,d", [(3 * 4096 + 1234 + 5, 512), (2 * 4096 + 1, 4096), (5000, 128),
+                                 (40000, 96), (777, 32), (1, 32), (33, 32), (4096, 4096)])
+@pytest.mark.parametrize("s", [1, 3, 15, 255])
+@pytest.mark.parametrize("norm_kind", [O.NORM_L2, O.NORM_MAX])
+@pytest.mark.parametrize("code_kind", CODES)
+def test_encode_decode_parity(n, d, s, norm_kind, code_kind):
+    K = 3
+    kinds = ["gauss", "sparse", "mix"]
+    msgs, infos = [], []
+    for w in range(K):
+        g = make(n, kinds[w], seed=10 * n + w)
+        m, info = encode_parity(g, d, s, norm_kind, code_kind, seed=7, step=2, worker=w)
+        msgs.append(m)
+        infos.append(info)
+    x0 = I.gaussian(n, 1.0, seed=99)
+    decode_parity(msgs, infos, n, d, s, code_kind, eta=0.1, x0=x0)
+
+
+@pytest.mark.parametrize("s", [2, 5, 7, 100, 127, 128, 200])
+@pytest.mark.parametrize("code_kind", CODES)
+def test_levels_not_power_of_two(s, code_kind):
+    n, d = 10000, 256
+    msgs, infos = [], []
+    for w in range(2):
+        g = make(n, "gauss", seed=w + 3)
+        m, info = encode_parity(g, d, s, O.NORM_MAX, code_kind, seed=11, step=0, worker=w)
+        msgs.append(m)
+        infos.append(info)
+    decode_parity(msgs, infos, n, d, s, code_kind)
+
+
+@pytest.mark.parametrize("code_kind", CODES)
+def test_degenerate_buckets(code_kind):
+    n, d, s = 4 * 512, 512, 15
+    g = np.zeros(n, dtype=np.float32)
+    g[512:1024] = 1e-41                       # subnormal bucket -> zero bucket
+    g[1024 + 7] = -2.5                        # single nonzero
+    g[1536:] = 3.0                            # all at the maximum
+    g[5] = -0.0
+    for norm_kind in (O.NORM_L2, O.NORM_MAX):
+        m, info = encode_parity(g, d, s, norm_kind, code_kind, seed=1, step=0, worker=0)
+        acc, _ = decode_parity([m], [info], n, d, s, code_kind, eta=1.0)
+        assert not acc[:1024].any() and not np.signbit(acc[:1024]).any()
+        assert acc[1024 + 7] == -2.5
+        if norm_kind == O.NORM_MAX:
+            assert np.all(acc[1536:] == 3.0)
+
+
+def test_many_peers_and_philox_keying():
+    n, d, s = 20000, 512, 15
+    g = make(n, "gauss", 5)
+    msgs, infos = [], []
+    for w in range(20):                       # same gradient, different worker ids
+        m, info = encode_parity(g, d, s, O.NORM_L2, O.CODE_FIXED, seed=2 ** 40 + 3, step=9, worker=w)
+        msgs.append(m)
+        infos.append(info)
+    assert not torch.equal(msgs[0], msgs[1])
+    acc, _ = decode_parity(msgs, infos, n, d, s, O.CODE_FIXED)
+    # the mean of 20 independent quantizations is close to g (unbiasedness, Lemma 3.1)
+    A = O.bucket_scales(g, d, O.NORM_L2)
+    err = np.abs(acc / 20 - g)
+    assert err.max() < 5 * np.repeat(A, d)[:n].max() / 15 / np.sqrt(20) * 0.5 + 1e-3
