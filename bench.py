@@ -1,0 +1,521 @@
+#!/usr/bin/env python
+"""Benchmark of the QSGD hot path on B200: Encode -> (K messages in HBM) -> Decode + aggregate +
+SGD step, through the C ABI (include/qsgd.h).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+One step = one pass of the whole hot path over one batch of synthetic gradients: for every code
+kind of the workload, K worker encodes followed by one fused decode + aggregate + SGD step.
+Prints ONE JSON line (rank 0). Timing is on the device with CUDA events; inputs are resident in
+HBM before the timed region for `value`, and copied from pinned host memory inside it for `e2e`.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+NORM = {"l2": 0, "max": 1}
+CODE = {"fixed": 0, "elias": 1, "elias_dense": 2}
+
+WORKLOADS = {
+    # BASELINE configs: name -> (n, d, s, norm, codes, K, generator)
+    "tiny": dict(n=2 ** 20, d=512, s=15, norm="l2", codes=["fixed"], K=4, gen="gauss0.01",
+                 desc="tiny ref: N(0,0.01^2), n=2^20"),
+    "sparse_elias": dict(n=2 ** 24, d=4096, s=1, norm="l2", codes=["elias"], K=8, gen="sparse_laplace",
+                         desc="sparse Elias regime: Laplace(0,1e-3) with 30% exact zeros, n=2^24"),
+    "alexnet": dict(n=61100840, d=512, s=255, norm="max", codes=["fixed"], K=16, gen="alexnet",
+                    desc="AlexNet-shaped flat gradient, layer sigma 1e-2/sqrt(fan_in)"),
+    "resnet152": dict(n=60192808, d=512, s=15, norm="l2", codes=["fixed", "elias"], K=16, gen="mixture",
+                      desc="ResNet-152-shaped flat gradient, 0.9 N(0,1e-4^2) + 0.1 N(0,1e-2^2)"),
+    "sweep_point": dict(n=2 ** 28, d=512, s=15, norm="l2", codes=["fixed"], K=16, gen="gauss1",
+                        desc="bandwidth sweep point: N(0,1), n=2^28"),
+}
+DEFAULT_WORKLOAD = "resnet152"
+ETA = 0.1
+PHILOX_SEED = 7
+
+
+def elen(k):
+    return 1 if k == 1 else k.bit_length() + elen(k.bit_length() - 1)
+
+
+def fixed_bytes(n, d, s):
+    lb = 1 if s <= 1 else 2 if s <= 3 else 4 if s <= 15 else 8
+    a16 = lambda x: (x + 15) // 16 * 16  # noqa: E731
+    B = (n + d - 1) // d
+    return a16(4 * B) + a16(4 * ((n + 31) // 32)) + a16(4 * ((n * lb + 31) // 32))
+
+
+# ------------------------------------------------------------------------------------------------
+# inputs
+# ------------------------------------------------------------------------------------------------
+def host_gradient(wl, worker, n=None):
+    from paper_1610_02132_b200 import inputs as I
+    n = wl["n"] if n is None else n
+    seed = 1 + worker
+    gen = wl["gen"]
+    if gen == "gauss0.01":
+        return I.gaussian(n, 0.01, seed)
+    if gen == "gauss1":
+        return I.gaussian(n, 1.0, seed)
+    if gen == "sparse_laplace":
+        return I.sparse_laplace(n, 1e-3, 0.3, seed)
+    if gen == "alexnet":
+        return I.layered_gaussian(I.alexnet_shapes(), seed)[:n]
+    return I.gaussian_mixture(n, seed)
+
+
+def device_gradient(wl, worker, device):
+    from paper_1610_02132_b200 import inputs as I
+    n, seed, gen = wl["n"], 1 + worker, wl["gen"]
+    if gen == "gauss0.01":
+        return I.gaussian_device(n, 0.01, seed, device)
+    if gen == "gauss1":
+        return I.gaussian_device(n, 1.0, seed, device)
+    if gen == "sparse_laplace":
+        return I.sparse_laplace_device(n, 1e-3, 0.3, seed, device)
+    if gen == "alexnet":
+        return I.layered_gaussian_device(I.alexnet_shapes(), seed, device=device)
+    return I.gaussian_mixture_device(n, seed, device=device)
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.idx = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile(prefix="clocks", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.idx), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1])); mx.append(float(p[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                    "sw_power_cap"), p[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            busy = [c for c in sm if c > 0.5 * max(sm)] or sm
+            out.update(sm_mhz=statistics.median(busy), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA arm
+# ------------------------------------------------------------------------------------------------
+class HotPath:
+    """Buffers and one step of the hot path for a workload on one GPU."""
+
+    def __init__(self, wl, device, rank=0):
+        import torch
+        import paper_1610_02132_b200 as Q
+        self.torch, self.Q, self.wl, self.dev = torch, Q, wl, device
+        n, d, s, K = wl["n"], wl["d"], wl["s"], wl["K"]
+        self.n, self.d, self.s, self.K = n, d, s, K
+        self.B = (n + d - 1) // d
+        self.norm = NORM[wl["norm"]]
+        self.codes = [CODE[c] for c in wl["codes"]]
+        # the K workers' gradients (rank shifts the seeds so replicas differ)
+        self.g = [device_gradient(wl, rank * K + w, device) for w in range(K)]
+        self.x = torch.zeros(n, dtype=torch.float32, device=device)
+        self.status = Q.new_status(device)
+        self.msgs, self.bits, self.ws, self.tables = {}, {}, {}, {}
+        for code in self.codes:
+            cap = self.message_capacity(code)
+            self.msgs[code] = [torch.empty(cap, dtype=torch.uint8, device=device) for _ in range(K)]
+            self.bits[code] = torch.zeros(K, 4, dtype=torch.int64, device=device)
+            wsb = max(Q.qsgd_workspace_bytes(n, d, s, code), 16)
+            self.ws[code] = torch.empty(wsb, dtype=torch.uint8, device=device)
+        self.info = {}
+
+    def message_capacity(self, code):
+        """Fixed-width: exact. Elias: the fixed-width size is used as capacity (an Elias message
+        longer than that is not worth sending); a first encode verifies it fits."""
+        Q = self.Q
+        if code == 0:
+            return Q.qsgd_message_capacity(self.n, self.d, self.s, code)
+        worst = Q.qsgd_message_capacity(self.n, self.d, self.s, code)
+        return min(worst, 2 * fixed_bytes(self.n, self.d, self.s) + 8 * (self.B + 1))
+
+    def encode_all(self, code, step, src=None):
+        Q = self.Q
+        g = self.g if src is None else src
+        for w in range(self.K):
+            Q.qsgd_encode(g[w], self.d, self.s, self.norm, code, PHILOX_SEED, step, w,
+                          self.msgs[code][w], self.bits[code][w], self.ws[code], self.status)
+
+    def resolve_tables(self, code):
+        """Elias: the sender reads the message length back (it needs it to send the message);
+        the offset table sits at byte out_bits[1] of each message."""
+        if code == 0:
+            return None
+        info = self.bits[code].cpu().numpy().view(np.uint64)        # synchronises the stream
+        self.info[code] = info
+        nb = 8 * (self.B + 1)
+        return [self.msgs[code][w][int(info[w, 1]): int(info[w, 1]) + nb].view(self.torch.int64)
+                for w in range(self.K)]
+
+    def step(self, step_idx, src=None):
+        for code in self.codes:
+            self.encode_all(code, step_idx, src)
+            tables = self.resolve_tables(code)
+            self.Q.qsgd_decode_sgd_step(self.msgs[code], tables, self.n, self.d, self.s, code, self.x,
+                                        ETA, self.status)
+
+    def message_bytes(self, code):
+        if code == 0:
+            return float(fixed_bytes(self.n, self.d, self.s))
+        info = self.info[code]
+        return float(np.mean(info[:, 2].astype(np.float64)))
+
+    def payload_bits_per_coord(self, code):
+        if code == 0:
+            return 8.0 * fixed_bytes(self.n, self.d, self.s) / self.n
+        return float(np.mean(self.info[code][:, 0].astype(np.float64))) / self.n
+
+
+def kernel_algorithmic_bytes(hp, code_name):
+    """Bytes each kernel must move per launch (the method's own inputs and outputs)."""
+    n, d, s, K, B = hp.n, hp.d, hp.s, hp.K, hp.B
+    MF = fixed_bytes(n, d, s)
+    out = {"quantize_fixed": 4 * n + MF, "decode_fixed": K * MF + 8 * n, "sgd_step": 12 * n}
+    if 1 in hp.info:
+        info = hp.info[1]
+        msg = float(np.mean(info[:, 2].astype(np.float64)))
+        pay = float(np.mean(info[:, 1].astype(np.float64)))
+        out.update({"decode_elias": K * msg + 8 * n, "elias_scatter": MF + pay,
+                    "elias_length": MF - 4 * ((n + 31) // 32) + 4 * B, "zero_payload": pay,
+                    "scan_block_sums": 4 * B, "scan_downsweep": 4 * B + 16 * (B + 1)})
+    return out
+
+
+def load_traffic():
+    p = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        return json.load(open(p))
+    except Exception:
+        return {}
+
+
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+    import paper_1610_02132_b200 as Q
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    wl = dict(WORKLOADS[args.workload])
+    for k in ("n", "d", "s", "K"):
+        if getattr(args, k) is not None:
+            wl[k] = getattr(args, k)
+    if args.norm:
+        wl["norm"] = args.norm
+    if args.codes:
+        wl["codes"] = args.codes.split(",")
+
+    hp = HotPath(wl, device, rank)
+    n, K = hp.n, hp.K
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ---------------------------------------------------------------
+    for i in range(args.warmup):
+        hp.step(i)
+    barrier()
+    assert int(hp.status.item()) == 0, "device status %d after warm-up" % int(hp.status.item())
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    launches0 = Q.qsgd_launch_count()
+    Q.qsgd_profile_enable(True)
+    Q.qsgd_profile_collect()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for i in range(args.steps):
+        hp.step(args.warmup + i)
+    ev1.record()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    Q.qsgd_profile_enable(False)
+    kern = Q.qsgd_profile_collect()
+    launches = Q.qsgd_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    assert int(hp.status.item()) == 0
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+
+    # fp32 gradient bytes that went through Encode plus through Decode, per step, all ranks
+    grad_bytes = world * len(hp.codes) * 2 * K * 4 * n
+    value = grad_bytes / (ms_step * 1e-3) / 1e9
+
+    # ---- per-phase figures (one extra pass, per-call events) ----------------------------------
+    phases = {}
+    for code_name, code in zip(wl["codes"], hp.codes):
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        torch.cuda.synchronize()
+        e[0].record()
+        hp.encode_all(code, 1000)
+        e[1].record()
+        tables = hp.resolve_tables(code)
+        torch.cuda.synchronize()
+        e[1].record()
+        Q.qsgd_decode_sgd_step(hp.msgs[code], tables, hp.n, hp.d, hp.s, code, hp.x, ETA, hp.status)
+        e[2].record()
+        torch.cuda.synchronize()
+        t_enc, t_dec = e[0].elapsed_time(e[1]) * 1e-3 / K, e[1].elapsed_time(e[2]) * 1e-3
+        # encode time above includes the table read-back for Elias; re-time encode alone
+        torch.cuda.synchronize(); e[0].record(); hp.encode_all(code, 1001); e[1].record()
+        torch.cuda.synchronize()
+        t_enc = e[0].elapsed_time(e[1]) * 1e-3 / K
+        M = hp.message_bytes(code)
+        phases[code_name] = {
+            "encode_GBps_fp32": 4 * n / t_enc / 1e9,
+            "decode_sgd_GBps_fp32": K * 4 * n / t_dec / 1e9,
+            "encode_us": t_enc * 1e6, "decode_sgd_us": t_dec * 1e6,
+            "encode_alg_GBps": (4 * n + M) / t_enc / 1e9,
+            "decode_alg_GBps": (K * M + 8 * n) / t_dec / 1e9,
+            "message_bytes": M, "bits_per_coord_payload": hp.payload_bits_per_coord(code),
+            "bits_per_coord_message": 8 * M / n,
+        }
+
+    # ---- roofline of the dominant kernel ------------------------------------------------------
+    hbm_peak, peak_src = (peaks.get("hbm_gbs"), "measured") if peaks.get("hbm_gbs") else (6650.0, "fallback")
+    alg = kernel_algorithmic_bytes(hp, None)
+    kern_tab = {k: {"ms_total": v[0], "launches": v[1], "avg_us": 1e3 * v[0] / v[1]} for k, v in kern.items()}
+    tot = sum(v[0] for v in kern.values()) or 1.0
+    for k in kern_tab:
+        kern_tab[k]["share"] = kern_tab[k]["ms_total"] / tot
+        if k in alg:
+            kern_tab[k]["alg_GBps"] = alg[k] / (kern_tab[k]["avg_us"] * 1e-6) / 1e9
+            kern_tab[k]["frac_of_%s_hbm" % peak_src] = kern_tab[k]["alg_GBps"] / hbm_peak
+    dom = max(kern, key=lambda k: kern[k][0])
+    traffic_tab = load_traffic().get(dom)
+    traffic = None
+    if traffic_tab and traffic_tab.get("bytes_per_coord") is not None:
+        traffic = traffic_tab["bytes_per_coord"] * n
+    achieved = alg.get(dom, 0) / (kern_tab[dom]["avg_us"] * 1e-6) / 1e9
+    roofline = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+                "frac": achieved / hbm_peak, "peak_source": peak_src, "frac_of_nominal_8000": achieved / 8000.0,
+                "traffic": traffic, "alg_bytes_per_launch": alg.get(dom),
+                "avg_launch_us": kern_tab[dom]["avg_us"], "share_of_kernel_time": kern_tab[dom]["share"]}
+
+    # ---- end to end: host buffers, copies inside the timed region -----------------------------
+    e2e = None
+    if not args.no_e2e:
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        pinned = [torch.empty(n, dtype=torch.float32).pin_memory() for _ in range(K)]
+        for w in range(K):
+            pinned[w].copy_(hp.g[w])
+        x_host = torch.empty(n, dtype=torch.float32).pin_memory()
+        stage = [torch.empty(n, dtype=torch.float32, device=device) for _ in range(2)]
+
+        def e2e_step(i):
+            for code in hp.codes:
+                for w in range(K):
+                    buf = stage[w & 1]
+                    buf.copy_(pinned[w], non_blocking=True)
+                    Q.qsgd_encode(buf, hp.d, hp.s, hp.norm, code, PHILOX_SEED, i, w, hp.msgs[code][w],
+                                  hp.bits[code][w], hp.ws[code], hp.status)
+                tables = hp.resolve_tables(code)
+                Q.qsgd_decode_sgd_step(hp.msgs[code], tables, hp.n, hp.d, hp.s, code, hp.x, ETA, hp.status)
+                x_host.copy_(hp.x, non_blocking=True)
+            torch.cuda.synchronize()
+
+        e2e_step(0)
+        barrier()
+        ev0.record()
+        for i in range(e2e_steps):
+            e2e_step(1 + i)
+        ev1.record()
+        barrier()
+        t = torch.tensor([ev0.elapsed_time(ev1)], dtype=torch.float64, device=device)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item()) / e2e_steps
+        e2e = {"value": grad_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
+               "steps": e2e_steps, "h2d_bytes_per_step": len(hp.codes) * K * 4 * n,
+               "d2h_bytes_per_step": len(hp.codes) * (4 * n + 32 * K * (1 if 1 in hp.codes else 0))}
+        del pinned, x_host, stage
+
+    # ---- CPU baseline: the oracle on a bounded sample -----------------------------------------
+    cpu = None
+    if rank == 0 and not args.no_cpu:
+        cpu = run_oracle_sample(wl, steps=1)
+
+    if rank == 0:
+        line = {
+            "metric": "QSGD encode + decode+aggregate throughput, fp32 gradient GB/s",
+            "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload + ": " + wl["desc"], "n": n, "bucket": hp.d, "s": hp.s,
+                       "norm": wl["norm"], "codes": wl["codes"], "K": K,
+                       "l2": "inputs larger than L2 (K gradients = %.0f MB rotate through 126 MB)" % (K * 4 * n / 1e6),
+                       "step": "per code kind: K encodes, message-size read-back (Elias), fused decode+aggregate+SGD"},
+            "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "roofline": roofline, "cpu_baseline": cpu, "phases": phases, "kernels": kern_tab,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+# the reference arm / CPU baseline: the oracle, as it stands, on host cores
+# ------------------------------------------------------------------------------------------------
+def run_oracle_sample(wl, steps=1, workers=2):
+    """Times the oracle on a bounded sample: the first `workers` of the K workers' gradients at
+    full n (capped at 2^25 coordinates), every code kind of the workload: encode each, then
+    decode + aggregate + SGD step."""
+    from oracle import oracle as O
+    n = min(wl["n"], 2 ** 25)
+    n -= n % wl["d"] if n > wl["d"] else 0
+    d, s, norm = wl["d"], wl["s"], NORM[wl["norm"]]
+    gs = [host_gradient(wl, w, n) for w in range(workers)]
+    x = np.zeros(n, dtype=np.float32)
+    t_total, bytes_total = 0.0, 0
+    for it in range(steps):
+        for code_name in wl["codes"]:
+            code = CODE[code_name]
+            t0 = time.perf_counter()
+            msgs, tabs = [], []
+            for w, g in enumerate(gs):
+                m, info = O.encode(g, d, s, norm, code, PHILOX_SEED, it, w)
+                msgs.append(m)
+                tabs.append(None if code == 0 else O.message_table(m, info, n, d))
+            st, acc = O.decode_accumulate(msgs, None if code == 0 else tabs, n, d, s, code)
+            x = O.sgd_step(x, acc, ETA, workers)
+            t_total += time.perf_counter() - t0
+            bytes_total += 2 * workers * 4 * n
+    return {"value": bytes_total / t_total / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "seconds": t_total,
+            "sample": "%d of %d workers, first %d of %d coordinates, codes %s, %d step(s)" % (
+                workers, wl["K"], n, wl["n"], ",".join(wl["codes"]), steps)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = dict(WORKLOADS[args.workload])
+    for k in ("n", "d", "s", "K"):
+        if getattr(args, k) is not None:
+            wl[k] = getattr(args, k)
+    for i in range(args.warmup):
+        run_oracle_sample(wl, steps=1, workers=1)
+        break                                         # one warm-up pass pages the library in
+    t0 = time.perf_counter()
+    cpu = run_oracle_sample(wl, steps=args.steps, workers=2)
+    dt = time.perf_counter() - t0
+    line = {
+        "impl": "reference", "metric": "QSGD encode + decode+aggregate throughput, fp32 gradient GB/s",
+        "value": cpu["value"], "unit": "GB/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * cpu["seconds"] / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic", "wall_s": dt,
+        "config": {"workload": args.workload + ": " + wl["desc"], "n": wl["n"], "bucket": wl["d"],
+                   "s": wl["s"], "norm": wl["norm"], "codes": wl["codes"], "K": wl["K"]},
+        "cpu_baseline": cpu,
+        "e2e": {"value": cpu["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--n", type=int, default=None)
+    ap.add_argument("--d", type=int, default=None)
+    ap.add_argument("--s", type=int, default=None)
+    ap.add_argument("--K", type=int, default=None)
+    ap.add_argument("--norm", default=None, choices=["l2", "max"])
+    ap.add_argument("--codes", default=None, help="comma list of fixed,elias,elias_dense")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--capture", action="store_true",
+                    help="for runs under a profiler: keep --warmup as given, skip e2e and the CPU baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 1 if args.steps is None else min(args.steps, 4)
+        run_reference(args)
+        return
+    if args.steps is None:
+        args.steps = 10
+    if args.capture:
+        args.no_e2e = args.no_cpu = True
+    else:
+        args.warmup = max(args.warmup, 3)
+    run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -142,6 +142,18 @@ const char* qsgd_status_string(int status);
 /* Number of kernels this library has launched in this process (all calls, all streams). */
 uint64_t qsgd_launch_count(void);
 
+/*
+ * Per-kernel timing (measurement aid; the paper has no counterpart). While enabled, every
+ * kernel launch of the library is bracketed by two CUDA events on its stream.
+ * qsgd_profile_collect waits for the recorded events, adds each kernel's elapsed time and
+ * launch count into the host arrays total_ms[] / launches[] (qsgd_profile_kernel_count()
+ * entries, indexed by kernel id) and forgets them. Returns 0 or a cudaError_t.
+ */
+void qsgd_profile_enable(int on);
+int qsgd_profile_kernel_count(void);
+const char* qsgd_profile_kernel_name(int id);
+int qsgd_profile_collect(double* total_ms, uint64_t* launches);
+
 #ifdef __cplusplus
 }
 #endif

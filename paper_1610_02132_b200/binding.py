@@ -17,7 +17,8 @@ DEV_CAPACITY, DEV_OVERRUN, DEV_POSITION, DEV_LEVEL, DEV_TABLE, DEV_TIMEOUT = 1, 
 
 EXPORTS = ["qsgd_message_capacity", "qsgd_workspace_bytes", "qsgd_fixed_layout", "qsgd_encode",
            "qsgd_decode_accumulate", "qsgd_sgd_step", "qsgd_decode_sgd_step",
-           "qsgd_status_string", "qsgd_launch_count"]
+           "qsgd_status_string", "qsgd_launch_count", "qsgd_profile_enable",
+           "qsgd_profile_kernel_count", "qsgd_profile_kernel_name", "qsgd_profile_collect"]
 
 _lib = None
 
@@ -55,6 +56,14 @@ def lib():
         L.qsgd_status_string.restype = C.c_char_p
         L.qsgd_launch_count.argtypes = []
         L.qsgd_launch_count.restype = u64
+        L.qsgd_profile_enable.argtypes = [C.c_int]
+        L.qsgd_profile_enable.restype = None
+        L.qsgd_profile_kernel_count.argtypes = []
+        L.qsgd_profile_kernel_count.restype = C.c_int
+        L.qsgd_profile_kernel_name.argtypes = [C.c_int]
+        L.qsgd_profile_kernel_name.restype = C.c_char_p
+        L.qsgd_profile_collect.argtypes = [C.POINTER(C.c_double), C.POINTER(u64)]
+        L.qsgd_profile_collect.restype = C.c_int
         _lib = L
     return _lib
 
@@ -91,6 +100,23 @@ def qsgd_fixed_layout(n, bucket, s):
 
 def qsgd_launch_count():
     return int(lib().qsgd_launch_count())
+
+
+def qsgd_profile_enable(on):
+    lib().qsgd_profile_enable(1 if on else 0)
+
+
+def qsgd_profile_collect():
+    """Returns {kernel name: (total ms, launches)} for the launches recorded since the last call."""
+    L = lib()
+    k = L.qsgd_profile_kernel_count()
+    ms = (C.c_double * k)()
+    cnt = (C.c_uint64 * k)()
+    st = L.qsgd_profile_collect(ms, cnt)
+    if st != 0:
+        raise QsgdError("qsgd_profile_collect: cuda error %d" % st)
+    return {L.qsgd_profile_kernel_name(i).decode(): (float(ms[i]), int(cnt[i]))
+            for i in range(k) if cnt[i]}
 
 
 def qsgd_encode(g, bucket, s, norm_kind, code_kind, seed, step, worker, out, out_bits,

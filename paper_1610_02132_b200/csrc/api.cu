@@ -1,13 +1,41 @@
 // C ABI of the QSGD codec: argument validation and dispatch to the kernels. See include/qsgd.h
 // for the contract of every entry point.
 #include <atomic>
+#include <mutex>
+#include <vector>
 
 #include "qsgd_common.cuh"
 
 namespace qsgd {
 
 static std::atomic<uint64_t> g_launches{0};
-void count_launch(int k) { g_launches.fetch_add((uint64_t)k, std::memory_order_relaxed); }
+static std::atomic<int> g_profile{0};
+static std::mutex g_prof_mu;
+struct TimedLaunch { KernelId id; cudaEvent_t a, b; };
+static std::vector<TimedLaunch> g_timed;
+
+ScopedKernel::ScopedKernel(KernelId id_, cudaStream_t stream_) : id(id_), stream(stream_), start(nullptr) {
+  g_launches.fetch_add(1, std::memory_order_relaxed);
+  if (g_profile.load(std::memory_order_relaxed)) {
+    cudaEventCreate(&start);
+    cudaEventRecord(start, stream);
+  }
+}
+
+ScopedKernel::~ScopedKernel() {
+  if (start) {
+    cudaEvent_t stop;
+    cudaEventCreate(&stop);
+    cudaEventRecord(stop, stream);
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_timed.push_back({id, start, stop});
+  }
+}
+
+static const char* const kKernelNames[kKernCount] = {
+    "quantize_fixed", "fixed_info", "decode_fixed", "sgd_step", "elias_length",
+    "scan_block_sums", "scan_sums", "scan_downsweep", "zero_payload", "elias_scatter",
+    "decode_elias"};
 
 namespace {
 
@@ -112,8 +140,10 @@ int qsgd_encode(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int nor
     st = launch_quantize_fixed(g, n, bucket, s, norm_kind, seed, step, worker,
                                static_cast<uint8_t*>(out), cs);
     if (st) return st;
-    write_fixed_info_kernel<<<1, 1, 0, cs>>>(out_bits, L.total);
-    count_launch();
+    {
+      ScopedKernel sk(kKernFixedInfo, cs);
+      write_fixed_info_kernel<<<1, 1, 0, cs>>>(out_bits, L.total);
+    }
     return (int)cudaGetLastError();
   }
   if (!workspace) return QSGD_ERR_NULL;
@@ -183,5 +213,33 @@ const char* qsgd_status_string(int status) {
 }
 
 uint64_t qsgd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+void qsgd_profile_enable(int on) { g_profile.store(on ? 1 : 0, std::memory_order_relaxed); }
+
+int qsgd_profile_kernel_count(void) { return (int)kKernCount; }
+
+const char* qsgd_profile_kernel_name(int id) {
+  return (id >= 0 && id < (int)kKernCount) ? kKernelNames[id] : "";
+}
+
+int qsgd_profile_collect(double* total_ms, uint64_t* launches) {
+  std::vector<TimedLaunch> mine;
+  {
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    mine.swap(g_timed);
+  }
+  for (int i = 0; i < (int)kKernCount; ++i) { total_ms[i] = 0.0; launches[i] = 0; }
+  int rc = 0;
+  for (const TimedLaunch& t : mine) {
+    float ms = 0.f;
+    cudaError_t e = cudaEventSynchronize(t.b);
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, t.a, t.b);
+    if (e != cudaSuccess) rc = (int)e;
+    else { total_ms[t.id] += (double)ms; launches[t.id] += 1; }
+    cudaEventDestroy(t.a);
+    cudaEventDestroy(t.b);
+  }
+  return rc;
+}
 
 }  // extern "C"

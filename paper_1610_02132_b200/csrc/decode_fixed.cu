@@ -106,9 +106,11 @@ __global__ void __launch_bounds__(kThreads) sgd_step_kernel(float* __restrict__ 
 
 template <int LB>
 int launch_lb(const DecodeParams& p, bool fused, uint32_t grid, cudaStream_t stream) {
-  if (fused) decode_fixed_kernel<LB, true><<<grid, kThreads, 0, stream>>>(p);
-  else decode_fixed_kernel<LB, false><<<grid, kThreads, 0, stream>>>(p);
-  count_launch();
+  {
+    ScopedKernel sk(kKernDecodeFixed, stream);
+    if (fused) decode_fixed_kernel<LB, true><<<grid, kThreads, 0, stream>>>(p);
+    else decode_fixed_kernel<LB, false><<<grid, kThreads, 0, stream>>>(p);
+  }
   return (int)cudaGetLastError();
 }
 
@@ -134,8 +136,10 @@ int launch_sgd_step(float* x, const float* acc, float eta, uint32_t K, uint64_t 
   const float c = eta / (float)K;
   const uint64_t quads = (n + 3) / 4;
   const uint32_t grid = (uint32_t)((quads + kThreads - 1) / kThreads);
-  sgd_step_kernel<<<grid, kThreads, 0, stream>>>(x, acc, c, n);
-  count_launch();
+  {
+    ScopedKernel sk(kKernSgdStep, stream);
+    sgd_step_kernel<<<grid, kThreads, 0, stream>>>(x, acc, c, n);
+  }
   return (int)cudaGetLastError();
 }
 

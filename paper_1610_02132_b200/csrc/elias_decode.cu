@@ -188,8 +188,10 @@ int launch_t(EliasDecodeParams& p, bool fused, cudaStream_t stream) {
   const uint64_t want = (p.B + kWarps - 1) / kWarps;
   const uint64_t cap = (uint64_t)sms * 16;
   const uint32_t grid = (uint32_t)(want < cap ? want : cap);
-  kern<<<grid, kThreads, smem, stream>>>(p);
-  count_launch();
+  {
+    ScopedKernel sk(kKernDecodeElias, stream);
+    kern<<<grid, kThreads, smem, stream>>>(p);
+  }
   return (int)cudaGetLastError();
 }
 

@@ -321,15 +321,32 @@ int run_pipeline(const BucketParams& bp, const EliasWs& w, uint8_t* out, size_t 
                  uint64_t* out_bits, uint32_t* status_dev, cudaStream_t stream) {
   const uint32_t bucket_grid = (uint32_t)((bp.B + kWarps - 1) / kWarps);
   const uint64_t nblk = (bp.B + kScanBlock - 1) / kScanBlock;
-  elias_length_kernel<LB, DENSE><<<bucket_grid, kThreads, 0, stream>>>(bp, w.len);
-  scan_block_sums_kernel<<<(uint32_t)nblk, kThreads, 0, stream>>>(w.len, bp.B, w.block_sums);
-  scan_sums_kernel<<<1, kThreads, 0, stream>>>(w.block_sums, nblk, bp.B, out_capacity, w.ctrl,
-                                               out_bits, status_dev);
-  scan_downsweep_kernel<<<(uint32_t)nblk, kThreads, 0, stream>>>(w.len, bp.B, w.block_sums, w.ctrl,
-                                                                 w.off, out);
-  zero_payload_kernel<<<148 * 8, kThreads, 0, stream>>>(out, w.ctrl);
-  elias_scatter_kernel<LB, DENSE><<<bucket_grid, kThreads, 0, stream>>>(bp, w.off, w.ctrl, out);
-  count_launch(6);
+  {
+    ScopedKernel sk(kKernEliasLength, stream);
+    elias_length_kernel<LB, DENSE><<<bucket_grid, kThreads, 0, stream>>>(bp, w.len);
+  }
+  {
+    ScopedKernel sk(kKernScanBlockSums, stream);
+    scan_block_sums_kernel<<<(uint32_t)nblk, kThreads, 0, stream>>>(w.len, bp.B, w.block_sums);
+  }
+  {
+    ScopedKernel sk(kKernScanSums, stream);
+    scan_sums_kernel<<<1, kThreads, 0, stream>>>(w.block_sums, nblk, bp.B, out_capacity, w.ctrl,
+                                                 out_bits, status_dev);
+  }
+  {
+    ScopedKernel sk(kKernScanDownsweep, stream);
+    scan_downsweep_kernel<<<(uint32_t)nblk, kThreads, 0, stream>>>(w.len, bp.B, w.block_sums,
+                                                                   w.ctrl, w.off, out);
+  }
+  {
+    ScopedKernel sk(kKernZeroPayload, stream);
+    zero_payload_kernel<<<148 * 8, kThreads, 0, stream>>>(out, w.ctrl);
+  }
+  {
+    ScopedKernel sk(kKernEliasScatter, stream);
+    elias_scatter_kernel<LB, DENSE><<<bucket_grid, kThreads, 0, stream>>>(bp, w.off, w.ctrl, out);
+  }
   return (int)cudaGetLastError();
 }
 

@@ -113,6 +113,21 @@ int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d
                         bool dense, float* acc_or_x, bool fused, float eta, uint32_t* status_dev,
                         cudaStream_t stream);
 
-void count_launch(int k = 1);
+// Every kernel launch is bracketed by one of these: it counts the launch and, while kernel
+// timing is switched on (qsgd_profile_enable), records a CUDA event before and after it on the
+// launching stream.
+enum KernelId {
+  kKernQuantize = 0, kKernFixedInfo, kKernDecodeFixed, kKernSgdStep, kKernEliasLength,
+  kKernScanBlockSums, kKernScanSums, kKernScanDownsweep, kKernZeroPayload, kKernEliasScatter,
+  kKernDecodeElias, kKernCount
+};
+
+struct ScopedKernel {
+  ScopedKernel(KernelId id, cudaStream_t stream);
+  ~ScopedKernel();
+  KernelId id;
+  cudaStream_t stream;
+  cudaEvent_t start;
+};
 
 }  // namespace qsgd

@@ -179,9 +179,11 @@ __global__ void __launch_bounds__(kThreads) quantize_fixed_kernel(const Quantize
 
 template <int LB>
 int launch_lb(const QuantizeParams& p, int norm_kind, uint32_t grid, cudaStream_t stream) {
-  if (norm_kind == QSGD_NORM_L2) quantize_fixed_kernel<LB, QSGD_NORM_L2><<<grid, kThreads, 0, stream>>>(p);
-  else quantize_fixed_kernel<LB, QSGD_NORM_MAX><<<grid, kThreads, 0, stream>>>(p);
-  count_launch();
+  {
+    ScopedKernel sk(kKernQuantize, stream);
+    if (norm_kind == QSGD_NORM_L2) quantize_fixed_kernel<LB, QSGD_NORM_L2><<<grid, kThreads, 0, stream>>>(p);
+    else quantize_fixed_kernel<LB, QSGD_NORM_MAX><<<grid, kThreads, 0, stream>>>(p);
+  }
   return (int)cudaGetLastError();
 }
 
