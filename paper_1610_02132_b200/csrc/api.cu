@@ -138,7 +138,7 @@ int qsgd_encode(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int nor
     const FixedLayout L = make_fixed_layout(n, bucket, s);
     if (out_capacity < L.total) return QSGD_ERR_CAPACITY;
     st = launch_quantize_fixed(g, n, bucket, s, norm_kind, seed, step, worker,
-                               static_cast<uint8_t*>(out), cs);
+                               static_cast<uint8_t*>(out), status_dev, cs);
     if (st) return st;
     {
       ScopedKernel sk(kKernFixedInfo, cs);

@@ -1,8 +1,15 @@
 // Decode-and-aggregate, fixed-width path, optionally fused with the SGD step (Algorithm 1:
-// g^l <- Decode(M^l); x <- x - (eta / K) * sum_l g^l). A thread owns 8 consecutive
-// coordinates and walks the K messages in ascending k, so every coordinate's sum has the fixed
-// order ((0 + g^0) + g^1) + ... . Reconstruction is A * (level / s): level / s comes from a
-// table of correctly rounded quotients, then one multiply (Eq. 2).
+// g^l <- Decode(M^l); x <- x - (eta / K) * sum_l g^l).
+//
+// A warp owns chunks of 512 consecutive coordinates, a lane 16 of them, and walks the K
+// messages in ascending k, so every coordinate's sum has the fixed order ((0 + g^0) + g^1) ...
+// With K = 16 peers there are only a handful of issue slots per (peer, coordinate) at HBM
+// speed, so reconstruction A * (level / s) * sign is a table lookup:
+//   * s <= 15: the 2 * (s + 1) possible values +-A * (level / s) of one (peer, bucket) live one
+//     per lane and are fetched with a warp shuffle indexed by "sign | level"; the sign bits are
+//     spread next to the level nibbles with one multiply per four coordinates;
+//   * s >= 16: level / s (correctly rounded) comes from a shared-memory table replicated per
+//     lane (bank-conflict free), followed by the multiply with A and a sign flip.
 #include "qsgd_common.cuh"
 
 namespace qsgd {
@@ -10,6 +17,8 @@ namespace qsgd {
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kChunk = 512;            // coordinates per warp iteration
 
 struct DecodeParams {
   PeerSet peers;
@@ -17,72 +26,131 @@ struct DecodeParams {
   uint64_t n;
   uint32_t d;
   uint32_t s;
+  uint32_t log2_chunks_per_bucket;   // valid when single_scale
   float* out;      // acc (overwritten) or x (updated in place)
   float c;         // eta / K (fused only)
+  uint64_t chunks;
 };
 
-template <int LB, bool FUSED>
-__global__ void __launch_bounds__(kThreads) decode_fixed_kernel(const __grid_constant__ DecodeParams p) {
-  __shared__ float xi[256];
-  const float sf = (float)p.s;
-  for (uint32_t l = threadIdx.x; l < (1u << LB); l += kThreads) xi[l] = __fdiv_rn((float)l, sf);
-  __syncthreads();
+__device__ __forceinline__ float shfl_f(float v, uint32_t src) {
+  return __shfl_sync(0xffffffffu, v, (int)src);
+}
 
-  const uint64_t grp = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
-  const uint64_t i0 = grp * 8;
-  if (i0 >= p.n) return;
-  const uint64_t b = i0 / p.d;
-  constexpr uint32_t kMask = (1u << LB) - 1u;
-
-  float acc[8];
+// Adds peer k's 16 values to acc[]. SINGLE: the whole chunk lies in one bucket and `lut` is
+// already scaled by A; otherwise `lut` holds +-(level / s) and A is this lane's bucket scale.
+template <int LB, bool SINGLE>
+__device__ __forceinline__ void add_peer_lut(float (&acc)[16], const uint32_t (&w)[4], uint32_t sb,
+                                             float lut, float A) {
+  if (LB == 4) {
 #pragma unroll
-  for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-
-  for (uint32_t k = 0; k < p.K; ++k) {
-    const float A = __ldg(p.peers.A[k] + b);
-    const uint32_t sb = __ldg(reinterpret_cast<const uint8_t*>(p.peers.sign[k]) + grp);
-    uint32_t w0, w1 = 0;
-    if (LB == 8) {
-      const uint2 t = __ldg(reinterpret_cast<const uint2*>(p.peers.level[k]) + grp);
-      w0 = t.x; w1 = t.y;
-    } else if (LB == 4) {
-      w0 = __ldg(p.peers.level[k] + grp);
-    } else if (LB == 2) {
-      w0 = __ldg(reinterpret_cast<const uint16_t*>(p.peers.level[k]) + grp);
-    } else {
-      w0 = __ldg(reinterpret_cast<const uint8_t*>(p.peers.level[k]) + grp);
+    for (int h = 0; h < 2; ++h) {
+      const uint32_t word = w[h], s8 = sb >> (8 * h);
+      const uint32_t ev = word & 0x0F0F0F0Fu, od = (word >> 4) & 0x0F0F0F0Fu;
+      const uint32_t ie = (((s8 & 0x55u) * 0x00410410u) & 0x10101010u) | ev;   // coords 0,2,4,6
+      const uint32_t io = (((s8 & 0xAAu) * 0x00208208u) & 0x10101010u) | od;   // coords 1,3,5,7
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float a = shfl_f(lut, ie >> (8 * j));
+        float b = shfl_f(lut, io >> (8 * j));
+        if (!SINGLE) { a = __fmul_rn(A, a); b = __fmul_rn(A, b); }
+        acc[8 * h + 2 * j] = __fadd_rn(acc[8 * h + 2 * j], a);
+        acc[8 * h + 2 * j + 1] = __fadd_rn(acc[8 * h + 2 * j + 1], b);
+      }
     }
+  } else {
+    // LB = 1 or 2: 16 fields in w[0]
+    constexpr uint32_t kMask = (1u << LB) - 1u;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      uint32_t l;
-      if (LB == 8) l = ((e < 4 ? w0 : w1) >> (8 * (e & 3))) & 0xFFu;
-      else l = (w0 >> (LB * e)) & kMask;
-      float m = __fmul_rn(A, xi[l]);
-      if ((sb >> e) & 1u) m = -m;
-      acc[e] = __fadd_rn(acc[e], m);
+    for (int e = 0; e < 16; ++e) {
+      const uint32_t idx = ((w[0] >> (LB * e)) & kMask) | (((sb >> e) & 1u) << LB);
+      float a = shfl_f(lut, idx);
+      if (!SINGLE) a = __fmul_rn(A, a);
+      acc[e] = __fadd_rn(acc[e], a);
     }
   }
+}
 
-  float* o = p.out + i0;
-  if (i0 + 8 <= p.n) {
-    float4 r0, r1;
-    if (FUSED) {
-      const float4 x0 = *reinterpret_cast<const float4*>(o);
-      const float4 x1 = *reinterpret_cast<const float4*>(o + 4);
-      r0.x = __fsub_rn(x0.x, __fmul_rn(p.c, acc[0])); r0.y = __fsub_rn(x0.y, __fmul_rn(p.c, acc[1]));
-      r0.z = __fsub_rn(x0.z, __fmul_rn(p.c, acc[2])); r0.w = __fsub_rn(x0.w, __fmul_rn(p.c, acc[3]));
-      r1.x = __fsub_rn(x1.x, __fmul_rn(p.c, acc[4])); r1.y = __fsub_rn(x1.y, __fmul_rn(p.c, acc[5]));
-      r1.z = __fsub_rn(x1.z, __fmul_rn(p.c, acc[6])); r1.w = __fsub_rn(x1.w, __fmul_rn(p.c, acc[7]));
-    } else {
-      r0 = make_float4(acc[0], acc[1], acc[2], acc[3]);
-      r1 = make_float4(acc[4], acc[5], acc[6], acc[7]);
-    }
-    *reinterpret_cast<float4*>(o) = r0;
-    *reinterpret_cast<float4*>(o + 4) = r1;
-  } else {
+// LB = 8: table lookup of level / s in shared memory (entry l of lane t at word l * 32 + t).
+__device__ __forceinline__ void add_peer_tab(float (&acc)[16], const uint32_t (&w)[4], uint32_t sb,
+                                             const uint8_t* tab_lane, float A) {
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      if (i0 + e < p.n) o[e] = FUSED ? __fsub_rn(o[e], __fmul_rn(p.c, acc[e])) : acc[e];
+  for (int h = 0; h < 4; ++h) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t off = (j == 0 ? (w[h] << 7) : (w[h] >> (8 * j - 7))) & 0x7F80u;
+      const float xi = *reinterpret_cast<const float*>(tab_lane + off);
+      const uint32_t m = __float_as_uint(__fmul_rn(A, xi)) ^ ((sb << (31 - (4 * h + j))) & 0x80000000u);
+      acc[4 * h + j] = __fadd_rn(acc[4 * h + j], __uint_as_float(m));
+    }
+  }
+}
+
+template <int LB, bool FUSED, bool SINGLE>
+__global__ void __launch_bounds__(kThreads) decode_fixed_kernel(const __grid_constant__ DecodeParams p) {
+  __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const float sf = (float)p.s;
+  float lut0 = 0.f;                                  // this lane's +-(level / s)
+  if (LB == 8) {
+    for (uint32_t i = tid; i < 256 * 32; i += kThreads) xi_tab[i] = __fdiv_rn((float)(i >> 5), sf);
+    __syncthreads();
+  } else {
+    const uint32_t level = lane & ((1u << LB) - 1u), neg = (lane >> LB) & 1u;
+    const float q = __fdiv_rn((float)level, sf);
+    lut0 = neg ? -q : q;
+  }
+  const uint8_t* tab_lane = reinterpret_cast<const uint8_t*>(xi_tab) + 4 * lane;
+
+  for (uint64_t ch = (uint64_t)blockIdx.x * kWarps + warp; ch < p.chunks; ch += (uint64_t)gridDim.x * kWarps) {
+    const uint64_t i0 = ch * kChunk + (uint64_t)lane * 16;       // first coordinate of this lane
+    const bool live = i0 < p.n;                                   // lanes past n only help shuffles
+    const uint64_t b = SINGLE ? (ch >> p.log2_chunks_per_bucket) : (live ? i0 / p.d : 0);
+    float acc[16];
+#pragma unroll
+    for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+
+#pragma unroll 4
+    for (uint32_t k = 0; k < p.K; ++k) {
+      uint32_t w[4] = {0u, 0u, 0u, 0u};
+      uint32_t sb = 0;
+      float A = 0.f;
+      if (live) {
+        A = __ldg(p.peers.A[k] + b);
+        sb = __ldg(reinterpret_cast<const uint16_t*>(p.peers.sign[k]) + (i0 >> 4));
+        if (LB == 8) {
+          const uint4 t = __ldg(reinterpret_cast<const uint4*>(p.peers.level[k]) + (i0 >> 4));
+          w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
+        } else if (LB == 4) {
+          const uint2 t = __ldg(reinterpret_cast<const uint2*>(p.peers.level[k]) + (i0 >> 4));
+          w[0] = t.x; w[1] = t.y;
+        } else if (LB == 2) {
+          w[0] = __ldg(p.peers.level[k] + (i0 >> 4));
+        } else {
+          w[0] = __ldg(reinterpret_cast<const uint16_t*>(p.peers.level[k]) + (i0 >> 4));
+        }
+      }
+      if (LB == 8) add_peer_tab(acc, w, sb, tab_lane, A);
+      else if (SINGLE) add_peer_lut<LB, true>(acc, w, sb, __fmul_rn(__shfl_sync(0xffffffffu, A, 0), lut0), A);
+      else add_peer_lut<LB, false>(acc, w, sb, lut0, A);
+    }
+
+    if (!live) continue;
+    float* o = p.out + i0;
+    if (i0 + 16 <= p.n) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float4 r = make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+        if (FUSED) {
+          const float4 x = *reinterpret_cast<const float4*>(o + 4 * j);
+          r.x = __fsub_rn(x.x, __fmul_rn(p.c, r.x)); r.y = __fsub_rn(x.y, __fmul_rn(p.c, r.y));
+          r.z = __fsub_rn(x.z, __fmul_rn(p.c, r.z)); r.w = __fsub_rn(x.w, __fmul_rn(p.c, r.w));
+        }
+        *reinterpret_cast<float4*>(o + 4 * j) = r;
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 16; ++e)
+        if (i0 + e < p.n) o[e] = FUSED ? __fsub_rn(o[e], __fmul_rn(p.c, acc[e])) : acc[e];
     }
   }
 }
@@ -104,14 +172,31 @@ __global__ void __launch_bounds__(kThreads) sgd_step_kernel(float* __restrict__ 
   }
 }
 
-template <int LB>
-int launch_lb(const DecodeParams& p, bool fused, uint32_t grid, cudaStream_t stream) {
+template <int LB, bool FUSED, bool SINGLE>
+int launch_one(const DecodeParams& p, cudaStream_t stream) {
+  static int sms = 0, occ = 0;
+  auto kern = decode_fixed_kernel<LB, FUSED, SINGLE>;
+  if (sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, 0);
+    if (occ < 1) occ = 1;
+  }
+  const uint64_t want = (p.chunks + kWarps - 1) / kWarps;
+  const uint64_t cap = (uint64_t)sms * occ;
+  const uint32_t grid = (uint32_t)(want < cap ? want : cap);
   {
     ScopedKernel sk(kKernDecodeFixed, stream);
-    if (fused) decode_fixed_kernel<LB, true><<<grid, kThreads, 0, stream>>>(p);
-    else decode_fixed_kernel<LB, false><<<grid, kThreads, 0, stream>>>(p);
+    kern<<<grid, kThreads, 0, stream>>>(p);
   }
   return (int)cudaGetLastError();
+}
+
+template <int LB>
+int launch_lb(const DecodeParams& p, bool fused, bool single, cudaStream_t stream) {
+  if (fused) return single ? launch_one<LB, true, true>(p, stream) : launch_one<LB, true, false>(p, stream);
+  return single ? launch_one<LB, false, true>(p, stream) : launch_one<LB, false, false>(p, stream);
 }
 
 }  // namespace
@@ -121,13 +206,16 @@ int launch_decode_fixed(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d
   DecodeParams p;
   p.peers = peers; p.K = K; p.n = n; p.d = d; p.s = s; p.out = acc_or_x;
   p.c = eta / (float)K;
-  const uint64_t groups = (n + 7) / 8;
-  const uint32_t grid = (uint32_t)((groups + kThreads - 1) / kThreads);
+  p.chunks = (n + kChunk - 1) / kChunk;
+  // one scale per chunk when the bucket size is 512 * 2^j
+  const bool single = d >= (uint32_t)kChunk && (d & (d - 1)) == 0;
+  p.log2_chunks_per_bucket = 0;
+  for (uint32_t t = d / kChunk; single && t > 1; t >>= 1) ++p.log2_chunks_per_bucket;
   switch (level_bits_for(s)) {
-    case 1: return launch_lb<1>(p, fused, grid, stream);
-    case 2: return launch_lb<2>(p, fused, grid, stream);
-    case 4: return launch_lb<4>(p, fused, grid, stream);
-    default: return launch_lb<8>(p, fused, grid, stream);
+    case 1: return launch_lb<1>(p, fused, single, stream);
+    case 2: return launch_lb<2>(p, fused, single, stream);
+    case 4: return launch_lb<4>(p, fused, single, stream);
+    default: return launch_lb<8>(p, fused, false, stream);
   }
 }
 

@@ -361,7 +361,7 @@ int launch_elias_encode(const float* g, uint64_t n, uint32_t d, uint32_t s, int 
                         size_t out_capacity, uint64_t* out_bits, uint8_t* workspace,
                         uint32_t* status_dev, cudaStream_t stream) {
   const EliasWs w = carve(workspace, n, d, s);
-  int st = launch_quantize_fixed(g, n, d, s, norm_kind, seed, step, worker, w.fixed, stream);
+  int st = launch_quantize_fixed(g, n, d, s, norm_kind, seed, step, worker, w.fixed, status_dev, stream);
   if (st) return st;
   const FixedLayout L = make_fixed_layout(n, d, s);
   BucketParams bp;

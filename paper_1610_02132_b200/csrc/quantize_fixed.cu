@@ -1,12 +1,22 @@
 // Encode, fixed-width path: bucket scale + Philox stochastic rounding + bit packing in one pass
 // over the gradient (Section 3.1, Eq. 2; Section 4 bucketing / max-norm; Section 5 bit widths).
 //
-// One CTA owns a tile of whole buckets (<= 4096 coordinates) staged in shared memory. A thread
-// owns groups of 8 consecutive coordinates: it reads them once, contributes a partial sum of
-// squares (or maximum) to the bucket reduction, and after the scales are known quantizes the
-// same registers, so the gradient is read from HBM exactly once. Sign bits and level fields
-// of neighbouring lanes are merged with shuffles into whole 32-bit words before they are
-// stored.
+// Main kernel (bucket size a power of two): persistent CTAs walk tiles of 4096 coordinates.
+// Tiles arrive in shared memory through a ring of 1-D TMA bulk copies (cp.async.bulk +
+// mbarrier), so no thread spends instructions on loads. A thread owns 16 consecutive
+// coordinates: it pulls them into registers once, the bucket scale is reduced with shuffles
+// (plus one shared-memory exchange when a bucket spans several warps), and the same registers
+// are then quantized, so the gradient is read from HBM exactly once. The arithmetic is written
+// to keep the instruction count per coordinate low, because at HBM speed this kernel has only
+// about 25 issue slots per coordinate:
+//   * the uniform u = m * 2^-24 (m = top 24 Philox bits) enters as fma(m, 2^-24, t), which
+//     rounds exactly like t + u because m * 2^-24 is exact;
+//   * floor(c) is the round-down add c + 2^23, whose mantissa then holds the integer;
+//   * level fields are packed by Horner multiply-adds on those raw float bits, the constant
+//     exponent bits being removed once per word;
+//   * the sign bit "negative and level > 0" is the sign of fma(level, v, +0), shifted into the
+//     sign word with a funnel shift.
+// A generic kernel (any bucket size that is a multiple of 32) keeps the simple structure.
 #include <float.h>
 
 #include "qsgd_common.cuh"
@@ -17,24 +27,309 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kTile = 4096;           // coordinates per tile
-constexpr int kGroupsPerThread = kTile / 8 / kThreads;  // 2
-constexpr int kMaxBucketsPerTile = kTile / 32;          // 128
 
 struct QuantizeParams {
   const float* g;
   uint64_t n;
   uint32_t d;
   uint32_t s;
-  uint32_t tile_coords;   // coordinates per tile = whole buckets, <= kTile
+  uint32_t tile_coords;   // generic kernel: coordinates per tile = whole buckets, <= kTile
   uint32_t k0, k1, step, worker;
   float* A_out;
   uint32_t* sign_out;
   uint32_t* level_out;
   uint64_t B, sign_words, level_words;
+  uint64_t tiles;
+  uint32_t* status;
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX helpers: mbarrier and 1-D bulk copy global -> shared.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_u32(dst)),
+      "l"(src), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after ~2^22 polls and reports it instead of spinning forever.
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+  for (uint32_t it = 0; it < (1u << 22); ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+__device__ __forceinline__ float fma_rn(float a, float b, float c) {
+  float r;
+  asm("fma.rn.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10 with the round keys supplied as kernel-uniform values.
+// ---------------------------------------------------------------------------------------------
+struct RoundKeys { uint32_t k[10][2]; };
+
+__device__ __forceinline__ uint4 philox_rk(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                           const RoundKeys& rk) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
+    c0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk.k[r][0];
+    c1 = (uint32_t)p1;
+    c2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk.k[r][1];
+    c3 = (uint32_t)p0;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+constexpr float kTwo23 = 8388608.0f;
+constexpr uint32_t kTwo23Bits = 0x4B000000u;
+
+// One coordinate. Returns the raw bits of 2^23 + level (level clamped to s); pushes the sign
+// bit into `sw`.
+__device__ __forceinline__ uint32_t quantize_one(float v, float r, float sf, float cap, uint32_t rnd,
+                                                 uint32_t& sw) {
+  const float t = __fmul_rn(__fmul_rn(sf, fabsf(v)), r);
+  const float c = fma_rn(__uint2float_rn(rnd >> 8), 5.9604644775390625e-08f, t);
+  const float fl = fminf(__fadd_rd(c, kTwo23), cap);       // 2^23 + min(floor(c), s)
+  const float lf = __fsub_rn(fl, kTwo23);                   // the level as a float, exact
+  const float sv = fma_rn(lf, v, 0.0f);                     // sign set iff level > 0 and v < 0
+  sw = __funnelshift_l(__float_as_uint(sv), sw, 1);
+  return __float_as_uint(fl);
+}
+
+constexpr int kStages = 3;
+
+struct __align__(16) TileSmem {
+  float tile[kStages][kTile];
+  double wsum[2][kThreads / 32];
+  uint64_t full[kStages];
 };
 
 template <int LB, int NORM>
-__global__ void __launch_bounds__(kThreads) quantize_fixed_kernel(const QuantizeParams p) {
+__global__ void __launch_bounds__(kThreads, 3)
+quantize_pow2_kernel(const __grid_constant__ QuantizeParams p, const __grid_constant__ RoundKeys rk) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
+
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) mbar_init(&sm.full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const uint64_t full_tiles = p.n / kTile;            // tiles fetched by bulk copy
+  // prologue: fill the ring
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      const uint64_t t = (uint64_t)blockIdx.x + (uint64_t)s * gridDim.x;
+      if (t < full_tiles) {
+        mbar_expect_tx(&sm.full[s], kTile * 4);
+        bulk_load(sm.tile[s], p.g + t * kTile, kTile * 4, &sm.full[s]);
+      }
+    }
+  }
+
+  const float sf = (float)p.s;
+  const float cap = kTwo23 + sf;
+  const uint32_t team = p.d >> 4;                      // threads per bucket (2 .. 256)
+  const uint32_t team_w = team < 32 ? team : 32;       // shuffle width
+  const uint32_t warps_per_bucket = p.d >> 9;          // 0 when a bucket fits in a warp
+
+  uint32_t it = 0;
+  for (uint64_t t = blockIdx.x; t < p.tiles; t += gridDim.x, ++it) {
+    const uint32_t stage = it % kStages, parity = (it / kStages) & 1;
+    float* tile = sm.tile[stage];
+    uint32_t failed = 0;
+    if (t < full_tiles) {
+      if (!mbar_wait_bounded(&sm.full[stage], parity)) failed = 1;
+    } else {
+      // ragged last tile: plain loads, zero beyond n
+      const uint64_t t0 = t * kTile;
+      for (uint32_t i = tid; i < kTile; i += kThreads) tile[i] = (t0 + i < p.n) ? p.g[t0 + i] : 0.f;
+      __syncthreads();
+    }
+
+    // ---- registers <- 16 consecutive coordinates; partial of the scale ----------------------
+    float v[16];
+    if (!failed) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float4 a = *reinterpret_cast<const float4*>(tile + tid * 16 + j * 4);
+        v[4 * j] = a.x; v[4 * j + 1] = a.y; v[4 * j + 2] = a.z; v[4 * j + 3] = a.w;
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < 16; ++e) v[e] = 0.f;
+    }
+    float part = 0.f;
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      if (NORM == QSGD_NORM_L2) part = fmaf(v[e], v[e], part);
+      else part = fmaxf(part, fabsf(v[e]));
+    }
+    for (uint32_t o = team_w >> 1; o > 0; o >>= 1) {
+      const float q = __shfl_xor_sync(0xffffffffu, part, o);
+      part = (NORM == QSGD_NORM_L2) ? part + q : fmaxf(part, q);
+    }
+    // 2-norm: if the fp32 sum of squares may have lost bits to underflow or overflowed, redo
+    // this warp's share in fp64 (rare; whole warp takes the branch together)
+    double wide = (double)part;
+    if (NORM == QSGD_NORM_L2) {
+      const bool shaky = !(part >= 8.0e-28f && part <= 1.0e30f) && part != 0.f;
+      if (__any_sync(0xffffffffu, shaky)) {
+        double acc = 0.0;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc = fma((double)v[e], (double)v[e], acc);
+        for (uint32_t o = team_w >> 1; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        wide = acc;
+      }
+    }
+    if (warps_per_bucket > 1 && lane == 0) sm.wsum[it & 1][warp] = wide;
+
+    // ---- one CTA barrier per tile: every thread holds its values, the stage can be refilled --
+    if (__syncthreads_or((int)failed)) {
+      if (tid == 0) atomicOr(p.status, QSGD_DEV_TIMEOUT);
+      break;
+    }
+    if (tid == 0) {
+      const uint64_t tn = t + (uint64_t)kStages * gridDim.x;
+      if (tn < full_tiles) {
+        mbar_expect_tx(&sm.full[stage], kTile * 4);
+        bulk_load(tile, p.g + tn * kTile, kTile * 4, &sm.full[stage]);
+      }
+    }
+    if (warps_per_bucket > 1) {
+      const uint32_t w0 = warp & ~(warps_per_bucket - 1);
+      double acc = 0.0;
+      for (uint32_t w = 0; w < warps_per_bucket; ++w) {
+        const double q = sm.wsum[it & 1][w0 + w];
+        acc = (NORM == QSGD_NORM_L2) ? acc + q : fmax(acc, q);
+      }
+      wide = acc;
+    }
+    float A;
+    if (NORM == QSGD_NORM_L2) {
+      const float sum = (float)wide;
+      A = (wide == (double)part && sum >= 8.0e-28f) ? __fsqrt_rn(sum) : __double2float_rn(sqrt(wide));
+    } else {
+      A = (float)wide;
+    }
+    if (!(A >= FLT_MIN)) A = 0.f;                      // zero bucket: Q(0) = 0
+    const float r = A > 0.f ? __frcp_rn(A) : 0.f;
+    const uint64_t i0 = t * kTile + (uint64_t)tid * 16;   // global index of v[0]
+    if ((tid & (team - 1)) == 0) {
+      const uint64_t b = i0 / p.d;
+      if (b < p.B) p.A_out[b] = A;
+    }
+
+    // ---- stochastic rounding and packing, highest coordinate first --------------------------
+    const uint64_t q0 = i0 >> 2;
+    uint32_t sw = 0;
+    uint32_t lw[4] = {0u, 0u, 0u, 0u};                 // LB = 8: 4 words; 4: 2; 2: 1; 1: half
+#pragma unroll
+    for (int c4 = 3; c4 >= 0; --c4) {
+      const uint64_t q = q0 + c4;
+      const uint4 rnd = philox_rk((uint32_t)q, (uint32_t)(q >> 32), p.step, p.worker, rk);
+      const uint32_t rr[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
+#pragma unroll
+      for (int e = 3; e >= 0; --e) {
+        const uint32_t bits = quantize_one(v[4 * c4 + e], r, sf, cap, rr[e], sw);
+        if (LB == 8) lw[c4] = lw[c4] * 256u + bits;
+        else if (LB == 4) lw[c4 >> 1] = lw[c4 >> 1] * 16u + bits;
+        else if (LB == 2) lw[0] = lw[0] * 4u + bits;
+        else lw[0] = lw[0] * 2u + bits;
+      }
+    }
+    // remove the exponent bits that rode along: sum over the fields of 0x4B000000 << (LB * e)
+    if (LB == 8) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) lw[j] -= kTwo23Bits * 0x01010101u;
+    } else if (LB == 4) {
+      lw[0] -= kTwo23Bits * 0x11111111u;
+      lw[1] -= kTwo23Bits * 0x11111111u;
+    } else if (LB == 2) {
+      lw[0] -= kTwo23Bits * 0x55555555u;
+    } else {
+      lw[0] = (lw[0] - kTwo23Bits * 0xFFFFu) & 0xFFFFu;
+    }
+
+    // ---- stores -------------------------------------------------------------------------------
+    const uint64_t c0 = t * kTile;                     // first coordinate of the tile
+    {
+      uint32_t w = (sw & 0xFFFFu) << (16 * (lane & 1));
+      w |= __shfl_xor_sync(0xffffffffu, w, 1);
+      const uint64_t idx = (c0 >> 5) + (tid >> 1);
+      if ((lane & 1) == 0 && idx < p.sign_words) p.sign_out[idx] = w;
+    }
+    const uint64_t lpad = (p.level_words + 3) & ~3ull;
+    if (LB == 8) {
+      const uint64_t idx = (c0 >> 2) + (uint64_t)tid * 4;
+      if (idx < lpad) *reinterpret_cast<uint4*>(p.level_out + idx) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+    } else if (LB == 4) {
+      const uint64_t idx = (c0 >> 3) + (uint64_t)tid * 2;
+      if (idx < lpad) *reinterpret_cast<uint2*>(p.level_out + idx) = make_uint2(lw[0], lw[1]);
+    } else if (LB == 2) {
+      const uint64_t idx = (c0 >> 4) + tid;
+      if (idx < lpad) p.level_out[idx] = lw[0];
+    } else {
+      uint32_t w = lw[0] << (16 * (lane & 1));
+      w |= __shfl_xor_sync(0xffffffffu, w, 1);
+      const uint64_t idx = (c0 >> 5) + (tid >> 1);
+      if ((lane & 1) == 0 && idx < lpad) p.level_out[idx] = w;
+    }
+
+    // ---- zero the padding of the three regions (the CTA that owns the last tile) -----------
+    if (t == p.tiles - 1 && tid < 4) {
+      if (p.B + tid < ((p.B + 3) & ~3ull)) p.A_out[p.B + tid] = 0.f;
+      if (p.sign_words + tid < ((p.sign_words + 3) & ~3ull)) p.sign_out[p.sign_words + tid] = 0u;
+      if (p.level_words + tid < lpad) p.level_out[p.level_words + tid] = 0u;
+    }
+  }
+
+  // Leave no bulk copy in flight: a CTA that stops early waits (bounded) for its ring.
+  __syncthreads();
+  if (tid == 0) {
+    for (uint32_t j = 0; j < (uint32_t)kStages; ++j) {
+      const uint32_t itj = it + j;                                   // next uses of the ring
+      const uint64_t t = (uint64_t)blockIdx.x + (uint64_t)itj * gridDim.x;
+      if (t < full_tiles) mbar_wait_bounded(&sm.full[itj % kStages], (itj / kStages) & 1);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Generic kernel: any bucket size that is a multiple of 32. One CTA per tile of whole buckets.
+// ---------------------------------------------------------------------------------------------
+constexpr int kGroupsPerThread = kTile / 8 / kThreads;  // 2
+constexpr int kMaxBucketsPerTile = kTile / 32;          // 128
+
+template <int LB, int NORM>
+__global__ void __launch_bounds__(kThreads) quantize_generic_kernel(const QuantizeParams p) {
   __shared__ __align__(16) float tile[kTile];
   __shared__ float part[kTile / 8];
   __shared__ float s_rcp[kMaxBucketsPerTile];
@@ -44,7 +339,6 @@ __global__ void __launch_bounds__(kThreads) quantize_fixed_kernel(const Quantize
   const uint64_t left = p.n - t0;
   const uint32_t valid = left < p.tile_coords ? (uint32_t)left : p.tile_coords;
 
-  // ---- stage the tile (coalesced 16-byte loads; zero beyond n) -----------------------------
   for (uint32_t i = tid * 4; i < p.tile_coords; i += kThreads * 4) {
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     if (i + 4 <= valid) {
@@ -58,7 +352,6 @@ __global__ void __launch_bounds__(kThreads) quantize_fixed_kernel(const Quantize
   }
   __syncthreads();
 
-  // ---- per-group partial of the bucket scale; values stay in registers ---------------------
   float v[kGroupsPerThread][8];
   const uint32_t groups = p.tile_coords >> 3;
 #pragma unroll
@@ -81,15 +374,27 @@ __global__ void __launch_bounds__(kThreads) quantize_fixed_kernel(const Quantize
   }
   __syncthreads();
 
-  // ---- bucket scales: one warp per bucket, fp64 across the group partials ------------------
   const uint32_t nb = p.tile_coords / p.d;     // buckets in a full tile
   const uint32_t gpb = p.d >> 3;               // groups per bucket
   const uint64_t b0 = t0 / p.d;                // first bucket of the tile
   for (uint32_t b = warp; b < nb; b += kThreads / 32) {
     float A;
     if (NORM == QSGD_NORM_L2) {
+      // fp32 partials of 8 squares each; redo in fp64 from the tile when they may have lost bits
       double acc = 0.0;
-      for (uint32_t j = lane; j < gpb; j += 32) acc += (double)part[b * gpb + j];
+      bool shaky = false;
+      for (uint32_t j = lane; j < gpb; j += 32) {
+        const float q = part[b * gpb + j];
+        shaky |= !(q >= 8.0e-28f && q <= 1.0e30f) && q != 0.f;
+        acc += (double)q;
+      }
+      if (__any_sync(0xffffffffu, shaky)) {
+        acc = 0.0;
+        for (uint32_t i = lane; i < p.d; i += 32) {
+          const double x = (double)tile[b * p.d + i];
+          acc = fma(x, x, acc);
+        }
+      }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
       A = __double2float_rn(__dsqrt_rn(acc));
@@ -100,7 +405,7 @@ __global__ void __launch_bounds__(kThreads) quantize_fixed_kernel(const Quantize
       for (int o = 16; o > 0; o >>= 1) acc = fmaxf(acc, __shfl_xor_sync(0xffffffffu, acc, o));
       A = acc;
     }
-    if (!(A >= FLT_MIN)) A = 0.f;              // zero bucket: Q(0) = 0
+    if (!(A >= FLT_MIN)) A = 0.f;
     if (lane == 0) {
       s_rcp[b] = A > 0.f ? __frcp_rn(A) : 0.f;
       if (b0 + b < p.B) p.A_out[b0 + b] = A;
@@ -108,14 +413,13 @@ __global__ void __launch_bounds__(kThreads) quantize_fixed_kernel(const Quantize
   }
   __syncthreads();
 
-  // ---- stochastic rounding and packing -----------------------------------------------------
   const float sf = (float)p.s;
 #pragma unroll
   for (int j = 0; j < kGroupsPerThread; ++j) {
     const uint32_t grp = tid + j * kThreads;
     const uint32_t bl = (grp * 8) / p.d;
     const float r = (grp < groups) ? s_rcp[bl] : 0.f;
-    const uint64_t i0 = t0 + (uint64_t)grp * 8;       // global index of the group's first value
+    const uint64_t i0 = t0 + (uint64_t)grp * 8;
     const uint64_t q = i0 >> 2;
     const uint4 ra = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), p.step, p.worker, p.k0, p.k1);
     const uint4 rb = philox4x32_10((uint32_t)(q + 1), (uint32_t)((q + 1) >> 32), p.step, p.worker,
@@ -128,7 +432,6 @@ __global__ void __launch_bounds__(kThreads) quantize_fixed_kernel(const Quantize
       lv[e] = quantize_level(v[j][e], r, sf, p.s, rnd[e]);
       sb |= (uint32_t)(lv[e] != 0 && v[j][e] < 0.f) << e;
     }
-    // sign bitmap: 4 lanes -> one word
     uint32_t sw = sb << (8 * (lane & 3));
     sw |= __shfl_xor_sync(0xffffffffu, sw, 1);
     sw |= __shfl_xor_sync(0xffffffffu, sw, 2);
@@ -169,7 +472,6 @@ __global__ void __launch_bounds__(kThreads) quantize_fixed_kernel(const Quantize
     }
   }
 
-  // ---- zero the padding of the three regions (last CTA) ------------------------------------
   if (blockIdx.x == gridDim.x - 1 && tid < 4) {
     if (p.B + tid < ((p.B + 3) & ~3ull)) p.A_out[p.B + tid] = 0.f;
     if (p.sign_words + tid < ((p.sign_words + 3) & ~3ull)) p.sign_out[p.sign_words + tid] = 0u;
@@ -177,37 +479,73 @@ __global__ void __launch_bounds__(kThreads) quantize_fixed_kernel(const Quantize
   }
 }
 
-template <int LB>
-int launch_lb(const QuantizeParams& p, int norm_kind, uint32_t grid, cudaStream_t stream) {
-  {
+RoundKeys make_round_keys(uint64_t seed) {
+  RoundKeys rk;
+  uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
+  for (int r = 0; r < 10; ++r) {
+    rk.k[r][0] = k0; rk.k[r][1] = k1;
+    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+  }
+  return rk;
+}
+
+template <int LB, int NORM>
+int launch_one(const QuantizeParams& p, bool pow2, uint64_t seed, cudaStream_t stream) {
+  if (pow2) {
+    static int ctas_per_sm = 0, sms = 0;
+    auto kern = quantize_pow2_kernel<LB, NORM>;
+    const size_t smem = sizeof(TileSmem) + 128;
+    if (ctas_per_sm == 0) {
+      int dev = 0;
+      cudaGetDevice(&dev);
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return (int)e;
+      int occ = 0;
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, smem);
+      if (e != cudaSuccess) return (int)e;
+      ctas_per_sm = occ > 0 ? occ : 1;
+    }
+    const uint64_t cap = (uint64_t)sms * ctas_per_sm;
+    const uint32_t grid = (uint32_t)(p.tiles < cap ? p.tiles : cap);
+    const RoundKeys rk = make_round_keys(seed);
     ScopedKernel sk(kKernQuantize, stream);
-    if (norm_kind == QSGD_NORM_L2) quantize_fixed_kernel<LB, QSGD_NORM_L2><<<grid, kThreads, 0, stream>>>(p);
-    else quantize_fixed_kernel<LB, QSGD_NORM_MAX><<<grid, kThreads, 0, stream>>>(p);
+    kern<<<grid, kThreads, smem, stream>>>(p, rk);
+  } else {
+    ScopedKernel sk(kKernQuantize, stream);
+    quantize_generic_kernel<LB, NORM><<<(uint32_t)p.tiles, kThreads, 0, stream>>>(p);
   }
   return (int)cudaGetLastError();
+}
+
+template <int LB>
+int launch_lb(const QuantizeParams& p, int norm_kind, bool pow2, uint64_t seed, cudaStream_t stream) {
+  return norm_kind == QSGD_NORM_L2 ? launch_one<LB, QSGD_NORM_L2>(p, pow2, seed, stream)
+                                   : launch_one<LB, QSGD_NORM_MAX>(p, pow2, seed, stream);
 }
 
 }  // namespace
 
 int launch_quantize_fixed(const float* g, uint64_t n, uint32_t d, uint32_t s, int norm_kind,
                           uint64_t seed, uint32_t step, uint32_t worker, uint8_t* out,
-                          cudaStream_t stream) {
+                          uint32_t* status_dev, cudaStream_t stream) {
   const FixedLayout L = make_fixed_layout(n, d, s);
+  const bool pow2 = (d & (d - 1)) == 0;
   QuantizeParams p;
   p.g = g; p.n = n; p.d = d; p.s = s;
-  p.tile_coords = (kTile / d) * d;
+  p.tile_coords = pow2 ? kTile : (kTile / d) * d;
   p.k0 = (uint32_t)seed; p.k1 = (uint32_t)(seed >> 32); p.step = step; p.worker = worker;
   p.A_out = reinterpret_cast<float*>(out);
   p.sign_out = reinterpret_cast<uint32_t*>(out + L.off_sign);
   p.level_out = reinterpret_cast<uint32_t*>(out + L.off_level);
   p.B = L.B; p.sign_words = L.sign_words; p.level_words = L.level_words;
-  const uint64_t tiles = (n + p.tile_coords - 1) / p.tile_coords;
-  const uint32_t grid = (uint32_t)tiles;
+  p.tiles = (n + p.tile_coords - 1) / p.tile_coords;
+  p.status = status_dev;
   switch (L.lb) {
-    case 1: return launch_lb<1>(p, norm_kind, grid, stream);
-    case 2: return launch_lb<2>(p, norm_kind, grid, stream);
-    case 4: return launch_lb<4>(p, norm_kind, grid, stream);
-    default: return launch_lb<8>(p, norm_kind, grid, stream);
+    case 1: return launch_lb<1>(p, norm_kind, pow2, seed, stream);
+    case 2: return launch_lb<2>(p, norm_kind, pow2, seed, stream);
+    case 4: return launch_lb<4>(p, norm_kind, pow2, seed, stream);
+    default: return launch_lb<8>(p, norm_kind, pow2, seed, stream);
   }
 }
 
