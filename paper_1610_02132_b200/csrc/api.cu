@@ -33,7 +33,7 @@ ScopedKernel::~ScopedKernel() {
 }
 
 static const char* const kKernelNames[kKernCount] = {
-    "quantize_fixed", "fixed_info", "decode_fixed", "sgd_step", "elias_length",
+    "quantize_fixed", "quantize_tail", "fixed_info", "decode_fixed", "sgd_step", "elias_length",
     "scan_block_sums", "scan_sums", "scan_downsweep", "zero_payload", "elias_scatter",
     "decode_elias"};
 

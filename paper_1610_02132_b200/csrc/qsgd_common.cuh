@@ -117,7 +117,7 @@ int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d
 // timing is switched on (qsgd_profile_enable), records a CUDA event before and after it on the
 // launching stream.
 enum KernelId {
-  kKernQuantize = 0, kKernFixedInfo, kKernDecodeFixed, kKernSgdStep, kKernEliasLength,
+  kKernQuantize = 0, kKernQuantizeTail, kKernFixedInfo, kKernDecodeFixed, kKernSgdStep, kKernEliasLength,
   kKernScanBlockSums, kKernScanSums, kKernScanDownsweep, kKernZeroPayload, kKernEliasScatter,
   kKernDecodeElias, kKernCount
 };

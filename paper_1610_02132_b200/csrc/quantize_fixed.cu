@@ -34,6 +34,7 @@ struct QuantizeParams {
   uint32_t d;
   uint32_t s;
   uint32_t tile_coords;   // generic kernel: coordinates per tile = whole buckets, <= kTile
+  uint64_t coord_base;    // generic kernel: first coordinate it is responsible for
   uint32_t k0, k1, step, worker;
   float* A_out;
   uint32_t* sign_out;
@@ -80,6 +81,9 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ float fma_rn(float a, float b, float c) {
   float r;
   asm("fma.rn.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
@@ -87,19 +91,43 @@ __device__ __forceinline__ float fma_rn(float a, float b, float c) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Philox4x32-10 with the round keys supplied as kernel-uniform values.
+// Philox4x32-10 for the counter (q, 0, step, worker) with everything that does not depend on q
+// folded into kernel-uniform constants on the host: after round 0 two of the four words are
+// constants, which also makes one product of round 1 a constant. 37 instead of 40
+// multiply / xor instructions per block of four uniforms.
 // ---------------------------------------------------------------------------------------------
-struct RoundKeys { uint32_t k[10][2]; };
+struct PhiloxConsts {
+  uint32_t y0;        // worker ^ k1[0]
+  uint32_t z0;        // lo(M1 * step) ^ k0[1]
+  uint32_t z1;        // hi(M0 * x0) ^ k1[1],  x0 = hi(M1 * step) ^ k0[0]
+  uint32_t z2;        // lo(M0 * x0) ^ k1[2]
+  uint32_t k0_2;      // k0[2]
+  uint32_t k[7][2];   // round keys 3 .. 9
+};
 
-__device__ __forceinline__ uint4 philox_rk(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                           const RoundKeys& rk) {
+constexpr uint32_t kM0 = 0xD2511F53u, kM1 = 0xCD9E8D57u;
+
+__device__ __forceinline__ uint4 philox_q(uint32_t q, const PhiloxConsts& pc) {
+  // round 0: (q, 0, step, worker) -> (x0, l1, hi(M0 q) ^ y0, lo(M0 q))
+  uint64_t p0 = (uint64_t)kM0 * q;
+  uint32_t a2 = (uint32_t)(p0 >> 32) ^ pc.y0, a3 = (uint32_t)p0;
+  // round 1: (x0, l1, a2, a3) -> (hi(M1 a2) ^ z0, lo(M1 a2), a3 ^ z1, lo(M0 x0))
+  uint64_t p1 = (uint64_t)kM1 * a2;
+  uint32_t c0 = (uint32_t)(p1 >> 32) ^ pc.z0, c1 = (uint32_t)p1, c2 = a3 ^ pc.z1;
+  // round 2: c3 = lo(M0 x0) is folded into z2
+  p0 = (uint64_t)kM0 * c0;
+  p1 = (uint64_t)kM1 * c2;
+  c0 = (uint32_t)(p1 >> 32) ^ c1 ^ pc.k0_2;
+  c1 = (uint32_t)p1;
+  c2 = (uint32_t)(p0 >> 32) ^ pc.z2;
+  uint32_t c3 = (uint32_t)p0;
 #pragma unroll
-  for (int r = 0; r < 10; ++r) {
-    const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
-    const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
-    c0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk.k[r][0];
+  for (int r = 0; r < 7; ++r) {
+    p0 = (uint64_t)kM0 * c0;
+    p1 = (uint64_t)kM1 * c2;
+    c0 = (uint32_t)(p1 >> 32) ^ c1 ^ pc.k[r][0];
     c1 = (uint32_t)p1;
-    c2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk.k[r][1];
+    c2 = (uint32_t)(p0 >> 32) ^ c3 ^ pc.k[r][1];
     c3 = (uint32_t)p0;
   }
   return make_uint4(c0, c1, c2, c3);
@@ -113,7 +141,8 @@ constexpr uint32_t kTwo23Bits = 0x4B000000u;
 __device__ __forceinline__ uint32_t quantize_one(float v, float r, float sf, float cap, uint32_t rnd,
                                                  uint32_t& sw) {
   const float t = __fmul_rn(__fmul_rn(sf, fabsf(v)), r);
-  const float c = fma_rn(__uint2float_rn(rnd >> 8), 5.9604644775390625e-08f, t);
+  // rnd >> 8 as a multiply-high keeps the shift off the (busier) integer/logic pipe
+  const float c = fma_rn(__uint2float_rn(__umulhi(rnd, 1u << 24)), 5.9604644775390625e-08f, t);
   const float fl = fminf(__fadd_rd(c, kTwo23), cap);       // 2^23 + min(floor(c), s)
   const float lf = __fsub_rn(fl, kTwo23);                   // the level as a float, exact
   const float sv = fma_rn(lf, v, 0.0f);                     // sign set iff level > 0 and v < 0
@@ -125,66 +154,70 @@ constexpr int kStages = 3;
 
 struct __align__(16) TileSmem {
   float tile[kStages][kTile];
-  double wsum[2][kThreads / 32];
-  uint64_t full[kStages];
+  float wsum[2][kThreads / 32];
+  double wsum64[kThreads / 32];
+  uint64_t full[kStages];    // bulk copy landed
+  uint64_t empty[kStages];   // all warps have taken their values out of the stage
 };
 
-template <int LB, int NORM>
-__global__ void __launch_bounds__(kThreads, 3)
-quantize_pow2_kernel(const __grid_constant__ QuantizeParams p, const __grid_constant__ RoundKeys rk) {
+struct FastParams {
+  const float* g;
+  uint32_t full_tiles;      // tiles of 4096 coordinates, all complete
+  uint32_t log2d;           // bucket size 2^log2d, 5 .. 12
+  uint32_t s;
+  float* A_out;
+  uint32_t* sign_out;
+  uint32_t* level_out;
+  uint32_t* status;
+  PhiloxConsts pc;
+};
+
+// CROSS: a bucket spans several warps (d >= 1024); otherwise a bucket is d / 16 <= 32 lanes.
+template <int LB, int NORM, bool CROSS>
+__global__ void __launch_bounds__(kThreads, 4)
+quantize_pow2_kernel(const __grid_constant__ FastParams p) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
 
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t grid = gridDim.x;
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) mbar_init(&sm.full[s], 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sm.full[s], 1);
+      mbar_init(&sm.empty[s], kThreads / 32);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-
-  const uint64_t full_tiles = p.n / kTile;            // tiles fetched by bulk copy
-  // prologue: fill the ring
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
-      const uint64_t t = (uint64_t)blockIdx.x + (uint64_t)s * gridDim.x;
-      if (t < full_tiles) {
+      const uint32_t t = blockIdx.x + (uint32_t)s * grid;
+      if (t < p.full_tiles) {
         mbar_expect_tx(&sm.full[s], kTile * 4);
-        bulk_load(sm.tile[s], p.g + t * kTile, kTile * 4, &sm.full[s]);
+        bulk_load(sm.tile[s], p.g + (size_t)t * kTile, kTile * 4, &sm.full[s]);
       }
     }
   }
 
   const float sf = (float)p.s;
   const float cap = kTwo23 + sf;
-  const uint32_t team = p.d >> 4;                      // threads per bucket (2 .. 256)
-  const uint32_t team_w = team < 32 ? team : 32;       // shuffle width
-  const uint32_t warps_per_bucket = p.d >> 9;          // 0 when a bucket fits in a warp
+  const uint32_t team_w = CROSS ? 32u : (1u << (p.log2d - 4));   // lanes per bucket (<= 32)
+  const uint32_t wpb = CROSS ? (1u << (p.log2d - 9)) : 1u;       // warps per bucket
+  const bool leader = CROSS ? ((tid & (32u * wpb - 1u)) == 0) : ((lane & (team_w - 1u)) == 0);
+  const uint32_t my_bucket = (tid * 16u) >> p.log2d;             // bucket of this thread in a tile
+  const uint32_t buckets_per_tile_log2 = 12u - p.log2d;
 
-  uint32_t it = 0;
-  for (uint64_t t = blockIdx.x; t < p.tiles; t += gridDim.x, ++it) {
-    const uint32_t stage = it % kStages, parity = (it / kStages) & 1;
-    float* tile = sm.tile[stage];
-    uint32_t failed = 0;
-    if (t < full_tiles) {
-      if (!mbar_wait_bounded(&sm.full[stage], parity)) failed = 1;
-    } else {
-      // ragged last tile: plain loads, zero beyond n
-      const uint64_t t0 = t * kTile;
-      for (uint32_t i = tid; i < kTile; i += kThreads) tile[i] = (t0 + i < p.n) ? p.g[t0 + i] : 0.f;
-      __syncthreads();
-    }
+  uint32_t stage = 0, phase = 0, it = 0;
+  for (uint32_t t = blockIdx.x; t < p.full_tiles; t += grid, ++it) {
+    const float* tile = sm.tile[stage];
+    const bool arrived = mbar_wait_bounded(&sm.full[stage], phase);
 
     // ---- registers <- 16 consecutive coordinates; partial of the scale ----------------------
     float v[16];
-    if (!failed) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float4 a = *reinterpret_cast<const float4*>(tile + tid * 16 + j * 4);
-        v[4 * j] = a.x; v[4 * j + 1] = a.y; v[4 * j + 2] = a.z; v[4 * j + 3] = a.w;
-      }
-    } else {
-#pragma unroll
-      for (int e = 0; e < 16; ++e) v[e] = 0.f;
+    for (int j = 0; j < 4; ++j) {
+      const float4 a = *reinterpret_cast<const float4*>(tile + tid * 16 + j * 4);
+      v[4 * j] = a.x; v[4 * j + 1] = a.y; v[4 * j + 2] = a.z; v[4 * j + 3] = a.w;
     }
     float part = 0.f;
 #pragma unroll
@@ -192,69 +225,94 @@ quantize_pow2_kernel(const __grid_constant__ QuantizeParams p, const __grid_cons
       if (NORM == QSGD_NORM_L2) part = fmaf(v[e], v[e], part);
       else part = fmaxf(part, fabsf(v[e]));
     }
-    for (uint32_t o = team_w >> 1; o > 0; o >>= 1) {
-      const float q = __shfl_xor_sync(0xffffffffu, part, o);
-      part = (NORM == QSGD_NORM_L2) ? part + q : fmaxf(part, q);
-    }
-    // 2-norm: if the fp32 sum of squares may have lost bits to underflow or overflowed, redo
-    // this warp's share in fp64 (rare; whole warp takes the branch together)
-    double wide = (double)part;
-    if (NORM == QSGD_NORM_L2) {
-      const bool shaky = !(part >= 8.0e-28f && part <= 1.0e30f) && part != 0.f;
-      if (__any_sync(0xffffffffu, shaky)) {
-        double acc = 0.0;
 #pragma unroll
-        for (int e = 0; e < 16; ++e) acc = fma((double)v[e], (double)v[e], acc);
-        for (uint32_t o = team_w >> 1; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        wide = acc;
-      }
+    for (uint32_t o = 16; o > 0; o >>= 1) {
+      const float q = __shfl_xor_sync(0xffffffffu, part, o);
+      const float merged = (NORM == QSGD_NORM_L2) ? part + q : fmaxf(part, q);
+      part = (o < team_w) ? merged : part;
     }
-    if (warps_per_bucket > 1 && lane == 0) sm.wsum[it & 1][warp] = wide;
+    // 2-norm: an fp32 sum of squares outside [8e-28, 1e30] may have lost bits to underflow or
+    // overflowed; such buckets are redone in fp64 (rare, the warp / CTA branches together)
+    bool shaky = false;
+    if (NORM == QSGD_NORM_L2) shaky = !(part >= 8.0e-28f && part <= 1.0e30f) && part != 0.f;
+    if (CROSS && lane == 0) sm.wsum[it & 1][warp] = part;
 
-    // ---- one CTA barrier per tile: every thread holds its values, the stage can be refilled --
-    if (__syncthreads_or((int)failed)) {
-      if (tid == 0) atomicOr(p.status, QSGD_DEV_TIMEOUT);
+    // ---- release the stage: every warp signals that its values are in registers; the producer
+    // thread refills the stage that was released one iteration ago (its arrivals are long in) ----
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.empty[stage]);
+    int flags = arrived ? 0 : 1;
+    if (CROSS) flags = __syncthreads_or(flags | (shaky ? 2 : 0));
+    if (flags & 1) {
+      atomicOr(p.status, QSGD_DEV_TIMEOUT);
       break;
     }
-    if (tid == 0) {
-      const uint64_t tn = t + (uint64_t)kStages * gridDim.x;
-      if (tn < full_tiles) {
-        mbar_expect_tx(&sm.full[stage], kTile * 4);
-        bulk_load(tile, p.g + tn * kTile, kTile * 4, &sm.full[stage]);
+    if (tid == 0 && it > 0) {
+      const uint32_t ps = stage == 0 ? kStages - 1 : stage - 1;           // stage of iteration it - 1
+      const uint32_t pphase = stage == 0 ? phase ^ 1 : phase;
+      const uint32_t tn = t + (uint32_t)(kStages - 1) * grid;             // tile of iteration it - 1 + kStages
+      if (tn < p.full_tiles) {
+        if (mbar_wait_bounded(&sm.empty[ps], pphase)) {
+          mbar_expect_tx(&sm.full[ps], kTile * 4);
+          bulk_load(sm.tile[ps], p.g + (size_t)tn * kTile, kTile * 4, &sm.full[ps]);
+        } else {
+          atomicOr(p.status, QSGD_DEV_TIMEOUT);
+        }
       }
-    }
-    if (warps_per_bucket > 1) {
-      const uint32_t w0 = warp & ~(warps_per_bucket - 1);
-      double acc = 0.0;
-      for (uint32_t w = 0; w < warps_per_bucket; ++w) {
-        const double q = sm.wsum[it & 1][w0 + w];
-        acc = (NORM == QSGD_NORM_L2) ? acc + q : fmax(acc, q);
-      }
-      wide = acc;
     }
     float A;
-    if (NORM == QSGD_NORM_L2) {
-      const float sum = (float)wide;
-      A = (wide == (double)part && sum >= 8.0e-28f) ? __fsqrt_rn(sum) : __double2float_rn(sqrt(wide));
+    if (CROSS) {
+      const uint32_t w0 = warp & ~(wpb - 1u);
+      float acc = 0.f;
+      for (uint32_t w = 0; w < wpb; ++w) {
+        const float q = sm.wsum[it & 1][w0 + w];
+        acc = (NORM == QSGD_NORM_L2) ? acc + q : fmaxf(acc, q);
+      }
+      if (NORM == QSGD_NORM_L2) {
+        A = __fsqrt_rn(acc);
+        if (flags & 2) {                      // some bucket of this tile needs the fp64 path
+          double wide = 0.0;
+#pragma unroll
+          for (int e = 0; e < 16; ++e) wide = fma((double)v[e], (double)v[e], wide);
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) wide += __shfl_xor_sync(0xffffffffu, wide, o);
+          if (lane == 0) sm.wsum64[warp] = wide;
+          __syncthreads();
+          wide = 0.0;
+          for (uint32_t w = 0; w < wpb; ++w) wide += sm.wsum64[w0 + w];
+          A = __double2float_rn(sqrt(wide));
+          __syncthreads();
+        }
+      } else {
+        A = acc;
+      }
+    } else if (NORM == QSGD_NORM_L2) {
+      A = __fsqrt_rn(part);
+      if (__any_sync(0xffffffffu, shaky)) {
+        double wide = 0.0;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) wide = fma((double)v[e], (double)v[e], wide);
+#pragma unroll
+        for (uint32_t o = 16; o > 0; o >>= 1) {
+          const double q = __shfl_xor_sync(0xffffffffu, wide, o);
+          wide = (o < team_w) ? wide + q : wide;
+        }
+        if (shaky) A = __double2float_rn(sqrt(wide));
+      }
     } else {
-      A = (float)wide;
+      A = part;
     }
     if (!(A >= FLT_MIN)) A = 0.f;                      // zero bucket: Q(0) = 0
     const float r = A > 0.f ? __frcp_rn(A) : 0.f;
-    const uint64_t i0 = t * kTile + (uint64_t)tid * 16;   // global index of v[0]
-    if ((tid & (team - 1)) == 0) {
-      const uint64_t b = i0 / p.d;
-      if (b < p.B) p.A_out[b] = A;
-    }
+    if (leader) p.A_out[(t << buckets_per_tile_log2) + my_bucket] = A;
 
     // ---- stochastic rounding and packing, highest coordinate first --------------------------
-    const uint64_t q0 = i0 >> 2;
+    const uint32_t q0 = t * (kTile / 4) + tid * 4;     // Philox block of v[0..3]
     uint32_t sw = 0;
     uint32_t lw[4] = {0u, 0u, 0u, 0u};                 // LB = 8: 4 words; 4: 2; 2: 1; 1: half
 #pragma unroll
     for (int c4 = 3; c4 >= 0; --c4) {
-      const uint64_t q = q0 + c4;
-      const uint4 rnd = philox_rk((uint32_t)q, (uint32_t)(q >> 32), p.step, p.worker, rk);
+      const uint4 rnd = philox_q(q0 + c4, p.pc);
       const uint32_t rr[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
 #pragma unroll
       for (int e = 3; e >= 0; --e) {
@@ -278,46 +336,34 @@ quantize_pow2_kernel(const __grid_constant__ QuantizeParams p, const __grid_cons
       lw[0] = (lw[0] - kTwo23Bits * 0xFFFFu) & 0xFFFFu;
     }
 
-    // ---- stores -------------------------------------------------------------------------------
-    const uint64_t c0 = t * kTile;                     // first coordinate of the tile
+    // ---- stores (full tiles only: no bounds to check) -----------------------------------------
     {
       uint32_t w = (sw & 0xFFFFu) << (16 * (lane & 1));
       w |= __shfl_xor_sync(0xffffffffu, w, 1);
-      const uint64_t idx = (c0 >> 5) + (tid >> 1);
-      if ((lane & 1) == 0 && idx < p.sign_words) p.sign_out[idx] = w;
+      if ((lane & 1) == 0) p.sign_out[t * (kTile / 32) + (tid >> 1)] = w;
     }
-    const uint64_t lpad = (p.level_words + 3) & ~3ull;
     if (LB == 8) {
-      const uint64_t idx = (c0 >> 2) + (uint64_t)tid * 4;
-      if (idx < lpad) *reinterpret_cast<uint4*>(p.level_out + idx) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+      *reinterpret_cast<uint4*>(p.level_out + (size_t)(t * (kTile / 4) + tid * 4)) =
+          make_uint4(lw[0], lw[1], lw[2], lw[3]);
     } else if (LB == 4) {
-      const uint64_t idx = (c0 >> 3) + (uint64_t)tid * 2;
-      if (idx < lpad) *reinterpret_cast<uint2*>(p.level_out + idx) = make_uint2(lw[0], lw[1]);
+      *reinterpret_cast<uint2*>(p.level_out + (size_t)(t * (kTile / 8) + tid * 2)) = make_uint2(lw[0], lw[1]);
     } else if (LB == 2) {
-      const uint64_t idx = (c0 >> 4) + tid;
-      if (idx < lpad) p.level_out[idx] = lw[0];
+      p.level_out[t * (kTile / 16) + tid] = lw[0];
     } else {
       uint32_t w = lw[0] << (16 * (lane & 1));
       w |= __shfl_xor_sync(0xffffffffu, w, 1);
-      const uint64_t idx = (c0 >> 5) + (tid >> 1);
-      if ((lane & 1) == 0 && idx < lpad) p.level_out[idx] = w;
+      if ((lane & 1) == 0) p.level_out[t * (kTile / 32) + (tid >> 1)] = w;
     }
-
-    // ---- zero the padding of the three regions (the CTA that owns the last tile) -----------
-    if (t == p.tiles - 1 && tid < 4) {
-      if (p.B + tid < ((p.B + 3) & ~3ull)) p.A_out[p.B + tid] = 0.f;
-      if (p.sign_words + tid < ((p.sign_words + 3) & ~3ull)) p.sign_out[p.sign_words + tid] = 0u;
-      if (p.level_words + tid < lpad) p.level_out[p.level_words + tid] = 0u;
-    }
+    if (++stage == kStages) { stage = 0; phase ^= 1; }
   }
 
-  // Leave no bulk copy in flight: a CTA that stops early waits (bounded) for its ring.
+  // Leave no bulk copy in flight: a CTA that stopped early waits (bounded) for its ring.
   __syncthreads();
   if (tid == 0) {
     for (uint32_t j = 0; j < (uint32_t)kStages; ++j) {
-      const uint32_t itj = it + j;                                   // next uses of the ring
-      const uint64_t t = (uint64_t)blockIdx.x + (uint64_t)itj * gridDim.x;
-      if (t < full_tiles) mbar_wait_bounded(&sm.full[itj % kStages], (itj / kStages) & 1);
+      const uint32_t itj = it + j;
+      const uint64_t t = (uint64_t)blockIdx.x + (uint64_t)itj * grid;
+      if (t < p.full_tiles) mbar_wait_bounded(&sm.full[itj % kStages], (itj / kStages) & 1);
     }
   }
 }
@@ -335,9 +381,17 @@ __global__ void __launch_bounds__(kThreads) quantize_generic_kernel(const Quanti
   __shared__ float s_rcp[kMaxBucketsPerTile];
 
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint64_t t0 = (uint64_t)blockIdx.x * p.tile_coords;   // first coordinate of the tile
+  const uint64_t t0 = p.coord_base + (uint64_t)blockIdx.x * p.tile_coords;   // first coordinate
   const uint64_t left = p.n - t0;
   const uint32_t valid = left < p.tile_coords ? (uint32_t)left : p.tile_coords;
+  if (valid == 0) {                            // nothing left to encode: only the padding
+    if (tid < 4) {
+      if (p.B + tid < ((p.B + 3) & ~3ull)) p.A_out[p.B + tid] = 0.f;
+      if (p.sign_words + tid < ((p.sign_words + 3) & ~3ull)) p.sign_out[p.sign_words + tid] = 0u;
+      if (p.level_words + tid < ((p.level_words + 3) & ~3ull)) p.level_out[p.level_words + tid] = 0u;
+    }
+    return;
+  }
 
   for (uint32_t i = tid * 4; i < p.tile_coords; i += kThreads * 4) {
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -479,49 +533,79 @@ __global__ void __launch_bounds__(kThreads) quantize_generic_kernel(const Quanti
   }
 }
 
-RoundKeys make_round_keys(uint64_t seed) {
-  RoundKeys rk;
-  uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
-  for (int r = 0; r < 10; ++r) {
-    rk.k[r][0] = k0; rk.k[r][1] = k1;
-    k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+PhiloxConsts make_philox_consts(uint64_t seed, uint32_t step, uint32_t worker) {
+  uint32_t k0[10], k1[10];
+  k0[0] = (uint32_t)seed; k1[0] = (uint32_t)(seed >> 32);
+  for (int r = 1; r < 10; ++r) { k0[r] = k0[r - 1] + 0x9E3779B9u; k1[r] = k1[r - 1] + 0xBB67AE85u; }
+  const uint64_t ps = (uint64_t)kM1 * step;
+  const uint32_t x0 = (uint32_t)(ps >> 32) ^ k0[0], l1 = (uint32_t)ps;
+  const uint64_t px = (uint64_t)kM0 * x0;
+  PhiloxConsts pc;
+  pc.y0 = worker ^ k1[0];
+  pc.z0 = l1 ^ k0[1];
+  pc.z1 = (uint32_t)(px >> 32) ^ k1[1];
+  pc.z2 = (uint32_t)px ^ k1[2];
+  pc.k0_2 = k0[2];
+  for (int r = 0; r < 7; ++r) { pc.k[r][0] = k0[r + 3]; pc.k[r][1] = k1[r + 3]; }
+  return pc;
+}
+
+template <int LB, int NORM, bool CROSS>
+int launch_fast(const FastParams& fp, cudaStream_t stream) {
+  static int ctas_per_sm = 0, sms = 0;
+  auto kern = quantize_pow2_kernel<LB, NORM, CROSS>;
+  const size_t smem = sizeof(TileSmem) + 128;
+  if (ctas_per_sm == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return (int)e;
+    int occ = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, smem);
+    if (e != cudaSuccess) return (int)e;
+    ctas_per_sm = occ > 0 ? occ : 1;
   }
-  return rk;
+  const uint32_t cap = (uint32_t)(sms * ctas_per_sm);
+  const uint32_t grid = fp.full_tiles < cap ? fp.full_tiles : cap;
+  ScopedKernel sk(kKernQuantize, stream);
+  kern<<<grid, kThreads, smem, stream>>>(fp);
+  return (int)cudaGetLastError();
 }
 
 template <int LB, int NORM>
-int launch_one(const QuantizeParams& p, bool pow2, uint64_t seed, cudaStream_t stream) {
-  if (pow2) {
-    static int ctas_per_sm = 0, sms = 0;
-    auto kern = quantize_pow2_kernel<LB, NORM>;
-    const size_t smem = sizeof(TileSmem) + 128;
-    if (ctas_per_sm == 0) {
-      int dev = 0;
-      cudaGetDevice(&dev);
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return (int)e;
-      int occ = 0;
-      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, smem);
-      if (e != cudaSuccess) return (int)e;
-      ctas_per_sm = occ > 0 ? occ : 1;
-    }
-    const uint64_t cap = (uint64_t)sms * ctas_per_sm;
-    const uint32_t grid = (uint32_t)(p.tiles < cap ? p.tiles : cap);
-    const RoundKeys rk = make_round_keys(seed);
-    ScopedKernel sk(kKernQuantize, stream);
-    kern<<<grid, kThreads, smem, stream>>>(p, rk);
-  } else {
-    ScopedKernel sk(kKernQuantize, stream);
-    quantize_generic_kernel<LB, NORM><<<(uint32_t)p.tiles, kThreads, 0, stream>>>(p);
+int launch_one(QuantizeParams& p, uint64_t seed, cudaStream_t stream) {
+  const uint32_t d = p.d;
+  const bool pow2 = (d & (d - 1)) == 0;
+  uint32_t full_tiles = 0;
+  if (pow2 && p.n <= (1ull << 32)) full_tiles = (uint32_t)(p.n / kTile);
+  if (full_tiles > 0) {
+    FastParams fp;
+    fp.g = p.g; fp.full_tiles = full_tiles; fp.s = p.s;
+    fp.log2d = 0;
+    while ((1u << fp.log2d) < d) ++fp.log2d;
+    fp.A_out = p.A_out; fp.sign_out = p.sign_out; fp.level_out = p.level_out; fp.status = p.status;
+    fp.pc = make_philox_consts(seed, p.step, p.worker);
+    const int st = d >= 1024 ? launch_fast<LB, NORM, true>(fp, stream) : launch_fast<LB, NORM, false>(fp, stream);
+    if (st) return st;
+  }
+  // whatever is left (a ragged tail, or everything when the fast path does not apply), and the
+  // zero padding of the three regions
+  p.coord_base = (uint64_t)full_tiles * kTile;
+  const uint64_t rem = p.n - p.coord_base;
+  uint64_t tiles = (rem + p.tile_coords - 1) / p.tile_coords;
+  if (tiles == 0) tiles = 1;
+  {
+    ScopedKernel sk(kKernQuantizeTail, stream);
+    quantize_generic_kernel<LB, NORM><<<(uint32_t)tiles, kThreads, 0, stream>>>(p);
   }
   return (int)cudaGetLastError();
 }
 
 template <int LB>
-int launch_lb(const QuantizeParams& p, int norm_kind, bool pow2, uint64_t seed, cudaStream_t stream) {
-  return norm_kind == QSGD_NORM_L2 ? launch_one<LB, QSGD_NORM_L2>(p, pow2, seed, stream)
-                                   : launch_one<LB, QSGD_NORM_MAX>(p, pow2, seed, stream);
+int launch_lb(QuantizeParams& p, int norm_kind, uint64_t seed, cudaStream_t stream) {
+  return norm_kind == QSGD_NORM_L2 ? launch_one<LB, QSGD_NORM_L2>(p, seed, stream)
+                                   : launch_one<LB, QSGD_NORM_MAX>(p, seed, stream);
 }
 
 }  // namespace
@@ -530,22 +614,22 @@ int launch_quantize_fixed(const float* g, uint64_t n, uint32_t d, uint32_t s, in
                           uint64_t seed, uint32_t step, uint32_t worker, uint8_t* out,
                           uint32_t* status_dev, cudaStream_t stream) {
   const FixedLayout L = make_fixed_layout(n, d, s);
-  const bool pow2 = (d & (d - 1)) == 0;
   QuantizeParams p;
   p.g = g; p.n = n; p.d = d; p.s = s;
-  p.tile_coords = pow2 ? kTile : (kTile / d) * d;
+  p.tile_coords = (kTile / d) * d;
+  p.coord_base = 0;
   p.k0 = (uint32_t)seed; p.k1 = (uint32_t)(seed >> 32); p.step = step; p.worker = worker;
   p.A_out = reinterpret_cast<float*>(out);
   p.sign_out = reinterpret_cast<uint32_t*>(out + L.off_sign);
   p.level_out = reinterpret_cast<uint32_t*>(out + L.off_level);
   p.B = L.B; p.sign_words = L.sign_words; p.level_words = L.level_words;
-  p.tiles = (n + p.tile_coords - 1) / p.tile_coords;
+  p.tiles = 0;
   p.status = status_dev;
   switch (L.lb) {
-    case 1: return launch_lb<1>(p, norm_kind, pow2, seed, stream);
-    case 2: return launch_lb<2>(p, norm_kind, pow2, seed, stream);
-    case 4: return launch_lb<4>(p, norm_kind, pow2, seed, stream);
-    default: return launch_lb<8>(p, norm_kind, pow2, seed, stream);
+    case 1: return launch_lb<1>(p, norm_kind, seed, stream);
+    case 2: return launch_lb<2>(p, norm_kind, seed, stream);
+    case 4: return launch_lb<4>(p, norm_kind, seed, stream);
+    default: return launch_lb<8>(p, norm_kind, seed, stream);
   }
 }
 
