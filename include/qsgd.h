@@ -74,6 +74,10 @@ extern "C" {
 #define QSGD_ERR_PEERS (-7)     /* K outside [1, 64]                                  */
 #define QSGD_ERR_KIND (-8)      /* unknown norm_kind or code_kind                     */
 #define QSGD_ERR_NO_DEVICE (-9) /* no usable CUDA device / kernel image for this GPU  */
+#define QSGD_ERR_SCRATCH (-10)  /* problem too large for the library's built-in scratch */
+
+/* Size of the scratch array built into the library for qsgd_encode_elias_static. */
+#define QSGD_STATIC_SCRATCH_BYTES (32u << 20)
 
 #define QSGD_DEV_CAPACITY 1u  /* encoded message would exceed out_capacity             */
 #define QSGD_DEV_OVERRUN 2u   /* an Elias code runs past the end of its bucket string  */
@@ -141,6 +145,39 @@ const char* qsgd_status_string(int status);
 
 /* Number of kernels this library has launched in this process (all calls, all streams). */
 uint64_t qsgd_launch_count(void);
+
+/*
+ * Elias Encode that allocates nothing and needs no caller-supplied workspace. (The paper has no
+ * counterpart: this is a packaging of qsgd_encode for one kind of caller.)
+ *
+ * Who needs it: code that may not obtain device memory at the moment it has to encode -- a
+ * gradient hook that fires inside a framework whose caching allocator is locked or whose memory
+ * budget was fixed at start-up, a communication plug-in that is handed buffers but no allocator,
+ * a latency-critical thread that must not enter cudaMalloc (which can synchronise the whole
+ * device). Such a caller still passes the gradient, the message buffer, the four info words and
+ * the status word, as for qsgd_encode; what it cannot provide is the qsgd_workspace_bytes() of
+ * scratch. Here that scratch is one array of QSGD_STATIC_SCRATCH_BYTES (32 MiB) compiled into
+ * the library as a device global, so every GPU that loads the library carries it until the
+ * process exits. The call itself performs no cudaMalloc, cudaFree or other allocating call.
+ *
+ *   - code_kind must be QSGD_CODE_ELIAS or QSGD_CODE_ELIAS_DENSE (fixed-width needs no scratch:
+ *     use qsgd_encode). Results are bit-identical to qsgd_encode with the same arguments.
+ *   - Limit: qsgd_workspace_bytes(n, bucket, s, code_kind) must not exceed
+ *     qsgd_static_scratch_bytes(); e.g. bucket 512, s = 15 fits up to about 51 million
+ *     coordinates. Larger problems are rejected with QSGD_ERR_SCRATCH and nothing is launched.
+ *   - The first call on each device looks up the device address of the built-in array (a host
+ *     side query, done with that device current and cached per device). Make that first call
+ *     outside of any stream capture.
+ *   - All calls on one device share the one array, which keeps whatever the previous call left
+ *     in it; every region the kernels read is rewritten by the same call first, so nothing needs
+ *     clearing between calls. Two calls that overlap on the GPU (different streams, or several
+ *     host threads) race on the array and corrupt each other's messages: serialise them.
+ */
+size_t qsgd_static_scratch_bytes(void);
+int qsgd_encode_elias_static(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int norm_kind,
+                             int code_kind, uint64_t seed, uint32_t step, uint32_t worker, void* out,
+                             size_t out_capacity, uint64_t* out_bits, uint32_t* status_dev,
+                             qsgd_stream_t stream);
 
 /*
  * Per-kernel timing (measurement aid; the paper has no counterpart). While enabled, every

@@ -18,7 +18,8 @@ DEV_CAPACITY, DEV_OVERRUN, DEV_POSITION, DEV_LEVEL, DEV_TABLE, DEV_TIMEOUT = 1, 
 EXPORTS = ["qsgd_message_capacity", "qsgd_workspace_bytes", "qsgd_fixed_layout", "qsgd_encode",
            "qsgd_decode_accumulate", "qsgd_sgd_step", "qsgd_decode_sgd_step",
            "qsgd_status_string", "qsgd_launch_count", "qsgd_profile_enable",
-           "qsgd_profile_kernel_count", "qsgd_profile_kernel_name", "qsgd_profile_collect"]
+           "qsgd_profile_kernel_count", "qsgd_profile_kernel_name", "qsgd_profile_collect",
+           "qsgd_static_scratch_bytes", "qsgd_encode_elias_static"]
 
 _lib = None
 
@@ -54,6 +55,11 @@ def lib():
         L.qsgd_decode_sgd_step.restype = C.c_int
         L.qsgd_status_string.argtypes = [C.c_int]
         L.qsgd_status_string.restype = C.c_char_p
+        L.qsgd_static_scratch_bytes.argtypes = []
+        L.qsgd_static_scratch_bytes.restype = sz
+        L.qsgd_encode_elias_static.argtypes = [vp, u64, u32, u32, C.c_int, C.c_int, u64, u32, u32, vp,
+                                               sz, vp, vp, vp]
+        L.qsgd_encode_elias_static.restype = C.c_int
         L.qsgd_launch_count.argtypes = []
         L.qsgd_launch_count.restype = u64
         L.qsgd_profile_enable.argtypes = [C.c_int]
@@ -131,6 +137,26 @@ def qsgd_encode(g, bucket, s, norm_kind, code_kind, seed, step, worker, out, out
     _check(lib().qsgd_encode(g.data_ptr(), n, bucket, s, norm_kind, code_kind, seed, step, worker,
                              out.data_ptr(), out.numel() * out.element_size(),
                              out_bits.data_ptr(), ws, status_dev.data_ptr(), _stream(stream)))
+
+
+def qsgd_static_scratch_bytes():
+    return int(lib().qsgd_static_scratch_bytes())
+
+
+def qsgd_encode_elias_static(g, bucket, s, norm_kind, code_kind, seed, step, worker, out, out_bits,
+                             status_dev, stream=None):
+    """Elias Encode without a workspace argument: the scratch is a 32 MiB array built into the
+    library, so this call allocates nothing (for callers that may not allocate device memory when
+    they encode). Same results as qsgd_encode; sizes beyond the built-in scratch raise. Calls
+    that overlap on the GPU share the scratch and must be serialised by the caller."""
+    _require_cuda(g, "g")
+    _require_cuda(out, "out")
+    _require_cuda(out_bits, "out_bits")
+    _require_cuda(status_dev, "status_dev")
+    _check(lib().qsgd_encode_elias_static(g.data_ptr(), g.numel(), bucket, s, norm_kind, code_kind,
+                                          seed, step, worker, out.data_ptr(),
+                                          out.numel() * out.element_size(), out_bits.data_ptr(),
+                                          status_dev.data_ptr(), _stream(stream)))
 
 
 def _ptr_array(tensors):

@@ -208,6 +208,7 @@ const char* qsgd_status_string(int status) {
     case QSGD_ERR_PEERS: return "K must lie in [1, 64]";
     case QSGD_ERR_KIND: return "unknown norm or code kind";
     case QSGD_ERR_NO_DEVICE: return "no usable CUDA device";
+    case QSGD_ERR_SCRATCH: return "problem too large for the built-in scratch array";
     default: return status > 0 ? cudaGetErrorString((cudaError_t)status) : "unknown status";
   }
 }

@@ -7,6 +7,8 @@
 //   4. zero the payload, then a warp-cooperative scatter writes every bucket's string at its
 //      bit offset: lanes own consecutive sub-ranges of the bucket, a warp scan gives each lane
 //      its first bit, words shared between lanes or buckets are merged with atomicOr.
+#include <mutex>
+
 #include "elias_common.cuh"
 
 namespace qsgd {
@@ -382,3 +384,72 @@ int launch_elias_encode(const float* g, uint64_t n, uint32_t d, uint32_t s, int 
 }
 
 }  // namespace qsgd
+
+// ================================================================================================
+// Elias encode with library-owned scratch (see qsgd_encode_elias_static in include/qsgd.h).
+//
+// The scratch lives in this translation unit as one file-scope device array, so the entry point
+// never asks the driver (or anybody's allocator) for memory. In host code the name of a
+// __device__ array is only a handle for the runtime: its device address has to be looked up with
+// cudaGetSymbolAddress, once per device, with that device current. The looked-up pointer is what
+// the kernels receive.
+// ================================================================================================
+namespace qsgd {
+namespace {
+
+constexpr size_t kStaticScratchBytes = (size_t)QSGD_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_scratch_mu;
+static uint8_t* g_scratch_ptr[kMaxDevices] = {};
+
+// Device address of the scratch array on the current device; looked up on first use.
+int static_scratch_pointer(uint8_t** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return (int)e;
+  if (dev < 0 || dev >= kMaxDevices) return (int)cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lk(g_scratch_mu);
+  if (!g_scratch_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_scratch);
+    if (e != cudaSuccess) return (int)e;
+    if (!p) return (int)cudaErrorInvalidSymbol;
+    g_scratch_ptr[dev] = static_cast<uint8_t*>(p);
+  }
+  *out = g_scratch_ptr[dev];
+  return 0;
+}
+
+}  // namespace
+}  // namespace qsgd
+
+extern "C" {
+
+size_t qsgd_static_scratch_bytes(void) { return qsgd::kStaticScratchBytes; }
+
+int qsgd_encode_elias_static(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int norm_kind,
+                             int code_kind, uint64_t seed, uint32_t step, uint32_t worker, void* out,
+                             size_t out_capacity, uint64_t* out_bits, uint32_t* status_dev,
+                             qsgd_stream_t stream) {
+  using namespace qsgd;
+  if (!g || !out || !out_bits || !status_dev) return QSGD_ERR_NULL;
+  if (n == 0) return QSGD_ERR_SIZE;
+  if (bucket < 32 || bucket > QSGD_MAX_BUCKET || (bucket & 31u)) return QSGD_ERR_BUCKET;
+  if (s < 1 || s > QSGD_MAX_LEVELS) return QSGD_ERR_LEVELS;
+  if (code_kind != QSGD_CODE_ELIAS && code_kind != QSGD_CODE_ELIAS_DENSE) return QSGD_ERR_KIND;
+  if (norm_kind != QSGD_NORM_L2 && norm_kind != QSGD_NORM_MAX) return QSGD_ERR_KIND;
+  if ((reinterpret_cast<uintptr_t>(g) & 15u) || (reinterpret_cast<uintptr_t>(out) & 15u)) return QSGD_ERR_ALIGN;
+  const uint64_t B = (n + bucket - 1) / bucket;
+  if (out_capacity < align16(4 * B) + 8 * (B + 1)) return QSGD_ERR_CAPACITY;
+  if (elias_workspace_bytes(n, bucket, s) > kStaticScratchBytes) return QSGD_ERR_SCRATCH;
+  uint8_t* scratch = nullptr;
+  const int st = static_scratch_pointer(&scratch);
+  if (st) return st;
+  return launch_elias_encode(g, n, bucket, s, norm_kind, code_kind == QSGD_CODE_ELIAS_DENSE, seed, step,
+                             worker, static_cast<uint8_t*>(out), out_capacity, out_bits, scratch,
+                             status_dev, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"
