@@ -1,13 +1,17 @@
 // Decode-and-aggregate, Elias path, optionally fused with the SGD step (Section 3.1: "read off
 // 32 bits to construct the norm, then iteratively ... read off the positions and values of the
-// nonzeros"; Algorithm 1 for the sum and the step).
+// nonzeros"; Appendix A.2 decoder; Algorithm 1 for the sum and the step).
 //
 // A string S can only be parsed front to back, but buckets and peers are independent once the
-// per-bucket offset table gives each string's first bit. One warp owns one bucket. Phase 1:
-// lane k parses peer k's string for this bucket (all peers in parallel) and drops a one-byte
-// (or two-byte) code "sign | level" at the coordinate's slot of a dense K x d scratch in shared
-// memory. Phase 2: every lane takes 4 consecutive coordinates and adds the peers' values in
-// ascending k, which fixes the summation order regardless of how phase 1 was scheduled.
+// per-bucket offset table gives each string's first bit. A warp owns a group of G buckets.
+// Phase 1 (parse): lane (g, k) reads peer k's string of bucket g through a 64-bit register
+// window (next word prefetched) and rebuilds that peer's *fixed-width fields* -- level fields
+// and sign bitmap -- for the bucket in shared memory. Phase 2 (apply): exactly the fixed-width
+// decoder's inner loop, reading the fields from shared memory: every lane takes 16 coordinates
+// and adds the peers in ascending k, which fixes the summation order however phase 1 was
+// scheduled. A slower kernel with byte codes covers shapes whose fields do not fit in shared
+// memory.
+#include "decode_common.cuh"
 #include "elias_common.cuh"
 
 namespace qsgd {
@@ -78,7 +82,7 @@ __device__ __forceinline__ uint32_t parse_bucket(const uint32_t* __restrict__ wo
 }
 
 template <typename CodeT, bool DENSE, bool FUSED>
-__global__ void __launch_bounds__(kThreads) decode_elias_kernel(const __grid_constant__ EliasDecodeParams p) {
+__global__ void __launch_bounds__(kThreads) decode_elias_slow_kernel(const __grid_constant__ EliasDecodeParams p) {
   extern __shared__ __align__(16) uint8_t smem[];
   __shared__ float xi[256];
   const float sf = (float)p.s;
@@ -168,7 +172,7 @@ __global__ void __launch_bounds__(kThreads) decode_elias_kernel(const __grid_con
 }
 
 template <typename CodeT, bool DENSE>
-int launch_t(EliasDecodeParams& p, bool fused, cudaStream_t stream) {
+int launch_slow(EliasDecodeParams& p, bool fused, cudaStream_t stream) {
   // shared memory per warp: d floats of acc, 64 floats of scales, Kc x d codes
   int dev = 0, max_smem = 0, sms = 0;
   cudaGetDevice(&dev);
@@ -182,7 +186,7 @@ int launch_t(EliasDecodeParams& p, bool fused, cudaStream_t stream) {
   p.Kc = (uint32_t)kc;
   p.warp_bytes = (uint32_t)align16(fixed + kc * p.d * sizeof(CodeT));
   const size_t smem = (size_t)p.warp_bytes * kWarps;
-  auto kern = fused ? decode_elias_kernel<CodeT, DENSE, true> : decode_elias_kernel<CodeT, DENSE, false>;
+  auto kern = fused ? decode_elias_slow_kernel<CodeT, DENSE, true> : decode_elias_slow_kernel<CodeT, DENSE, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return (int)e;
   const uint64_t want = (p.B + kWarps - 1) / kWarps;
@@ -195,17 +199,310 @@ int launch_t(EliasDecodeParams& p, bool fused, cudaStream_t stream) {
   return (int)cudaGetLastError();
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Field-rebuilding decoder
+// ------------------------------------------------------------------------------------------------
+struct FieldParams {
+  PeerSet peers;
+  uint32_t K;
+  uint32_t Kpad;        // lanes per bucket in the parse phase (power of two, <= 32)
+  uint32_t G;           // buckets per warp
+  uint64_t n;
+  uint32_t d;
+  uint32_t s;
+  uint64_t B;
+  float* out;
+  float c;
+  uint32_t* status;
+  uint32_t row_words;   // per peer row: d * lb / 32 level words, then d / 32 sign words (padded to 4)
+  uint32_t bucket_words;  // K rows + K scales, padded to 4
+};
+
+// Bit source over the payload: 64-bit left-aligned window, one word prefetched.
+struct BitSrc {
+  const uint32_t* words;
+  uint64_t widx;     // index of `nextw`
+  uint32_t nextw;
+  uint64_t win;
+  uint32_t avail;
+  __device__ __forceinline__ void open(const uint32_t* w, uint64_t bit) {
+    words = w;
+    widx = bit >> 5;
+    const uint32_t w0 = __ldg(words + widx), w1 = __ldg(words + widx + 1);
+    nextw = __ldg(words + widx + 2);
+    const uint32_t sh = (uint32_t)(bit & 31);
+    win = (((uint64_t)w0 << 32) | w1) << sh;
+    avail = 64 - sh;
+    widx += 2;
+  }
+  __device__ __forceinline__ void refill() {          // afterwards at least 33 valid bits
+    if (avail <= 32) {
+      win |= (uint64_t)nextw << (32 - avail);
+      avail += 32;
+      ++widx;
+      nextw = __ldg(words + widx);
+    }
+  }
+  __device__ __forceinline__ uint32_t take(uint32_t nb) {   // nb in [1, 32]
+    const uint32_t v = (uint32_t)(win >> (64 - nb));
+    win <<= nb;
+    avail -= nb;
+    return v;
+  }
+  // Definition A.1 decoder on the window; at most three groups (values < 2^16).
+  __device__ __forceinline__ bool elias(uint32_t& value, uint32_t& used) {
+    uint32_t N = 1;
+#pragma unroll
+    for (int it = 0; it < 3; ++it) {
+      if (!(win >> 63)) break;
+      const uint32_t nb = N + 1;
+      N = take(nb);
+      used += nb;
+    }
+    if (win >> 63) return false;
+    take(1);
+    used += 1;
+    value = N;
+    return true;
+  }
+};
+
+// Accumulates field bits for ascending positions and stores a word when the position moves on.
+struct FieldWriter {
+  uint32_t* row;
+  uint32_t cur_idx, cur_val;
+  __device__ __forceinline__ void begin(uint32_t* r) { row = r; cur_idx = 0xFFFFFFFFu; cur_val = 0; }
+  __device__ __forceinline__ void put(uint32_t idx, uint32_t bits) {
+    if (idx != cur_idx) {
+      if (cur_idx != 0xFFFFFFFFu) row[cur_idx] = cur_val;
+      cur_idx = idx;
+      cur_val = 0;
+    }
+    cur_val |= bits;
+  }
+  __device__ __forceinline__ void end() { if (cur_idx != 0xFFFFFFFFu) row[cur_idx] = cur_val; }
+};
+
+template <int LB, bool DENSE>
+__device__ __forceinline__ uint32_t parse_to_fields(const uint32_t* __restrict__ words,
+                                                    const uint64_t* __restrict__ table, uint64_t b,
+                                                    uint64_t B, uint32_t db, uint32_t d, uint32_t s,
+                                                    uint32_t* __restrict__ row, float* A_out) {
+  const uint64_t lo = __ldg(table + b), hi = __ldg(table + b + 1), all = __ldg(table + B);
+  *A_out = 0.f;
+  if (hi < lo || hi - lo < 32 || hi > all) return QSGD_DEV_TABLE;
+  const uint64_t cap_bits = (uint64_t)((const uint8_t*)table - (const uint8_t*)words) * 8ull;
+  if ((const uint8_t*)table > (const uint8_t*)words && all > cap_bits) return QSGD_DEV_TABLE;
+  if (hi - lo > 32ull + (uint64_t)db * 40ull) return QSGD_DEV_OVERRUN;   // longer than any legal string
+  const uint32_t total = (uint32_t)(hi - lo) - 32u;
+  BitSrc src;
+  src.open(words, lo);
+  *A_out = __uint_as_float(src.take(32));
+  FieldWriter lv, sg;
+  lv.begin(row);
+  sg.begin(row + (d * LB >> 5));
+  uint32_t used = 0, err = 0;
+  if (DENSE) {
+    for (uint32_t c = 0; c < db; ++c) {
+      src.refill();
+      const uint32_t neg = src.take(1);
+      uint32_t v;
+      if (!src.elias(v, used)) { err = QSGD_DEV_OVERRUN; break; }
+      used += 1;
+      if (used > total) { err = QSGD_DEV_OVERRUN; break; }
+      if (v - 1u > s) { err = QSGD_DEV_LEVEL; break; }
+      if (v > 1u) {
+        lv.put((c * LB) >> 5, (v - 1u) << ((c * LB) & 31));
+        if (neg) sg.put(c >> 5, 1u << (c & 31));
+      }
+    }
+    if (!err && used != total) err = QSGD_DEV_OVERRUN;
+  } else {
+    int32_t at = -1;
+    while (used < total) {
+      uint32_t gap, level;
+      src.refill();
+      if (!src.elias(gap, used) || used >= total) { err = QSGD_DEV_OVERRUN; break; }
+      at += (int32_t)gap;
+      if (at >= (int32_t)db) { err = QSGD_DEV_POSITION; break; }
+      const uint32_t neg = src.take(1);
+      used += 1;
+      src.refill();
+      if (!src.elias(level, used) || used > total) { err = QSGD_DEV_OVERRUN; break; }
+      if (level < 1u || level > s) { err = QSGD_DEV_LEVEL; break; }
+      lv.put(((uint32_t)at * LB) >> 5, level << (((uint32_t)at * LB) & 31));
+      if (neg) sg.put((uint32_t)at >> 5, 1u << ((uint32_t)at & 31));
+    }
+  }
+  lv.end();
+  sg.end();
+  return err;
+}
+
+template <int LB, bool DENSE, bool FUSED, bool SINGLE>
+__global__ void __launch_bounds__(128) decode_elias_fields_kernel(const __grid_constant__ FieldParams p) {
+  extern __shared__ __align__(16) uint32_t fsm[];
+  __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const float sf = (float)p.s;
+  float lut0 = 0.f;
+  if (LB == 8) {
+    for (uint32_t i = tid; i < 256 * 32; i += blockDim.x) xi_tab[i] = __fdiv_rn((float)(i >> 5), sf);
+    __syncthreads();
+  } else {
+    const uint32_t level = lane & ((1u << LB) - 1u), neg = (lane >> LB) & 1u;
+    const float q = __fdiv_rn((float)level, sf);
+    lut0 = neg ? -q : q;
+  }
+  const uint8_t* tab_lane = reinterpret_cast<const uint8_t*>(xi_tab) + 4 * lane;
+
+  const uint32_t warp_words = p.G * p.bucket_words;
+  uint32_t* mine = fsm + (size_t)warp * warp_words;
+  const uint32_t level_words = (p.d * LB) >> 5;
+  const uint32_t pg = lane / p.Kpad, pk = lane % p.Kpad;      // parse role: bucket in group, peer
+  const uint32_t slots_per_bucket = p.d >> 4;                 // 16-coordinate lane slots
+  const uint32_t total_slots = p.G * slots_per_bucket;
+  const uint64_t groups = (p.B + p.G - 1) / p.G;
+
+  for (uint64_t grp = (uint64_t)blockIdx.x * nwarps + warp; grp < groups; grp += (uint64_t)gridDim.x * nwarps) {
+    const uint64_t b0 = grp * p.G;
+    for (uint32_t q = lane; q < (warp_words >> 2); q += 32) reinterpret_cast<uint4*>(mine)[q] = make_uint4(0u, 0u, 0u, 0u);
+    __syncwarp();
+    // ---- phase 1: one lane per (bucket, peer) ------------------------------------------------
+    for (uint32_t k = pk; k < p.K; k += 32) {
+      const uint64_t b = b0 + pg;
+      if (pg < p.G && b < p.B) {
+        uint32_t* bucket = mine + pg * p.bucket_words;
+        const uint64_t base = b * p.d;
+        const uint32_t db = (uint32_t)min((uint64_t)p.d, p.n - base);
+        float A;
+        const uint32_t st = parse_to_fields<LB, DENSE>(p.peers.payload[k], p.peers.table[k], b, p.B, db, p.d,
+                                                       p.s, bucket + k * p.row_words, &A);
+        reinterpret_cast<float*>(bucket + p.K * p.row_words)[k] = A;
+        if (st) atomicOr(p.status, st);
+      }
+      if (p.Kpad < 32) break;
+    }
+    __syncwarp();
+    // ---- phase 2: the fixed-width decoder's inner loop over the rebuilt fields ----------------
+    for (uint32_t s0 = 0; s0 < total_slots; s0 += 32) {
+      const uint32_t slot = s0 + lane;
+      const uint32_t g = slot / slots_per_bucket, c = (slot - g * slots_per_bucket) << 4;
+      const uint64_t b = b0 + g;
+      const uint64_t i0 = b * p.d + c;
+      const bool live = slot < total_slots && b < p.B && i0 < p.n;
+      const uint32_t* bucket = mine + (live ? g : 0) * p.bucket_words;
+      const float* scales = reinterpret_cast<const float*>(bucket + p.K * p.row_words);
+      float acc[16];
+#pragma unroll
+      for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+#pragma unroll 2
+      for (uint32_t k = 0; k < p.K; ++k) {
+        const uint32_t* row = bucket + k * p.row_words;
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        uint32_t sb = 0;
+        float A = 0.f;
+        if (live) {
+          A = scales[k];
+          sb = (row[level_words + (c >> 5)] >> (c & 31)) & 0xFFFFu;
+          if (LB == 8) {
+            const uint4 t = *reinterpret_cast<const uint4*>(row + (c >> 2));
+            w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
+          } else if (LB == 4) {
+            const uint2 t = *reinterpret_cast<const uint2*>(row + (c >> 3));
+            w[0] = t.x; w[1] = t.y;
+          } else if (LB == 2) {
+            w[0] = row[c >> 4];
+          } else {
+            w[0] = (row[c >> 5] >> (c & 31)) & 0xFFFFu;
+          }
+        }
+        if (LB == 8) add_peer_tab(acc, w, sb, tab_lane, A);
+        else if (SINGLE) add_peer_lut<LB, true>(acc, w, sb, __fmul_rn(__shfl_sync(0xffffffffu, A, 0), lut0), A);
+        else add_peer_lut<LB, false>(acc, w, sb, lut0, A);
+      }
+      if (live) store_lane16<FUSED>(p.out + i0, acc, i0, p.n, p.c);
+    }
+    __syncwarp();
+  }
+}
+
+template <int LB, bool DENSE>
+int launch_fields(FieldParams& p, bool fused, cudaStream_t stream, bool* handled) {
+  *handled = false;
+  int dev = 0, max_smem = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const uint32_t level_words = (p.d * LB) >> 5, sign_words = p.d >> 5;
+  p.row_words = (level_words + sign_words + 3u) & ~3u;
+  p.bucket_words = (p.K * p.row_words + p.K + 3u) & ~3u;
+  uint32_t kpad = 1;
+  while (kpad < p.K && kpad < 32) kpad <<= 1;
+  p.Kpad = kpad;
+  uint32_t G = p.K <= 32 ? 32 / kpad : 1;
+  while (G > 1 && (size_t)G * p.bucket_words * 4 > (16u << 10)) G >>= 1;
+  p.G = G;
+  const size_t per_warp = (size_t)G * p.bucket_words * 4;
+  const size_t budget = (size_t)max_smem - (LB == 8 ? 32768 : 128) - 1024;
+  int warps = 4;
+  while (warps > 1 && (size_t)warps * per_warp > (warps == 4 ? (96u << 10) : budget)) warps >>= 1;
+  if ((size_t)warps * per_warp > budget) return 0;               // caller falls back to the slow kernel
+  const bool single = p.d >= 512 && (p.d & (p.d - 1)) == 0 && LB != 8;
+  void (*kern)(FieldParams);
+  if (fused) kern = single ? decode_elias_fields_kernel<LB, DENSE, true, true> : decode_elias_fields_kernel<LB, DENSE, true, false>;
+  else kern = single ? decode_elias_fields_kernel<LB, DENSE, false, true> : decode_elias_fields_kernel<LB, DENSE, false, false>;
+  const size_t smem = (size_t)warps * per_warp;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return (int)e;
+  int occ = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, warps * 32, smem);
+  if (e != cudaSuccess) return (int)e;
+  if (occ < 1) occ = 1;
+  const uint64_t groups = (p.B + G - 1) / G;
+  const uint64_t want = (groups + warps - 1) / warps;
+  const uint64_t cap = (uint64_t)sms * occ;
+  const uint32_t grid = (uint32_t)(want < cap ? want : cap);
+  {
+    ScopedKernel sk(kKernDecodeElias, stream);
+    kern<<<grid, warps * 32, smem, stream>>>(p);
+  }
+  *handled = true;
+  return (int)cudaGetLastError();
+}
+
+template <int LB>
+int launch_fields_lb(FieldParams& p, bool dense, bool fused, cudaStream_t stream, bool* handled) {
+  return dense ? launch_fields<LB, true>(p, fused, stream, handled) : launch_fields<LB, false>(p, fused, stream, handled);
+}
+
 }  // namespace
 
 int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s,
                         bool dense, float* acc_or_x, bool fused, float eta, uint32_t* status_dev,
                         cudaStream_t stream) {
+  {
+    FieldParams f;
+    f.peers = peers; f.K = K; f.n = n; f.d = d; f.s = s;
+    f.B = (n + d - 1) / d;
+    f.out = acc_or_x; f.c = eta / (float)K; f.status = status_dev;
+    bool handled = false;
+    int st;
+    switch (level_bits_for(s)) {
+      case 1: st = launch_fields_lb<1>(f, dense, fused, stream, &handled); break;
+      case 2: st = launch_fields_lb<2>(f, dense, fused, stream, &handled); break;
+      case 4: st = launch_fields_lb<4>(f, dense, fused, stream, &handled); break;
+      default: st = launch_fields_lb<8>(f, dense, fused, stream, &handled); break;
+    }
+    if (handled || st) return st;
+  }
   EliasDecodeParams p;
   p.peers = peers; p.K = K; p.Kc = K; p.n = n; p.d = d; p.s = s;
   p.B = (n + d - 1) / d;
   p.out = acc_or_x; p.c = eta / (float)K; p.status = status_dev; p.warp_bytes = 0;
-  if (s <= 127) return dense ? launch_t<uint8_t, true>(p, fused, stream) : launch_t<uint8_t, false>(p, fused, stream);
-  return dense ? launch_t<uint16_t, true>(p, fused, stream) : launch_t<uint16_t, false>(p, fused, stream);
+  if (s <= 127) return dense ? launch_slow<uint8_t, true>(p, fused, stream) : launch_slow<uint8_t, false>(p, fused, stream);
+  return dense ? launch_slow<uint16_t, true>(p, fused, stream) : launch_slow<uint16_t, false>(p, fused, stream);
 }
 
 }  // namespace qsgd
