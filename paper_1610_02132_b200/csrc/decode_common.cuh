@@ -31,13 +31,40 @@ __device__ __forceinline__ void add_peer_lut(float (&acc)[16], const uint32_t (&
         acc[8 * h + 2 * j + 1] = __fadd_rn(acc[8 * h + 2 * j + 1], b);
       }
     }
+  } else if (LB == 2) {
+    // 16 two-bit levels in w[0]. Per half (8 coordinates) spread the levels to nibble spacing
+    // and drop the sign bit at bit 2 of each nibble; the lookup table repeats every 8 lanes, so
+    // whatever follows in the shifted word is ignored by the shuffle (it reads 5 index bits).
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      uint32_t x = (w[0] >> (16 * h)) & 0xFFFFu;
+      x = (x | (x << 8)) & 0x00FF00FFu;
+      x = (x | (x << 4)) & 0x0F0F0F0Fu;
+      x = (x | (x << 2)) & 0x33333333u;
+      uint32_t y = (sb >> (8 * h)) & 0xFFu;
+      y = (y | (y << 12)) & 0x000F000Fu;
+      y = (y | (y << 6)) & 0x03030303u;
+      y = (y | (y << 3)) & 0x11111111u;
+      const uint32_t z = x | (y << 2);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        float a = shfl_f(lut, z >> (4 * j));
+        if (!SINGLE) a = __fmul_rn(A, a);
+        acc[8 * h + j] = __fadd_rn(acc[8 * h + j], a);
+      }
+    }
   } else {
-    // LB = 1 or 2: 16 fields in w[0]
-    constexpr uint32_t kMask = (1u << LB) - 1u;
+    // LB = 1: interleave the 16 level bits (even positions) with the 16 sign bits (odd); the
+    // lookup table repeats every 4 lanes.
+    uint32_t x = w[0] & 0xFFFFu, y = sb & 0xFFFFu;
+    x = (x | (x << 8)) & 0x00FF00FFu; y = (y | (y << 8)) & 0x00FF00FFu;
+    x = (x | (x << 4)) & 0x0F0F0F0Fu; y = (y | (y << 4)) & 0x0F0F0F0Fu;
+    x = (x | (x << 2)) & 0x33333333u; y = (y | (y << 2)) & 0x33333333u;
+    x = (x | (x << 1)) & 0x55555555u; y = (y | (y << 1)) & 0x55555555u;
+    const uint32_t z = x | (y << 1);
 #pragma unroll
     for (int e = 0; e < 16; ++e) {
-      const uint32_t idx = ((w[0] >> (LB * e)) & kMask) | (((sb >> e) & 1u) << LB);
-      float a = shfl_f(lut, idx);
+      float a = shfl_f(lut, z >> (2 * e));
       if (!SINGLE) a = __fmul_rn(A, a);
       acc[e] = __fadd_rn(acc[e], a);
     }

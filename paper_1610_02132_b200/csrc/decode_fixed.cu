@@ -33,7 +33,7 @@ struct DecodeParams {
 };
 
 template <int LB, bool FUSED, bool SINGLE>
-__global__ void __launch_bounds__(kThreads) decode_fixed_kernel(const __grid_constant__ DecodeParams p) {
+__global__ void __launch_bounds__(kThreads, 4) decode_fixed_kernel(const __grid_constant__ DecodeParams p) {
   __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float sf = (float)p.s;
@@ -56,7 +56,7 @@ __global__ void __launch_bounds__(kThreads) decode_fixed_kernel(const __grid_con
 #pragma unroll
     for (int e = 0; e < 16; ++e) acc[e] = 0.f;
 
-#pragma unroll 4
+#pragma unroll 8
     for (uint32_t k = 0; k < p.K; ++k) {
       uint32_t w[4] = {0u, 0u, 0u, 0u};
       uint32_t sb = 0;

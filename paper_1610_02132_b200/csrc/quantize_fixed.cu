@@ -141,8 +141,7 @@ constexpr uint32_t kTwo23Bits = 0x4B000000u;
 __device__ __forceinline__ uint32_t quantize_one(float v, float r, float sf, float cap, uint32_t rnd,
                                                  uint32_t& sw) {
   const float t = __fmul_rn(__fmul_rn(sf, fabsf(v)), r);
-  // rnd >> 8 as a multiply-high keeps the shift off the (busier) integer/logic pipe
-  const float c = fma_rn(__uint2float_rn(__umulhi(rnd, 1u << 24)), 5.9604644775390625e-08f, t);
+  const float c = fma_rn(__uint2float_rn(rnd >> 8), 5.9604644775390625e-08f, t);
   const float fl = fminf(__fadd_rd(c, kTwo23), cap);       // 2^23 + min(floor(c), s)
   const float lf = __fsub_rn(fl, kTwo23);                   // the level as a float, exact
   const float sv = fma_rn(lf, v, 0.0f);                     // sign set iff level > 0 and v < 0
