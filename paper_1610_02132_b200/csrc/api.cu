@@ -120,10 +120,6 @@ int qsgd_fixed_layout(uint64_t n, uint32_t bucket, uint32_t s, uint64_t* layout)
   return QSGD_OK;
 }
 
-__global__ void write_fixed_info_kernel(uint64_t* out_bits, uint64_t total) {
-  out_bits[0] = 8 * total; out_bits[1] = 0; out_bits[2] = total; out_bits[3] = 0;
-}
-
 int qsgd_encode(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int norm_kind,
                 int code_kind, uint64_t seed, uint32_t step, uint32_t worker, void* out,
                 size_t out_capacity, uint64_t* out_bits, void* workspace, uint32_t* status_dev,
@@ -137,14 +133,8 @@ int qsgd_encode(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int nor
   if (code_kind == QSGD_CODE_FIXED) {
     const FixedLayout L = make_fixed_layout(n, bucket, s);
     if (out_capacity < L.total) return QSGD_ERR_CAPACITY;
-    st = launch_quantize_fixed(g, n, bucket, s, norm_kind, seed, step, worker,
-                               static_cast<uint8_t*>(out), status_dev, cs);
-    if (st) return st;
-    {
-      ScopedKernel sk(kKernFixedInfo, cs);
-      write_fixed_info_kernel<<<1, 1, 0, cs>>>(out_bits, L.total);
-    }
-    return (int)cudaGetLastError();
+    return launch_quantize_fixed(g, n, bucket, s, norm_kind, seed, step, worker,
+                                 static_cast<uint8_t*>(out), status_dev, out_bits, cs);
   }
   if (!workspace) return QSGD_ERR_NULL;
   if (!aligned16(workspace)) return QSGD_ERR_ALIGN;

@@ -156,8 +156,8 @@ __global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketPara
 
 // ---- 3. exclusive scan of the lengths --------------------------------------------------------
 __device__ __forceinline__ uint64_t block_exclusive_scan(uint64_t v, uint64_t* total) {
-  __shared__ uint64_t warp_sums[kWarps];
-  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __shared__ uint64_t warp_sums[32];
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
   uint64_t inc = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -167,15 +167,50 @@ __device__ __forceinline__ uint64_t block_exclusive_scan(uint64_t v, uint64_t* t
   if (lane == 31) warp_sums[warp] = inc;
   __syncthreads();
   uint64_t before = 0, all = 0;
-#pragma unroll
-  for (int w = 0; w < kWarps; ++w) {
+  for (uint32_t w = 0; w < nwarps; ++w) {
     const uint64_t t = warp_sums[w];
-    if ((uint32_t)w < warp) before += t;
+    if (w < warp) before += t;
     all += t;
   }
   __syncthreads();
   *total = all;
   return before + inc - v;
+}
+
+// Message geometry once the payload length is known; capacity check.
+__device__ __forceinline__ void finish_totals(uint64_t bits, uint64_t B, size_t out_capacity, Ctrl* ctrl,
+                                              uint64_t* __restrict__ out_bits,
+                                              uint32_t* __restrict__ status_dev) {
+  const uint64_t pay = align16((bits + 7) / 8);
+  const uint64_t total_bytes = pay + 8 * (B + 1);
+  const bool ok = total_bytes <= out_capacity;
+  ctrl->total_bits = bits;
+  ctrl->payload_bytes = pay;
+  ctrl->ok = ok ? 1u : 0u;
+  out_bits[0] = bits; out_bits[1] = pay; out_bits[2] = total_bytes; out_bits[3] = 0;
+  if (!ok) atomicOr(status_dev, QSGD_DEV_CAPACITY);
+}
+
+// Publishes one bucket offset: workspace copy, table entry, and a zero in the payload word that
+// this bucket shares with its predecessor (the scatter ORs into such words, and stores all
+// others plainly, so nothing else of the payload needs clearing).
+__device__ __forceinline__ void publish_offset(uint64_t b, uint64_t B, uint64_t run, uint32_t len,
+                                               bool ok, uint64_t payload_bytes,
+                                               uint64_t* __restrict__ off, uint64_t* __restrict__ table,
+                                               uint32_t* __restrict__ words) {
+  off[b] = run;
+  if (ok) {
+    table[b] = run;
+    if (run & 31) words[run >> 5] = 0u;
+  }
+  if (b == B - 1) {
+    const uint64_t end = run + len;
+    off[B] = end;
+    if (ok) {
+      table[B] = end;
+      for (uint64_t w = end >> 5; w < payload_bytes / 4; ++w) words[w] = 0u;   // tail word + padding
+    }
+  }
 }
 
 __global__ void __launch_bounds__(kThreads) scan_block_sums_kernel(const uint32_t* __restrict__ len,
@@ -210,17 +245,7 @@ __global__ void __launch_bounds__(kThreads) scan_sums_kernel(uint64_t* __restric
     if (threadIdx.x == 0) carry_s = carry + total;
     __syncthreads();
   }
-  if (threadIdx.x == 0) {
-    const uint64_t bits = carry_s;
-    const uint64_t pay = align16((bits + 7) / 8);
-    const uint64_t total_bytes = pay + 8 * (B + 1);
-    const bool ok = total_bytes <= out_capacity;
-    ctrl->total_bits = bits;
-    ctrl->payload_bytes = pay;
-    ctrl->ok = ok ? 1u : 0u;
-    out_bits[0] = bits; out_bits[1] = pay; out_bits[2] = total_bytes; out_bits[3] = 0;
-    if (!ok) atomicOr(status_dev, QSGD_DEV_CAPACITY);
-  }
+  if (threadIdx.x == 0) finish_totals(carry_s, B, out_capacity, ctrl, out_bits, status_dev);
 }
 
 __global__ void __launch_bounds__(kThreads) scan_downsweep_kernel(const uint32_t* __restrict__ len,
@@ -237,43 +262,97 @@ __global__ void __launch_bounds__(kThreads) scan_downsweep_kernel(const uint32_t
   uint64_t total;
   uint64_t run = sums[blockIdx.x] + block_exclusive_scan(v, &total);
   const bool ok = ctrl->ok != 0;
-  uint64_t* table = reinterpret_cast<uint64_t*>(out + ctrl->payload_bytes);
+  const uint64_t pay = ctrl->payload_bytes;
+  uint64_t* table = reinterpret_cast<uint64_t*>(out + pay);
 #pragma unroll
   for (int j = 0; j < kScanItems; ++j) {
     if (i0 + j < B) {
-      off[i0 + j] = run;
-      if (ok) table[i0 + j] = run;
+      publish_offset(i0 + j, B, run, l[j], ok, pay, off, table, reinterpret_cast<uint32_t*>(out));
       run += l[j];
-      if (i0 + j == B - 1) { off[B] = run; if (ok) table[B] = run; }
     }
   }
 }
 
-// ---- 4a. zero the payload ----------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) zero_payload_kernel(uint8_t* __restrict__ out,
-                                                                const Ctrl* __restrict__ ctrl) {
-  if (!ctrl->ok) return;
-  const uint64_t quads = ctrl->payload_bytes / 16;
-  uint4* o = reinterpret_cast<uint4*>(out);
-  for (uint64_t i = (uint64_t)blockIdx.x * kThreads + threadIdx.x; i < quads;
-       i += (uint64_t)gridDim.x * kThreads)
-    o[i] = make_uint4(0u, 0u, 0u, 0u);
+// Whole scan in one CTA of 1024 threads, for messages with few buckets (saves two launches).
+constexpr int kSmallScanThreads = 1024;
+constexpr uint64_t kSmallScanMaxBuckets = 32768;
+
+__global__ void __launch_bounds__(kSmallScanThreads) scan_small_kernel(
+    const uint32_t* __restrict__ len, uint64_t B, size_t out_capacity, Ctrl* ctrl,
+    uint64_t* __restrict__ out_bits, uint32_t* __restrict__ status_dev, uint64_t* __restrict__ off,
+    uint8_t* __restrict__ out) {
+  __shared__ uint64_t carry_s;
+  // pass 1: payload length
+  uint64_t mine = 0;
+  for (uint64_t i = threadIdx.x; i < B; i += kSmallScanThreads) mine += len[i];
+  uint64_t total;
+  block_exclusive_scan(mine, &total);
+  if (threadIdx.x == 0) {
+    finish_totals(total, B, out_capacity, ctrl, out_bits, status_dev);
+    carry_s = 0;
+  }
+  __syncthreads();
+  const bool ok = ctrl->ok != 0;
+  const uint64_t pay = ctrl->payload_bytes;
+  uint64_t* table = reinterpret_cast<uint64_t*>(out + pay);
+  // pass 2: offsets
+  for (uint64_t base = 0; base < B; base += kSmallScanThreads) {
+    const uint64_t i = base + threadIdx.x;
+    const uint32_t l = i < B ? len[i] : 0u;
+    uint64_t chunk;
+    const uint64_t ex = block_exclusive_scan(l, &chunk);
+    const uint64_t carry = carry_s;
+    if (i < B) publish_offset(i, B, carry + ex, l, ok, pay, off, table, reinterpret_cast<uint32_t*>(out));
+    __syncthreads();
+    if (threadIdx.x == 0) carry_s = carry + chunk;
+    __syncthreads();
+  }
 }
 
-// ---- 4b. scatter ---------------------------------------------------------------------------------
+// ---- 4. scatter ----------------------------------------------------------------------------------
+// Lane-private writer into the warp's staging words in shared memory (bits of neighbouring lanes
+// meet inside a word, so words are OR-ed atomically; shared-memory atomics are cheap).
+struct StageWriter {
+  uint32_t* words;
+  uint32_t widx;
+  uint64_t buf;
+  uint32_t nbuf;
+  __device__ __forceinline__ void begin(uint32_t* w, uint32_t start_bit) {
+    words = w; widx = start_bit >> 5; buf = 0; nbuf = start_bit & 31;
+  }
+  __device__ __forceinline__ void put(uint32_t code, uint32_t len) {   // len in [1, 32]
+    buf |= (uint64_t)code << (64 - nbuf - len);
+    nbuf += len;
+    if (nbuf >= 32) {
+      atomicOr(words + widx, (uint32_t)(buf >> 32));
+      ++widx; buf <<= 32; nbuf -= 32;
+    }
+  }
+  __device__ __forceinline__ void finish() {
+    if (nbuf) atomicOr(words + widx, (uint32_t)(buf >> 32));
+  }
+};
+
 template <int LB, bool DENSE>
 __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketParams p,
                                                                  const uint64_t* __restrict__ off,
                                                                  const Ctrl* __restrict__ ctrl,
-                                                                 uint8_t* __restrict__ out) {
+                                                                 uint8_t* __restrict__ out,
+                                                                 uint32_t stage_words) {
+  extern __shared__ uint32_t stage_all[];
   if (!ctrl->ok) return;
   const uint32_t lane = threadIdx.x & 31;
+  uint32_t* stage = stage_all + (size_t)(threadIdx.x >> 5) * stage_words;
   const uint64_t b = (uint64_t)blockIdx.x * kWarps + (threadIdx.x >> 5);
   if (b >= p.B) return;
   const uint64_t base = b * p.d;
   const uint32_t db = (uint32_t)min((uint64_t)p.d, p.n - base);
   const uint32_t seg = p.d >> 5;
   const uint32_t c_lo = min(lane * seg, db), c_hi = min(c_lo + seg, db);
+  const uint64_t o0 = __ldg(off + b), o1 = __ldg(off + b + 1);
+  const uint32_t lead = (uint32_t)(o0 & 31);                       // bits of the first word owned by b - 1
+  const uint32_t nwords = (uint32_t)((lead + (o1 - o0) + 31) >> 5); // words this bucket touches
+  for (uint32_t j = lane; j < nwords; j += 32) stage[j] = 0u;
 
   uint32_t bits;
   int32_t prev = -1;
@@ -291,35 +370,47 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
     const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
     if (lane >= (uint32_t)o) inc += t;
   }
-  if (bits == 0) return;
-  BitWriter bw;
-  bw.begin(reinterpret_cast<uint32_t*>(out), off[b] + (inc - bits));
-  if (lane == 0) bw.put(__float_as_uint(__ldg(p.A + b)), 32);
-  if (DENSE) {
-    for (uint32_t c = c_lo; c < c_hi; ++c) {
-      const uint64_t i = base + c;
-      const uint32_t sg = (__ldg(p.sign + (i >> 5)) >> (i & 31)) & 1u;
-      uint32_t ln;
-      const uint32_t code = elias_code(level_at<LB>(p.level, i) + 1u, &ln);
-      bw.put((sg << ln) | code, ln + 1);
+  __syncwarp();                                     // staging is zeroed
+  if (bits != 0) {
+    StageWriter bw;
+    bw.begin(stage, lead + (inc - bits));
+    if (lane == 0) bw.put(__float_as_uint(__ldg(p.A + b)), 32);
+    if (DENSE) {
+      for (uint32_t c = c_lo; c < c_hi; ++c) {
+        const uint64_t i = base + c;
+        const uint32_t sg = (__ldg(p.sign + (i >> 5)) >> (i & 31)) & 1u;
+        uint32_t ln;
+        const uint32_t code = elias_code(level_at<LB>(p.level, i) + 1u, &ln);
+        bw.put((sg << ln) | code, ln + 1);
+      }
+    } else {
+      for_each_nonzero<LB>(p.level, base, c_lo, c_hi, [&](uint32_t pos, uint32_t level) {
+        uint32_t ln;
+        uint32_t code = elias_code(pos - (uint32_t)prev, &ln);
+        bw.put(code, ln);
+        const uint64_t i = base + pos;
+        const uint32_t sg = (__ldg(p.sign + (i >> 5)) >> (i & 31)) & 1u;
+        code = elias_code(level, &ln);
+        bw.put((sg << ln) | code, ln + 1);
+        prev = (int32_t)pos;
+      });
     }
-  } else {
-    for_each_nonzero<LB>(p.level, base, c_lo, c_hi, [&](uint32_t pos, uint32_t level) {
-      uint32_t ln;
-      uint32_t code = elias_code(pos - (uint32_t)prev, &ln);
-      bw.put(code, ln);
-      const uint64_t i = base + pos;
-      const uint32_t sg = (__ldg(p.sign + (i >> 5)) >> (i & 31)) & 1u;
-      code = elias_code(level, &ln);
-      bw.put((sg << ln) | code, ln + 1);
-      prev = (int32_t)pos;
-    });
+    bw.finish();
   }
-  bw.finish();
+  __syncwarp();
+  // flush: words owned by this bucket alone are stored, words shared with a neighbour are OR-ed
+  uint32_t* gw = reinterpret_cast<uint32_t*>(out) + (o0 >> 5);
+  const bool last_shared = ((lead + (o1 - o0)) & 31) != 0;
+  for (uint32_t j = lane; j < nwords; j += 32) {
+    const uint32_t v = stage[j];
+    const bool shared = (j == 0 && lead != 0) || (j == nwords - 1 && last_shared);
+    if (shared) atomicOr(gw + j, v);
+    else gw[j] = v;
+  }
 }
 
 template <int LB, bool DENSE>
-int run_pipeline(const BucketParams& bp, const EliasWs& w, uint8_t* out, size_t out_capacity,
+int run_pipeline(const BucketParams& bp, const EliasWs& w, uint32_t s, uint8_t* out, size_t out_capacity,
                  uint64_t* out_bits, uint32_t* status_dev, cudaStream_t stream) {
   const uint32_t bucket_grid = (uint32_t)((bp.B + kWarps - 1) / kWarps);
   const uint64_t nblk = (bp.B + kScanBlock - 1) / kScanBlock;
@@ -327,27 +418,40 @@ int run_pipeline(const BucketParams& bp, const EliasWs& w, uint8_t* out, size_t 
     ScopedKernel sk(kKernEliasLength, stream);
     elias_length_kernel<LB, DENSE><<<bucket_grid, kThreads, 0, stream>>>(bp, w.len);
   }
-  {
-    ScopedKernel sk(kKernScanBlockSums, stream);
-    scan_block_sums_kernel<<<(uint32_t)nblk, kThreads, 0, stream>>>(w.len, bp.B, w.block_sums);
-  }
-  {
+  if (bp.B <= kSmallScanMaxBuckets) {
     ScopedKernel sk(kKernScanSums, stream);
-    scan_sums_kernel<<<1, kThreads, 0, stream>>>(w.block_sums, nblk, bp.B, out_capacity, w.ctrl,
-                                                 out_bits, status_dev);
+    scan_small_kernel<<<1, kSmallScanThreads, 0, stream>>>(w.len, bp.B, out_capacity, w.ctrl, out_bits,
+                                                           status_dev, w.off, out);
+  } else {
+    {
+      ScopedKernel sk(kKernScanBlockSums, stream);
+      scan_block_sums_kernel<<<(uint32_t)nblk, kThreads, 0, stream>>>(w.len, bp.B, w.block_sums);
+    }
+    {
+      ScopedKernel sk(kKernScanSums, stream);
+      scan_sums_kernel<<<1, kThreads, 0, stream>>>(w.block_sums, nblk, bp.B, out_capacity, w.ctrl,
+                                                   out_bits, status_dev);
+    }
+    {
+      ScopedKernel sk(kKernScanDownsweep, stream);
+      scan_downsweep_kernel<<<(uint32_t)nblk, kThreads, 0, stream>>>(w.len, bp.B, w.block_sums,
+                                                                     w.ctrl, w.off, out);
+    }
   }
   {
-    ScopedKernel sk(kKernScanDownsweep, stream);
-    scan_downsweep_kernel<<<(uint32_t)nblk, kThreads, 0, stream>>>(w.len, bp.B, w.block_sums,
-                                                                   w.ctrl, w.off, out);
-  }
-  {
-    ScopedKernel sk(kKernZeroPayload, stream);
-    zero_payload_kernel<<<148 * 8, kThreads, 0, stream>>>(out, w.ctrl);
-  }
-  {
+    // staging: the longest legal string of one bucket, plus the shared lead-in word
+    uint32_t elen_max = 1;
+    for (uint32_t k = DENSE ? s + 1 : s; k > 1;) { uint32_t m = 0; for (uint32_t t = k; t; t >>= 1) ++m; elen_max += m; k = m - 1; }
+    const uint32_t per = DENSE ? 1 + elen_max : 2 + elen_max;
+    const uint32_t stage_words = ((32 + bp.d * per + 31) / 32 + 2 + 3) & ~3u;
+    const size_t smem = (size_t)stage_words * 4 * kWarps;
+    auto kern = elias_scatter_kernel<LB, DENSE>;
+    if (smem > 48 * 1024) {
+      cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return (int)e;
+    }
     ScopedKernel sk(kKernEliasScatter, stream);
-    elias_scatter_kernel<LB, DENSE><<<bucket_grid, kThreads, 0, stream>>>(bp, w.off, w.ctrl, out);
+    kern<<<bucket_grid, kThreads, smem, stream>>>(bp, w.off, w.ctrl, out, stage_words);
   }
   return (int)cudaGetLastError();
 }
@@ -363,7 +467,7 @@ int launch_elias_encode(const float* g, uint64_t n, uint32_t d, uint32_t s, int 
                         size_t out_capacity, uint64_t* out_bits, uint8_t* workspace,
                         uint32_t* status_dev, cudaStream_t stream) {
   const EliasWs w = carve(workspace, n, d, s);
-  int st = launch_quantize_fixed(g, n, d, s, norm_kind, seed, step, worker, w.fixed, status_dev, stream);
+  int st = launch_quantize_fixed(g, n, d, s, norm_kind, seed, step, worker, w.fixed, status_dev, nullptr, stream);
   if (st) return st;
   const FixedLayout L = make_fixed_layout(n, d, s);
   BucketParams bp;
@@ -372,8 +476,8 @@ int launch_elias_encode(const float* g, uint64_t n, uint32_t d, uint32_t s, int 
   bp.level = reinterpret_cast<const uint32_t*>(w.fixed + L.off_level);
   bp.n = n; bp.d = d; bp.B = L.B;
 #define QSGD_RUN(LBV)                                                                            \
-  (dense ? run_pipeline<LBV, true>(bp, w, out, out_capacity, out_bits, status_dev, stream)       \
-         : run_pipeline<LBV, false>(bp, w, out, out_capacity, out_bits, status_dev, stream))
+  (dense ? run_pipeline<LBV, true>(bp, w, s, out, out_capacity, out_bits, status_dev, stream)       \
+         : run_pipeline<LBV, false>(bp, w, s, out, out_capacity, out_bits, status_dev, stream))
   switch (L.lb) {
     case 1: return QSGD_RUN(1);
     case 2: return QSGD_RUN(2);

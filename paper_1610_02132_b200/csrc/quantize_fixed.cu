@@ -42,6 +42,8 @@ struct QuantizeParams {
   uint64_t B, sign_words, level_words;
   uint64_t tiles;
   uint32_t* status;
+  uint64_t* info;         // optional: the four message-info words of a fixed-width message
+  uint64_t total_bytes;
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -168,6 +170,8 @@ struct FastParams {
   uint32_t* sign_out;
   uint32_t* level_out;
   uint32_t* status;
+  uint64_t* info;           // optional message-info words, written by CTA 0
+  uint64_t total_bytes;
   PhiloxConsts pc;
 };
 
@@ -189,6 +193,9 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
   }
   __syncthreads();
   if (tid == 0) {
+    if (blockIdx.x == 0 && p.info) {
+      p.info[0] = 8 * p.total_bytes; p.info[1] = 0; p.info[2] = p.total_bytes; p.info[3] = 0;
+    }
     for (int s = 0; s < kStages; ++s) {
       const uint32_t t = blockIdx.x + (uint32_t)s * grid;
       if (t < p.full_tiles) {
@@ -381,6 +388,9 @@ __global__ void __launch_bounds__(kThreads) quantize_generic_kernel(const Quanti
 
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint64_t t0 = p.coord_base + (uint64_t)blockIdx.x * p.tile_coords;   // first coordinate
+  if (blockIdx.x == 0 && tid == 0 && p.info) {
+    p.info[0] = 8 * p.total_bytes; p.info[1] = 0; p.info[2] = p.total_bytes; p.info[3] = 0;
+  }
   const uint64_t left = p.n - t0;
   const uint32_t valid = left < p.tile_coords ? (uint32_t)left : p.tile_coords;
   if (valid == 0) {                            // nothing left to encode: only the padding
@@ -584,6 +594,7 @@ int launch_one(QuantizeParams& p, uint64_t seed, cudaStream_t stream) {
     fp.log2d = 0;
     while ((1u << fp.log2d) < d) ++fp.log2d;
     fp.A_out = p.A_out; fp.sign_out = p.sign_out; fp.level_out = p.level_out; fp.status = p.status;
+    fp.info = p.info; fp.total_bytes = p.total_bytes;
     fp.pc = make_philox_consts(seed, p.step, p.worker);
     const int st = d >= 1024 ? launch_fast<LB, NORM, true>(fp, stream) : launch_fast<LB, NORM, false>(fp, stream);
     if (st) return st;
@@ -592,6 +603,8 @@ int launch_one(QuantizeParams& p, uint64_t seed, cudaStream_t stream) {
   // zero padding of the three regions
   p.coord_base = (uint64_t)full_tiles * kTile;
   const uint64_t rem = p.n - p.coord_base;
+  if (full_tiles > 0 && rem == 0 && ((p.B | p.sign_words | p.level_words) & 3ull) == 0)
+    return (int)cudaGetLastError();                 // no ragged tail and no padding to write
   uint64_t tiles = (rem + p.tile_coords - 1) / p.tile_coords;
   if (tiles == 0) tiles = 1;
   {
@@ -611,7 +624,7 @@ int launch_lb(QuantizeParams& p, int norm_kind, uint64_t seed, cudaStream_t stre
 
 int launch_quantize_fixed(const float* g, uint64_t n, uint32_t d, uint32_t s, int norm_kind,
                           uint64_t seed, uint32_t step, uint32_t worker, uint8_t* out,
-                          uint32_t* status_dev, cudaStream_t stream) {
+                          uint32_t* status_dev, uint64_t* info, cudaStream_t stream) {
   const FixedLayout L = make_fixed_layout(n, d, s);
   QuantizeParams p;
   p.g = g; p.n = n; p.d = d; p.s = s;
@@ -624,6 +637,8 @@ int launch_quantize_fixed(const float* g, uint64_t n, uint32_t d, uint32_t s, in
   p.B = L.B; p.sign_words = L.sign_words; p.level_words = L.level_words;
   p.tiles = 0;
   p.status = status_dev;
+  p.info = info;
+  p.total_bytes = L.total;
   switch (L.lb) {
     case 1: return launch_lb<1>(p, norm_kind, seed, stream);
     case 2: return launch_lb<2>(p, norm_kind, seed, stream);
