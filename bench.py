@@ -355,8 +355,8 @@ def run_cuda(args):
     dom = max(kern, key=lambda k: kern[k][0])
     traffic_tab = load_traffic().get(dom)
     traffic = None
-    if traffic_tab and traffic_tab.get("bytes_per_coord") is not None:
-        traffic = traffic_tab["bytes_per_coord"] * n
+    if traffic_tab and traffic_tab.get("bytes_per_coord") is not None and traffic_tab.get("K", K) == K:
+        traffic = traffic_tab["bytes_per_coord"] * n          # ncu capture on a smaller n, scaled per coordinate
     achieved = alg.get(dom, 0) / (kern_tab[dom]["avg_us"] * 1e-6) / 1e9
     roofline = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
                 "frac": achieved / hbm_peak, "peak_source": peak_src, "frac_of_nominal_8000": achieved / 8000.0,
