@@ -424,6 +424,80 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
+def run_exchange(args):
+    """Algorithm 1 across GPUs: rank = worker. Per step and code kind: encode the local gradient,
+    all-gather the K = world-size messages over NCCL, fused decode + aggregate + SGD step."""
+    import torch
+    import torch.distributed as dist
+    import paper_1610_02132_b200 as Q
+    from paper_1610_02132_b200 import exchange as X
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    os.environ.setdefault("MASTER_PORT", "29533")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    dist.init_process_group("nccl", rank=rank, world_size=world, device_id=device)
+    wl = dict(WORKLOADS[args.workload])
+    for k in ("n", "d", "s"):
+        if getattr(args, k) is not None:
+            wl[k] = getattr(args, k)
+    if args.codes:
+        wl["codes"] = args.codes.split(",")
+    n, d, s, K = wl["n"], wl["d"], wl["s"], world
+    norm = NORM[args.norm or wl["norm"]]
+    g = device_gradient(wl, rank, device)
+    x = torch.zeros(n, dtype=torch.float32, device=device)
+    status = Q.new_status(device)
+    bufs = {}
+    for cname in wl["codes"]:
+        code = CODE[cname]
+        cap = Q.qsgd_message_capacity(n, d, s, code)
+        if code != 0:
+            cap = min(cap, 2 * fixed_bytes(n, d, s) + 8 * ((n + d - 1) // d + 1))
+        cap = X.slot_bytes(cap)
+        bufs[code] = (torch.zeros(cap, dtype=torch.uint8, device=device),
+                      torch.zeros(4, dtype=torch.int64, device=device),
+                      torch.empty(max(Q.qsgd_workspace_bytes(n, d, s, code), 16), dtype=torch.uint8, device=device))
+
+    def step(i):
+        for cname in wl["codes"]:
+            code = CODE[cname]
+            out, info, ws = bufs[code]
+            Q.qsgd_encode(g, d, s, norm, code, PHILOX_SEED, i, rank, out, info, ws, status)
+            msgs, tables, _ = X.exchange(out, info, n, d, code != 0, fixed_bytes=fixed_bytes(n, d, s))
+            Q.qsgd_decode_sgd_step(msgs, tables, n, d, s, code, x, ETA, status)
+
+    for i in range(args.warmup):
+        step(i)
+    dist.barrier(); torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0 = Q.qsgd_launch_count()
+    ev0.record()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    ev1.record()
+    dist.barrier(); torch.cuda.synchronize()
+    t = torch.tensor([ev0.elapsed_time(ev1)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    assert int(status.item()) == 0
+    ms_step = float(t.item()) / args.steps
+    grad_bytes = len(wl["codes"]) * (world * 4 * n + world * K * 4 * n)
+    if rank == 0:
+        print(json.dumps({
+            "metric": "QSGD encode + decode+aggregate throughput, fp32 gradient GB/s",
+            "value": grad_bytes / (ms_step * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload + " (exchange): " + wl["desc"], "n": n, "bucket": d, "s": s,
+                       "norm": args.norm or wl["norm"], "codes": wl["codes"], "K": K,
+                       "parallelism": "rank = worker, NCCL all-gather of messages"},
+            "gpu_launches": int(Q.qsgd_launch_count() - l0)}))
+    dist.destroy_process_group()
+
+
 # ------------------------------------------------------------------------------------------------
 # the reference arm / CPU baseline: the oracle, as it stands, on host cores
 # ------------------------------------------------------------------------------------------------
@@ -501,6 +575,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--exchange", action="store_true",
+                    help="rank = worker: encode own gradient, NCCL all-gather of the messages, decode all "
+                         "K = world-size messages (Algorithm 1 across GPUs) instead of independent replicas")
     ap.add_argument("--capture", action="store_true",
                     help="for runs under a profiler: keep --warmup as given, skip e2e and the CPU baseline")
     args = ap.parse_args()
@@ -514,7 +591,10 @@ def main():
         args.no_e2e = args.no_cpu = True
     else:
         args.warmup = max(args.warmup, 3)
-    run_cuda(args)
+    if args.exchange:
+        run_exchange(args)
+    else:
+        run_cuda(args)
 
 
 if __name__ == "__main__":
