@@ -1,12 +1,18 @@
 // Encode, Elias path (Section 3.1 "Efficient Coding of Gradients", string S; Appendix A.3 for
 // the dense variant). Pipeline on one stream:
 //   1. quantize into the fixed-width layout held in the workspace (quantize_fixed.cu);
-//   2. per-bucket string length L_b, one warp per bucket;
-//   3. device-wide exclusive scan of L_b -> bit offsets (block sums, scan of sums, downsweep
-//      that also writes the offset table into the message);
-//   4. zero the payload, then a warp-cooperative scatter writes every bucket's string at its
-//      bit offset: lanes own consecutive sub-ranges of the bucket, a warp scan gives each lane
-//      its first bit, words shared between lanes or buckets are merged with atomicOr.
+//   2. string length L_b of every bucket, and the sum of the lengths of each CTA's run of
+//      consecutive buckets (elias_length_kernel);
+//   3. one CTA scans the per-CTA sums, fixes the message geometry, checks the capacity and clears
+//      the few payload words that two CTAs will share (scan_sums_kernel);
+//   4. each CTA of the scatter kernel derives the bit offsets of its own buckets, writes their
+//      offset-table entries, assembles its run of strings in shared memory (lanes own
+//      consecutive sub-ranges of a bucket; bits of neighbouring lanes and buckets meet inside
+//      words and are merged with shared-memory atomics) and flushes whole words to the payload
+//      with coalesced stores; only the first and last word of a CTA's range, which it may share
+//      with its neighbours, are merged with atomicOr in global memory.
+// A bucket is handled by a team of d / 64 lanes (at most a warp, at least one lane), so that the
+// sequential walk over a lane's nonzeros is long enough to amortise the team's scans.
 #include <mutex>
 
 #include "elias_common.cuh"
@@ -17,8 +23,6 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kScanItems = 4;                         // buckets per thread in the scan kernels
-constexpr int kScanBlock = kThreads * kScanItems;     // 1024 buckets per CTA
 
 struct Ctrl {                 // control block at the end of the workspace
   uint64_t total_bits;
@@ -27,24 +31,39 @@ struct Ctrl {                 // control block at the end of the workspace
   uint32_t pad;
 };
 
+struct Teams {
+  uint32_t lpb;               // lanes per bucket (power of two, <= 32)
+  uint32_t seg;               // coordinates per lane
+  uint32_t nbc;               // buckets per CTA
+};
+
+Teams make_teams(uint32_t d) {
+  Teams t;
+  const bool pow2 = (d & (d - 1)) == 0;
+  t.lpb = 32;
+  if (pow2) { t.lpb = d / 64; if (t.lpb < 1) t.lpb = 1; if (t.lpb > 32) t.lpb = 32; }
+  t.seg = d / t.lpb;
+  t.nbc = kWarps * (32 / t.lpb);
+  return t;
+}
+
 struct EliasWs {
   uint8_t* fixed;             // fixed-width intermediate
   uint32_t* len;              // L_b
-  uint64_t* off;              // offsets (B + 1)
-  uint64_t* block_sums;       // per scan CTA
+  uint64_t* cta_sums;         // per scatter CTA: sum of its buckets' lengths, then exclusive prefix
   Ctrl* ctrl;
   size_t bytes;
 };
 
 EliasWs carve(uint8_t* ws, uint64_t n, uint32_t d, uint32_t s) {
   const FixedLayout L = make_fixed_layout(n, d, s);
+  const Teams tm = make_teams(d);
   EliasWs w;
   size_t o = 0;
   w.fixed = ws + o; o += align16(L.total);
   w.len = reinterpret_cast<uint32_t*>(ws + o); o += align16(4 * L.B);
-  w.off = reinterpret_cast<uint64_t*>(ws + o); o += align16(8 * (L.B + 1));
-  const uint64_t nblk = (L.B + kScanBlock - 1) / kScanBlock;
-  w.block_sums = reinterpret_cast<uint64_t*>(ws + o); o += align16(8 * (nblk + 1));
+  const uint64_t ctas = (L.B + tm.nbc - 1) / tm.nbc;
+  w.cta_sums = reinterpret_cast<uint64_t*>(ws + o); o += align16(8 * (ctas + 1));
   w.ctrl = reinterpret_cast<Ctrl*>(ws + o); o += align16(sizeof(Ctrl));
   w.bytes = o;
   return w;
@@ -109,16 +128,16 @@ __device__ __forceinline__ uint32_t summarize_dense(const uint32_t* __restrict__
   return bits;
 }
 
-// Position of the last nonzero in the lanes before this one (-1 if none).
-__device__ __forceinline__ int32_t prev_nonzero_before_lane(int32_t last, uint32_t lane) {
-  int32_t run = last;                           // inclusive max-scan of `last`
+// Position of the last nonzero in the team's lanes before this one (-1 if none).
+__device__ __forceinline__ int32_t prev_nonzero_before_lane(int32_t last, uint32_t tl, uint32_t lpb) {
+  int32_t run = last;                           // inclusive max-scan of `last` inside the team
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
-    const int32_t t = __shfl_up_sync(0xffffffffu, run, o);
-    if (lane >= (uint32_t)o) run = max(run, t);
+    const int32_t t = __shfl_up_sync(0xffffffffu, run, o, 32);
+    if ((uint32_t)o < lpb && tl >= (uint32_t)o) run = max(run, t);
   }
-  const int32_t excl = __shfl_up_sync(0xffffffffu, run, 1);
-  return lane == 0 ? -1 : excl;
+  const int32_t excl = __shfl_up_sync(0xffffffffu, run, 1, 32);
+  return tl == 0 ? -1 : excl;
 }
 
 struct BucketParams {
@@ -128,33 +147,71 @@ struct BucketParams {
   uint64_t n;
   uint32_t d;
   uint64_t B;
+  uint32_t lpb, seg, nbc;
 };
 
-// ---- 2. string length per bucket -------------------------------------------------------------
+// Bits of this lane's part of its bucket's string (the scale's 32 bits go with team lane 0).
 template <int LB, bool DENSE>
-__global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketParams p,
-                                                                uint32_t* __restrict__ len) {
-  const uint32_t lane = threadIdx.x & 31;
-  const uint64_t b = (uint64_t)blockIdx.x * kWarps + (threadIdx.x >> 5);
-  if (b >= p.B) return;
-  const uint64_t base = b * p.d;
-  const uint32_t db = (uint32_t)min((uint64_t)p.d, p.n - base);
-  const uint32_t seg = p.d >> 5;
-  const uint32_t c_lo = min(lane * seg, db), c_hi = min(c_lo + seg, db);
-  uint32_t bits;
+__device__ __forceinline__ uint32_t lane_bits(const BucketParams& p, uint64_t base, uint32_t c_lo,
+                                              uint32_t c_hi, uint32_t tl, bool live, int32_t* prev_out) {
+  uint32_t bits = 0;
+  int32_t prev = -1;
   if (DENSE) {
-    bits = summarize_dense<LB>(p.level, base, c_lo, c_hi);
+    if (live) bits = summarize_dense<LB>(p.level, base, c_lo, c_hi);
   } else {
-    const LaneSummary s = summarize_sparse<LB>(p.level, base, c_lo, c_hi);
-    const int32_t prev = prev_nonzero_before_lane(s.last, lane);
+    LaneSummary s{0u, -1, -1};
+    if (live) s = summarize_sparse<LB>(p.level, base, c_lo, c_hi);
+    prev = prev_nonzero_before_lane(s.last, tl, p.lpb);
     bits = s.bits + (s.first >= 0 ? elias_len((uint32_t)(s.first - prev)) : 0u);
   }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) bits += __shfl_xor_sync(0xffffffffu, bits, o);
-  if (lane == 0) len[b] = 32u + bits;
+  if (live && tl == 0) bits += 32u;
+  *prev_out = prev;
+  return bits;
 }
 
-// ---- 3. exclusive scan of the lengths --------------------------------------------------------
+// Sum over the lanes of a team (every lane of the team receives it).
+__device__ __forceinline__ uint32_t team_sum(uint32_t v, uint32_t lpb) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const uint32_t t = __shfl_xor_sync(0xffffffffu, v, o);
+    if ((uint32_t)o < lpb) v += t;
+  }
+  return v;
+}
+
+// ---- 2. string length per bucket, sum per CTA ------------------------------------------------------
+template <int LB, bool DENSE>
+__global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketParams p,
+                                                                uint32_t* __restrict__ len,
+                                                                uint64_t* __restrict__ cta_sums) {
+  __shared__ uint32_t warp_sum[kWarps];
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t tl = lane & (p.lpb - 1), team = lane / p.lpb, bpw = 32 / p.lpb;
+  const uint64_t b = (uint64_t)blockIdx.x * p.nbc + warp * bpw + team;
+  const bool live = b < p.B;
+  const uint64_t base = live ? b * p.d : 0;
+  const uint32_t db = live ? (uint32_t)min((uint64_t)p.d, p.n - base) : 0;
+  const uint32_t c_lo = min(tl * p.seg, db), c_hi = min(c_lo + p.seg, db);
+  int32_t prev;
+  const uint32_t bits = lane_bits<LB, DENSE>(p, base, c_lo, c_hi, tl, live, &prev);
+  const uint32_t L = team_sum(bits, p.lpb);
+  if (live && tl == 0) len[b] = L;
+  uint32_t w = (tl == 0) ? L : 0u;                 // one contribution per bucket
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) w += __shfl_xor_sync(0xffffffffu, w, o);
+  if (lane == 0) warp_sum[warp] = w;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint64_t s = 0;
+#pragma unroll
+    for (int i = 0; i < kWarps; ++i) s += warp_sum[i];
+    cta_sums[blockIdx.x] = s;
+  }
+}
+
+// ---- 3. scan of the per-CTA sums (one CTA) -------------------------------------------------------
+constexpr int kScanThreads = 1024;
+
 __device__ __forceinline__ uint64_t block_exclusive_scan(uint64_t v, uint64_t* total) {
   __shared__ uint64_t warp_sums[32];
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
@@ -177,141 +234,62 @@ __device__ __forceinline__ uint64_t block_exclusive_scan(uint64_t v, uint64_t* t
   return before + inc - v;
 }
 
-// Message geometry once the payload length is known; capacity check.
-__device__ __forceinline__ void finish_totals(uint64_t bits, uint64_t B, size_t out_capacity, Ctrl* ctrl,
-                                              uint64_t* __restrict__ out_bits,
-                                              uint32_t* __restrict__ status_dev) {
-  const uint64_t pay = align16((bits + 7) / 8);
-  const uint64_t total_bytes = pay + 8 * (B + 1);
-  const bool ok = total_bytes <= out_capacity;
-  ctrl->total_bits = bits;
-  ctrl->payload_bytes = pay;
-  ctrl->ok = ok ? 1u : 0u;
-  out_bits[0] = bits; out_bits[1] = pay; out_bits[2] = total_bytes; out_bits[3] = 0;
-  if (!ok) atomicOr(status_dev, QSGD_DEV_CAPACITY);
-}
-
-// Publishes one bucket offset: workspace copy, table entry, and a zero in the payload word that
-// this bucket shares with its predecessor (the scatter ORs into such words, and stores all
-// others plainly, so nothing else of the payload needs clearing).
-__device__ __forceinline__ void publish_offset(uint64_t b, uint64_t B, uint64_t run, uint32_t len,
-                                               bool ok, uint64_t payload_bytes,
-                                               uint64_t* __restrict__ off, uint64_t* __restrict__ table,
-                                               uint32_t* __restrict__ words) {
-  off[b] = run;
-  if (ok) {
-    table[b] = run;
-    if (run & 31) words[run >> 5] = 0u;
-  }
-  if (b == B - 1) {
-    const uint64_t end = run + len;
-    off[B] = end;
-    if (ok) {
-      table[B] = end;
-      for (uint64_t w = end >> 5; w < payload_bytes / 4; ++w) words[w] = 0u;   // tail word + padding
-    }
-  }
-}
-
-__global__ void __launch_bounds__(kThreads) scan_block_sums_kernel(const uint32_t* __restrict__ len,
-                                                                   uint64_t B,
-                                                                   uint64_t* __restrict__ sums) {
-  const uint64_t i0 = (uint64_t)blockIdx.x * kScanBlock + threadIdx.x * kScanItems;
-  uint64_t v = 0;
-#pragma unroll
-  for (int j = 0; j < kScanItems; ++j) if (i0 + j < B) v += len[i0 + j];
-  uint64_t total;
-  block_exclusive_scan(v, &total);
-  if (threadIdx.x == 0) sums[blockIdx.x] = total;
-}
-
-// One CTA: exclusive scan of the block sums in place; total, message size and capacity check.
-__global__ void __launch_bounds__(kThreads) scan_sums_kernel(uint64_t* __restrict__ sums,
-                                                             uint64_t nblk, uint64_t B,
-                                                             size_t out_capacity, Ctrl* ctrl,
-                                                             uint64_t* __restrict__ out_bits,
-                                                             uint32_t* __restrict__ status_dev) {
+// In place: cta_sums[c] becomes the first payload bit of CTA c's run, cta_sums[ctas] the payload
+// length. Also: message geometry, capacity check, and zeroes in every payload word that two
+// scatter CTAs share (they OR into those; all other words are stored whole) plus the padding.
+__global__ void __launch_bounds__(kScanThreads) scan_sums_kernel(uint64_t* __restrict__ cta_sums,
+                                                                 uint64_t ctas, uint64_t B,
+                                                                 size_t out_capacity, Ctrl* ctrl,
+                                                                 uint64_t* __restrict__ out_bits,
+                                                                 uint32_t* __restrict__ status_dev,
+                                                                 uint8_t* __restrict__ out) {
   __shared__ uint64_t carry_s;
-  if (threadIdx.x == 0) carry_s = 0;
-  __syncthreads();
-  for (uint64_t base = 0; base < nblk; base += kThreads) {
-    const uint64_t i = base + threadIdx.x;
-    const uint64_t v = i < nblk ? sums[i] : 0;
-    uint64_t total;
-    const uint64_t ex = block_exclusive_scan(v, &total);
-    const uint64_t carry = carry_s;
-    if (i < nblk) sums[i] = carry + ex;
-    __syncthreads();
-    if (threadIdx.x == 0) carry_s = carry + total;
-    __syncthreads();
-  }
-  if (threadIdx.x == 0) finish_totals(carry_s, B, out_capacity, ctrl, out_bits, status_dev);
-}
-
-__global__ void __launch_bounds__(kThreads) scan_downsweep_kernel(const uint32_t* __restrict__ len,
-                                                                  uint64_t B,
-                                                                  const uint64_t* __restrict__ sums,
-                                                                  const Ctrl* __restrict__ ctrl,
-                                                                  uint64_t* __restrict__ off,
-                                                                  uint8_t* __restrict__ out) {
-  const uint64_t i0 = (uint64_t)blockIdx.x * kScanBlock + threadIdx.x * kScanItems;
-  uint32_t l[kScanItems];
-  uint64_t v = 0;
-#pragma unroll
-  for (int j = 0; j < kScanItems; ++j) { l[j] = (i0 + j < B) ? len[i0 + j] : 0u; v += l[j]; }
-  uint64_t total;
-  uint64_t run = sums[blockIdx.x] + block_exclusive_scan(v, &total);
-  const bool ok = ctrl->ok != 0;
-  const uint64_t pay = ctrl->payload_bytes;
-  uint64_t* table = reinterpret_cast<uint64_t*>(out + pay);
-#pragma unroll
-  for (int j = 0; j < kScanItems; ++j) {
-    if (i0 + j < B) {
-      publish_offset(i0 + j, B, run, l[j], ok, pay, off, table, reinterpret_cast<uint32_t*>(out));
-      run += l[j];
-    }
-  }
-}
-
-// Whole scan in one CTA of 1024 threads, for messages with few buckets (saves two launches).
-constexpr int kSmallScanThreads = 1024;
-constexpr uint64_t kSmallScanMaxBuckets = 32768;
-
-__global__ void __launch_bounds__(kSmallScanThreads) scan_small_kernel(
-    const uint32_t* __restrict__ len, uint64_t B, size_t out_capacity, Ctrl* ctrl,
-    uint64_t* __restrict__ out_bits, uint32_t* __restrict__ status_dev, uint64_t* __restrict__ off,
-    uint8_t* __restrict__ out) {
-  __shared__ uint64_t carry_s;
+  __shared__ uint32_t ok_s;
   // pass 1: payload length
   uint64_t mine = 0;
-  for (uint64_t i = threadIdx.x; i < B; i += kSmallScanThreads) mine += len[i];
+  for (uint64_t i = threadIdx.x; i < ctas; i += kScanThreads) mine += cta_sums[i];
   uint64_t total;
   block_exclusive_scan(mine, &total);
   if (threadIdx.x == 0) {
-    finish_totals(total, B, out_capacity, ctrl, out_bits, status_dev);
+    const uint64_t pay = align16((total + 7) / 8);
+    const uint64_t total_bytes = pay + 8 * (B + 1);
+    const bool ok = total_bytes <= out_capacity;
+    ctrl->total_bits = total;
+    ctrl->payload_bytes = pay;
+    ctrl->ok = ok ? 1u : 0u;
+    out_bits[0] = total; out_bits[1] = pay; out_bits[2] = total_bytes; out_bits[3] = 0;
+    if (!ok) atomicOr(status_dev, QSGD_DEV_CAPACITY);
+    ok_s = ok ? 1u : 0u;
     carry_s = 0;
+    if (ok) {
+      uint32_t* words = reinterpret_cast<uint32_t*>(out);
+      for (uint64_t w = total >> 5; w < pay / 4; ++w) words[w] = 0u;      // tail word + padding
+    }
   }
   __syncthreads();
-  const bool ok = ctrl->ok != 0;
-  const uint64_t pay = ctrl->payload_bytes;
-  uint64_t* table = reinterpret_cast<uint64_t*>(out + pay);
-  // pass 2: offsets
-  for (uint64_t base = 0; base < B; base += kSmallScanThreads) {
+  const bool ok = ok_s != 0;
+  uint32_t* words = reinterpret_cast<uint32_t*>(out);
+  // pass 2: exclusive prefix, in place
+  for (uint64_t base = 0; base < ctas; base += kScanThreads) {
     const uint64_t i = base + threadIdx.x;
-    const uint32_t l = i < B ? len[i] : 0u;
+    const uint64_t v = i < ctas ? cta_sums[i] : 0;
     uint64_t chunk;
-    const uint64_t ex = block_exclusive_scan(l, &chunk);
+    const uint64_t ex = block_exclusive_scan(v, &chunk);
     const uint64_t carry = carry_s;
-    if (i < B) publish_offset(i, B, carry + ex, l, ok, pay, off, table, reinterpret_cast<uint32_t*>(out));
+    if (i < ctas) {
+      const uint64_t start = carry + ex;
+      cta_sums[i] = start;
+      if (ok && (start & 31)) words[start >> 5] = 0u;
+    }
     __syncthreads();
     if (threadIdx.x == 0) carry_s = carry + chunk;
     __syncthreads();
   }
+  if (threadIdx.x == 0) cta_sums[ctas] = carry_s;
 }
 
 // ---- 4. scatter ----------------------------------------------------------------------------------
-// Lane-private writer into the warp's staging words in shared memory (bits of neighbouring lanes
-// meet inside a word, so words are OR-ed atomically; shared-memory atomics are cheap).
+// Lane-private writer into the CTA's staging words in shared memory.
 struct StageWriter {
   uint32_t* words;
   uint32_t widx;
@@ -335,46 +313,62 @@ struct StageWriter {
 
 template <int LB, bool DENSE>
 __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketParams p,
-                                                                 const uint64_t* __restrict__ off,
+                                                                 const uint32_t* __restrict__ len,
+                                                                 const uint64_t* __restrict__ cta_start,
                                                                  const Ctrl* __restrict__ ctrl,
-                                                                 uint8_t* __restrict__ out,
-                                                                 uint32_t stage_words) {
-  extern __shared__ uint32_t stage_all[];
+                                                                 uint8_t* __restrict__ out) {
+  extern __shared__ uint32_t stage[];
+  __shared__ uint32_t warp_sum[kWarps];
   if (!ctrl->ok) return;
-  const uint32_t lane = threadIdx.x & 31;
-  uint32_t* stage = stage_all + (size_t)(threadIdx.x >> 5) * stage_words;
-  const uint64_t b = (uint64_t)blockIdx.x * kWarps + (threadIdx.x >> 5);
-  if (b >= p.B) return;
-  const uint64_t base = b * p.d;
-  const uint32_t db = (uint32_t)min((uint64_t)p.d, p.n - base);
-  const uint32_t seg = p.d >> 5;
-  const uint32_t c_lo = min(lane * seg, db), c_hi = min(c_lo + seg, db);
-  const uint64_t o0 = __ldg(off + b), o1 = __ldg(off + b + 1);
-  const uint32_t lead = (uint32_t)(o0 & 31);                       // bits of the first word owned by b - 1
-  const uint32_t nwords = (uint32_t)((lead + (o1 - o0) + 31) >> 5); // words this bucket touches
-  for (uint32_t j = lane; j < nwords; j += 32) stage[j] = 0u;
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t tl = lane & (p.lpb - 1), team = lane / p.lpb, bpw = 32 / p.lpb;
+  const uint64_t b = (uint64_t)blockIdx.x * p.nbc + warp * bpw + team;
+  const bool live = b < p.B;
+  const uint64_t base = live ? b * p.d : 0;
+  const uint32_t db = live ? (uint32_t)min((uint64_t)p.d, p.n - base) : 0;
+  const uint32_t c_lo = min(tl * p.seg, db), c_hi = min(c_lo + p.seg, db);
 
-  uint32_t bits;
-  int32_t prev = -1;
-  if (DENSE) {
-    bits = summarize_dense<LB>(p.level, base, c_lo, c_hi);
-  } else {
-    const LaneSummary s = summarize_sparse<LB>(p.level, base, c_lo, c_hi);
-    prev = prev_nonzero_before_lane(s.last, lane);
-    bits = s.bits + (s.first >= 0 ? elias_len((uint32_t)(s.first - prev)) : 0u);
-  }
-  if (lane == 0) bits += 32u;                       // the scale travels with lane 0
-  uint32_t inc = bits;
+  const uint64_t start = __ldg(cta_start + blockIdx.x), stop = __ldg(cta_start + blockIdx.x + 1);
+  const uint32_t lead = (uint32_t)(start & 31);                     // bits of the first word owned by the previous CTA
+  const uint32_t span = (uint32_t)(stop - start);                   // bits of this CTA's run
+  const uint32_t nwords = (lead + span + 31) >> 5;
+  for (uint32_t j = threadIdx.x; j < nwords; j += kThreads) stage[j] = 0u;
+
+  // bit offset of every bucket inside the CTA's run: scan of the bucket lengths
+  const uint32_t L = (live && tl == 0) ? __ldg(len + b) : 0u;
+  uint32_t inc = L;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     const uint32_t t = __shfl_up_sync(0xffffffffu, inc, o);
     if (lane >= (uint32_t)o) inc += t;
   }
-  __syncwarp();                                     // staging is zeroed
+  if (lane == 31) warp_sum[warp] = inc;
+  __syncthreads();                                                  // staging zeroed, warp sums visible
+  uint32_t before = 0;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) if ((uint32_t)w < warp) before += warp_sum[w];
+  uint32_t bucket_off = before + inc - L;                           // valid in team lane 0
+  bucket_off = __shfl_sync(0xffffffffu, bucket_off, (int)(lane - tl));
+  const uint32_t Lb = __shfl_sync(0xffffffffu, L, (int)(lane - tl));
+  if (live && tl == 0) {
+    uint64_t* table = reinterpret_cast<uint64_t*>(out + ctrl->payload_bytes);
+    table[b] = start + bucket_off;
+    if (b == p.B - 1) table[p.B] = start + bucket_off + Lb;
+  }
+
+  // this lane's first bit inside its bucket: scan of the lane lengths over the team
+  int32_t prev;
+  const uint32_t bits = lane_bits<LB, DENSE>(p, base, c_lo, c_hi, tl, live, &prev);
+  uint32_t linc = bits;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xffffffffu, linc, o);
+    if ((uint32_t)o < p.lpb && tl >= (uint32_t)o) linc += t;
+  }
   if (bits != 0) {
     StageWriter bw;
-    bw.begin(stage, lead + (inc - bits));
-    if (lane == 0) bw.put(__float_as_uint(__ldg(p.A + b)), 32);
+    bw.begin(stage, lead + bucket_off + (linc - bits));
+    if (tl == 0) bw.put(__float_as_uint(__ldg(p.A + b)), 32);
     if (DENSE) {
       for (uint32_t c = c_lo; c < c_hi; ++c) {
         const uint64_t i = base + c;
@@ -397,11 +391,11 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
     }
     bw.finish();
   }
-  __syncwarp();
-  // flush: words owned by this bucket alone are stored, words shared with a neighbour are OR-ed
-  uint32_t* gw = reinterpret_cast<uint32_t*>(out) + (o0 >> 5);
-  const bool last_shared = ((lead + (o1 - o0)) & 31) != 0;
-  for (uint32_t j = lane; j < nwords; j += 32) {
+  __syncthreads();
+  // flush: whole words are stored; the first / last word may be shared with the neighbouring CTA
+  uint32_t* gw = reinterpret_cast<uint32_t*>(out) + (start >> 5);
+  const bool last_shared = ((lead + span) & 31) != 0;
+  for (uint32_t j = threadIdx.x; j < nwords; j += kThreads) {
     const uint32_t v = stage[j];
     const bool shared = (j == 0 && lead != 0) || (j == nwords - 1 && last_shared);
     if (shared) atomicOr(gw + j, v);
@@ -409,49 +403,44 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
   }
 }
 
+uint32_t host_elias_len(uint32_t k) {
+  uint32_t len = 1;
+  while (k > 1) {
+    uint32_t m = 0;
+    for (uint32_t t = k; t; t >>= 1) ++m;
+    len += m;
+    k = m - 1;
+  }
+  return len;
+}
+
 template <int LB, bool DENSE>
-int run_pipeline(const BucketParams& bp, const EliasWs& w, uint32_t s, uint8_t* out, size_t out_capacity,
+int run_pipeline(BucketParams& bp, const EliasWs& w, uint32_t s, uint8_t* out, size_t out_capacity,
                  uint64_t* out_bits, uint32_t* status_dev, cudaStream_t stream) {
-  const uint32_t bucket_grid = (uint32_t)((bp.B + kWarps - 1) / kWarps);
-  const uint64_t nblk = (bp.B + kScanBlock - 1) / kScanBlock;
+  const Teams tm = make_teams(bp.d);
+  bp.lpb = tm.lpb; bp.seg = tm.seg; bp.nbc = tm.nbc;
+  const uint64_t ctas = (bp.B + tm.nbc - 1) / tm.nbc;
   {
     ScopedKernel sk(kKernEliasLength, stream);
-    elias_length_kernel<LB, DENSE><<<bucket_grid, kThreads, 0, stream>>>(bp, w.len);
-  }
-  if (bp.B <= kSmallScanMaxBuckets) {
-    ScopedKernel sk(kKernScanSums, stream);
-    scan_small_kernel<<<1, kSmallScanThreads, 0, stream>>>(w.len, bp.B, out_capacity, w.ctrl, out_bits,
-                                                           status_dev, w.off, out);
-  } else {
-    {
-      ScopedKernel sk(kKernScanBlockSums, stream);
-      scan_block_sums_kernel<<<(uint32_t)nblk, kThreads, 0, stream>>>(w.len, bp.B, w.block_sums);
-    }
-    {
-      ScopedKernel sk(kKernScanSums, stream);
-      scan_sums_kernel<<<1, kThreads, 0, stream>>>(w.block_sums, nblk, bp.B, out_capacity, w.ctrl,
-                                                   out_bits, status_dev);
-    }
-    {
-      ScopedKernel sk(kKernScanDownsweep, stream);
-      scan_downsweep_kernel<<<(uint32_t)nblk, kThreads, 0, stream>>>(w.len, bp.B, w.block_sums,
-                                                                     w.ctrl, w.off, out);
-    }
+    elias_length_kernel<LB, DENSE><<<(uint32_t)ctas, kThreads, 0, stream>>>(bp, w.len, w.cta_sums);
   }
   {
-    // staging: the longest legal string of one bucket, plus the shared lead-in word
-    uint32_t elen_max = 1;
-    for (uint32_t k = DENSE ? s + 1 : s; k > 1;) { uint32_t m = 0; for (uint32_t t = k; t; t >>= 1) ++m; elen_max += m; k = m - 1; }
-    const uint32_t per = DENSE ? 1 + elen_max : 2 + elen_max;
-    const uint32_t stage_words = ((32 + bp.d * per + 31) / 32 + 2 + 3) & ~3u;
-    const size_t smem = (size_t)stage_words * 4 * kWarps;
+    ScopedKernel sk(kKernScanSums, stream);
+    scan_sums_kernel<<<1, kScanThreads, 0, stream>>>(w.cta_sums, ctas, bp.B, out_capacity, w.ctrl, out_bits,
+                                                     status_dev, out);
+  }
+  {
+    // staging: the longest legal strings of a CTA's buckets, plus the shared lead-in word
+    const uint32_t per = DENSE ? 1 + host_elias_len(s + 1) : 2 + host_elias_len(s);
+    const size_t run_bits = (size_t)tm.nbc * (32 + (size_t)bp.d * per);
+    const size_t smem = ((run_bits + 31) / 32 + 4) * 4;
     auto kern = elias_scatter_kernel<LB, DENSE>;
     if (smem > 48 * 1024) {
       cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
       if (e != cudaSuccess) return (int)e;
     }
     ScopedKernel sk(kKernEliasScatter, stream);
-    kern<<<bucket_grid, kThreads, smem, stream>>>(bp, w.off, w.ctrl, out, stage_words);
+    kern<<<(uint32_t)ctas, kThreads, smem, stream>>>(bp, w.len, w.cta_sums, w.ctrl, out);
   }
   return (int)cudaGetLastError();
 }
