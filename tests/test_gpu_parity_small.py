@@ -85,3 +85,29 @@ def test_many_peers_and_philox_keying():
     A = O.bucket_scales(g, d, O.NORM_L2)
     err = np.abs(acc / 20 - g)
     assert err.max() < 5 * np.repeat(A, d)[:n].max() / 15 / np.sqrt(20) * 0.5 + 1e-3
+
+
+@pytest.mark.parametrize("K", [1, 5, 16, 33, 40])
+@pytest.mark.parametrize("code_kind", [O.CODE_ELIAS, O.CODE_ELIAS_DENSE])
+def test_elias_peer_counts(K, code_kind):
+    n, d, s = 3 * 512 + 77, 512, 7
+    msgs, infos = [], []
+    for w in range(K):
+        g = make(n, "mix", seed=100 + w)
+        m, info = encode_parity(g, d, s, O.NORM_L2, code_kind, seed=5, step=1, worker=w)
+        msgs.append(m)
+        infos.append(info)
+    decode_parity(msgs, infos, n, d, s, code_kind, eta=0.05, x0=I.gaussian(n, 1.0, seed=9))
+
+
+@pytest.mark.parametrize("d,s", [(4096, 255), (4096, 1), (2048, 15), (1024, 3), (64, 15), (32, 1)])
+def test_elias_bucket_shapes(d, s):
+    n, K = 5 * d + 123, 4
+    for code_kind in (O.CODE_ELIAS, O.CODE_ELIAS_DENSE):
+        msgs, infos = [], []
+        for w in range(K):
+            g = make(n, "gauss", seed=200 + w)
+            m, info = encode_parity(g, d, s, O.NORM_MAX, code_kind, seed=5, step=1, worker=w)
+            msgs.append(m)
+            infos.append(info)
+        decode_parity(msgs, infos, n, d, s, code_kind)
