@@ -424,6 +424,97 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Bandwidth sweep (n = 2^28 unless --n): bucket x levels x norm x code, K peers. One N(0,1)
+    gradient buffer is encoded under K worker ids (K x 1 GiB of distinct gradients is avoided);
+    it is 1 GiB, so every encode reads it HBM-cold. Per point: encode and decode+SGD times (median
+    of 3), GB/s of fp32 gradient, algorithmic GB/s and fraction of the HBM peak."""
+    import torch
+    import paper_1610_02132_b200 as Q
+    from paper_1610_02132_b200 import inputs as I
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    n = args.n or 2 ** 28
+    K = args.K or 16
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except Exception:
+        pass
+    hbm = peaks.get("hbm_gbs") or 6650.0
+    g = I.gaussian_device(n, 1.0, seed=1, device=dev)
+    x = torch.zeros(n, dtype=torch.float32, device=dev)
+    status = Q.new_status(dev)
+    points = []
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    for d in (128, 512, 4096):
+        for s in (1, 3, 15, 255):
+            for norm in ("l2", "max"):
+                for cname in ("fixed", "elias"):
+                    code = CODE[cname]
+                    B = (n + d - 1) // d
+                    MF = fixed_bytes(n, d, s)
+                    cap = MF if code == 0 else min(Q.qsgd_message_capacity(n, d, s, code), 2 * MF + 8 * (B + 1))
+                    msgs = [torch.empty(cap, dtype=torch.uint8, device=dev) for _ in range(K)]
+                    bits = torch.zeros(K, 4, dtype=torch.int64, device=dev)
+                    ws = torch.empty(max(Q.qsgd_workspace_bytes(n, d, s, code), 16), dtype=torch.uint8, device=dev)
+                    t_enc, t_dec, info = [], [], None
+                    for rep in range(4):
+                        torch.cuda.synchronize()
+                        ev[0].record()
+                        for w in range(K):
+                            Q.qsgd_encode(g, d, s, NORM[norm], code, PHILOX_SEED, rep, w, msgs[w], bits[w], ws, status)
+                        ev[1].record()
+                        tables = None
+                        info = bits.cpu().numpy().view(np.uint64)
+                        if code != 0:
+                            nb = 8 * (B + 1)
+                            tables = [msgs[w][int(info[w, 1]): int(info[w, 1]) + nb].view(torch.int64) for w in range(K)]
+                        torch.cuda.synchronize()
+                        ev[1].record()
+                        Q.qsgd_decode_sgd_step(msgs, tables, n, d, s, code, x, ETA, status)
+                        ev[2].record()
+                        torch.cuda.synchronize()
+                        if rep:                                        # first repetition warms up
+                            t_dec.append(ev[1].elapsed_time(ev[2]) * 1e-3)
+                        torch.cuda.synchronize()
+                        ev[0].record()
+                        for w in range(K):
+                            Q.qsgd_encode(g, d, s, NORM[norm], code, PHILOX_SEED, rep, w, msgs[w], bits[w], ws, status)
+                        ev[1].record()
+                        torch.cuda.synchronize()
+                        if rep:
+                            t_enc.append(ev[0].elapsed_time(ev[1]) * 1e-3 / K)
+                    st = int(status.item())
+                    assert st == 0, "device status %d at d=%d s=%d %s %s" % (st, d, s, norm, cname)
+                    te, td = statistics.median(t_enc), statistics.median(t_dec)
+                    M = float(MF) if code == 0 else float(np.mean(info[:, 2].astype(np.float64)))
+                    pay_bits = 8.0 * MF / n if code == 0 else float(np.mean(info[:, 0].astype(np.float64))) / n
+                    points.append({
+                        "d": d, "s": s, "norm": norm, "code": cname,
+                        "bits_per_coord_payload": round(pay_bits, 4), "bits_per_coord_message": round(8 * M / n, 4),
+                        "encode_us": round(te * 1e6, 1), "decode_sgd_us": round(td * 1e6, 1),
+                        "encode_GBps_fp32": round(4 * n / te / 1e9, 1), "decode_sgd_GBps_fp32": round(K * 4 * n / td / 1e9, 1),
+                        "encode_alg_GBps": round((4 * n + M) / te / 1e9, 1),
+                        "decode_alg_GBps": round((K * M + 8 * n) / td / 1e9, 1),
+                        "encode_frac_measured_hbm": round((4 * n + M) / te / 1e9 / hbm, 3),
+                        "decode_frac_measured_hbm": round((K * M + 8 * n) / td / 1e9 / hbm, 3),
+                        "encode_frac_nominal_8000": round((4 * n + M) / te / 1e9 / 8000.0, 3),
+                        "decode_frac_nominal_8000": round((K * M + 8 * n) / td / 1e9 / 8000.0, 3)})
+                    del msgs, ws
+    ref = [p for p in points if (p["d"], p["s"], p["norm"], p["code"]) == (512, 15, "l2", "fixed")][0]
+    value = (2 * K * 4 * n) / (K * ref["encode_us"] * 1e-6 + ref["decode_sgd_us"] * 1e-6) / 1e9
+    print(json.dumps({
+        "metric": "QSGD encode + decode+aggregate throughput, fp32 gradient GB/s", "value": value, "unit": "GB/s",
+        "n_gpus": 1, "steps": 3, "warmup": 1, "ms_per_step": (K * ref["encode_us"] + ref["decode_sgd_us"]) * 1e-3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "sweep: N(0,1), n=%d, K=%d, bucket x s x norm x code; value quoted at d=512, s=15, "
+                               "2-norm, fixed-width" % (n, K), "hbm_peak_GBps": hbm},
+        "points": points}))
+
+
 def run_exchange(args):
     """Algorithm 1 across GPUs: rank = worker. Per step and code kind: encode the local gradient,
     all-gather the K = world-size messages over NCCL, fused decode + aggregate + SGD step."""
@@ -565,7 +656,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS) + ["sweep"])
     ap.add_argument("--n", type=int, default=None)
     ap.add_argument("--d", type=int, default=None)
     ap.add_argument("--s", type=int, default=None)
@@ -591,7 +682,9 @@ def main():
         args.no_e2e = args.no_cpu = True
     else:
         args.warmup = max(args.warmup, 3)
-    if args.exchange:
+    if args.workload == "sweep":
+        run_sweep(args)
+    elif args.exchange:
         run_exchange(args)
     else:
         run_cuda(args)
