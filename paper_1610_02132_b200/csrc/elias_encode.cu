@@ -69,32 +69,112 @@ EliasWs carve(uint8_t* ws, uint64_t n, uint32_t d, uint32_t s) {
   return w;
 }
 
-// Level field of global coordinate i.
+// Code table indexed by the bit length m of the integer (1 .. 16), kept in shared memory so that
+// lanes with different m read it without divergence:
+//   bits 0..7 prefix value P(m), bits 8..15 total code length, bit 17 set for m = 1 (whose code is
+//   the single bit 0: the generic formula would leave a 1 in bit 1, this bit removes it).
+__device__ __forceinline__ void fill_code_table(uint32_t* tab) {
+  const uint32_t m = threadIdx.x;
+  if (m < 17) {
+    uint32_t pv = 0;
+    if (m > 8) pv = (3u << 4) | (m - 1u);
+    else if (m > 4) pv = (2u << 3) | (m - 1u);
+    else if (m > 2) pv = m - 1u;
+    const uint32_t len = m <= 1 ? 1u : m + 1u + elias_prefix_len(m);
+    tab[m] = pv | (len << 8) | (m == 1 ? (2u << 16) : 0u);
+  }
+}
+
+__device__ __forceinline__ uint32_t bit_length(uint32_t k) { return 32u - (uint32_t)__clz((int)k); }
+
+// |Elias(k)| from the table.
+__device__ __forceinline__ uint32_t tab_len(const uint32_t* tab, uint32_t k) {
+  return (tab[bit_length(k)] >> 8) & 0xFFu;
+}
+
+// Elias(k), right-aligned; *len receives its length.
+__device__ __forceinline__ uint32_t tab_code(const uint32_t* tab, uint32_t k, uint32_t* len) {
+  const uint32_t m = bit_length(k);
+  const uint32_t e = tab[m];
+  *len = (e >> 8) & 0xFFu;
+  return ((((e & 0xFFu) << m) | k) << 1) ^ (e >> 16);
+}
+
+// Level field c of a bucket whose level fields start at word pointer lwb.
 template <int LB>
-__device__ __forceinline__ uint32_t level_at(const uint32_t* __restrict__ lw, uint64_t i) {
-  const uint64_t bit = i * LB;
-  return (__ldg(lw + (bit >> 5)) >> (bit & 31)) & ((1u << LB) - 1u);
+__device__ __forceinline__ uint32_t level_at(const uint32_t* __restrict__ lwb, uint32_t c) {
+  const uint32_t bit = c * LB;
+  return (__ldg(lwb + (bit >> 5)) >> (bit & 31)) & ((1u << LB) - 1u);
+}
+
+// Bit j of the result is set iff field j of the level word is nonzero (32 / LB fields).
+template <int LB>
+__device__ __forceinline__ uint32_t nonzero_mask(uint32_t w) {
+  if (LB == 1) return w;
+  if (LB == 2) {
+    uint32_t y = (w | (w >> 1)) & 0x55555555u;
+    y = (y | (y >> 1)) & 0x33333333u;
+    y = (y | (y >> 2)) & 0x0F0F0F0Fu;
+    y = (y | (y >> 4)) & 0x00FF00FFu;
+    return (y | (y >> 8)) & 0xFFFFu;
+  }
+  if (LB == 4) {
+    uint32_t y = w | (w >> 1);
+    y = (y | (y >> 2)) & 0x11111111u;
+    y = (y | (y >> 3)) & 0x03030303u;
+    y = (y | (y >> 6)) & 0x000F000Fu;
+    return (y | (y >> 12)) & 0xFFu;
+  }
+  uint32_t y = w | (w >> 4);
+  y |= y >> 2;
+  y = (y | (y >> 1)) & 0x01010101u;
+  y = (y | (y >> 7)) & 0x00030003u;
+  return (y | (y >> 14)) & 0xFu;
 }
 
 // Walks the nonzero levels of bucket-relative coordinates [c_lo, c_hi) in index order and
-// calls visit(position, level). Whole zero words are skipped.
+// calls visit(position, level). When the range starts on a 32-coordinate boundary (every
+// power-of-two bucket size) it is processed in blocks of 64 coordinates: the nonzero fields of a
+// block are first condensed into a 64-bit mask, so the visiting loop runs once per nonzero of
+// the lane and not once per (word, most loaded lane) pair. Otherwise words are walked one by one.
 template <int LB, typename F>
-__device__ __forceinline__ void for_each_nonzero(const uint32_t* __restrict__ lw, uint64_t base,
-                                                 uint32_t c_lo, uint32_t c_hi, F&& visit) {
+__device__ __forceinline__ void for_each_nonzero(const uint32_t* __restrict__ lwb, uint32_t c_lo,
+                                                 uint32_t c_hi, F&& visit) {
   constexpr uint32_t kMask = (1u << LB) - 1u;
+  constexpr uint32_t kFields = 32u / LB;           // fields per word
+  if ((c_lo & 31u) == 0u) {
+    for (uint32_t c0 = c_lo; c0 < c_hi; c0 += 64u) {
+      const uint32_t* wp = lwb + ((c0 * LB) >> 5);
+      unsigned long long m = 0ull;
+#pragma unroll
+      for (uint32_t j = 0; j < 2u * LB; ++j) {
+        const uint32_t w = (c0 + j * kFields < c_hi) ? __ldg(wp + j) : 0u;
+        m |= (unsigned long long)nonzero_mask<LB>(w) << (j * kFields);
+      }
+      while (m) {
+        const uint32_t pos = c0 + (uint32_t)__ffsll((long long)m) - 1u;
+        m &= m - 1ull;
+        if (pos < c_hi) {
+          const uint32_t bit = pos * LB;
+          visit(pos, (__ldg(lwb + (bit >> 5)) >> (bit & 31u)) & kMask);
+        }
+      }
+    }
+    return;
+  }
   uint32_t c = c_lo;
   while (c < c_hi) {
-    const uint64_t bit = (base + c) * LB;
-    const uint32_t sh = (uint32_t)(bit & 31);
-    uint32_t w = __ldg(lw + (bit >> 5)) >> sh;
+    const uint32_t bit = c * LB;
+    const uint32_t sh = bit & 31u;
+    uint32_t w = __ldg(lwb + (bit >> 5)) >> sh;
     const uint32_t fields = (32u - sh) / LB;
     const uint32_t cnt = min(fields, c_hi - c);
     if (cnt * LB < 32u) w &= (1u << (cnt * LB)) - 1u;
     while (w) {
-      const uint32_t f = (uint32_t)(__ffs((int)w) - 1) / LB;
-      const uint32_t level = (w >> (f * LB)) & kMask;
-      visit(c + f, level);
-      w &= ~(kMask << (f * LB));
+      const uint32_t fb = ((uint32_t)__ffs((int)w) - 1u) & ~(uint32_t)(LB - 1);   // first bit of the field
+      const uint32_t level = (w >> fb) & kMask;
+      visit(c + fb / LB, level);
+      w &= ~(kMask << fb);
     }
     c += cnt;
   }
@@ -107,24 +187,24 @@ struct LaneSummary {
 };
 
 template <int LB>
-__device__ __forceinline__ LaneSummary summarize_sparse(const uint32_t* __restrict__ lw,
-                                                        uint64_t base, uint32_t c_lo,
-                                                        uint32_t c_hi) {
+__device__ __forceinline__ LaneSummary summarize_sparse(const uint32_t* tab, const uint32_t* __restrict__ lwb,
+                                                        uint32_t c_lo, uint32_t c_hi) {
   LaneSummary s{0u, -1, -1};
-  for_each_nonzero<LB>(lw, base, c_lo, c_hi, [&](uint32_t pos, uint32_t level) {
-    if (s.first < 0) s.first = (int32_t)pos;
-    else s.bits += elias_len(pos - (uint32_t)s.last);
-    s.bits += 1u + elias_len(level);
+  for_each_nonzero<LB>(lwb, c_lo, c_hi, [&](uint32_t pos, uint32_t level) {
+    const bool is_first = s.first < 0;
+    const uint32_t gap_bits = tab_len(tab, is_first ? 1u : pos - (uint32_t)s.last);
+    s.first = is_first ? (int32_t)pos : s.first;
+    s.bits += (is_first ? 0u : gap_bits) + 1u + tab_len(tab, level);
     s.last = (int32_t)pos;
   });
   return s;
 }
 
 template <int LB>
-__device__ __forceinline__ uint32_t summarize_dense(const uint32_t* __restrict__ lw, uint64_t base,
+__device__ __forceinline__ uint32_t summarize_dense(const uint32_t* tab, const uint32_t* __restrict__ lwb,
                                                     uint32_t c_lo, uint32_t c_hi) {
   uint32_t bits = 0;
-  for (uint32_t c = c_lo; c < c_hi; ++c) bits += 1u + elias_len(level_at<LB>(lw, base + c) + 1u);
+  for (uint32_t c = c_lo; c < c_hi; ++c) bits += 1u + tab_len(tab, level_at<LB>(lwb, c) + 1u);
   return bits;
 }
 
@@ -152,17 +232,18 @@ struct BucketParams {
 
 // Bits of this lane's part of its bucket's string (the scale's 32 bits go with team lane 0).
 template <int LB, bool DENSE>
-__device__ __forceinline__ uint32_t lane_bits(const BucketParams& p, uint64_t base, uint32_t c_lo,
-                                              uint32_t c_hi, uint32_t tl, bool live, int32_t* prev_out) {
+__device__ __forceinline__ uint32_t lane_bits(const uint32_t* tab, const uint32_t* __restrict__ lwb, uint32_t lpb,
+                                              uint32_t c_lo, uint32_t c_hi, uint32_t tl, bool live,
+                                              int32_t* prev_out) {
   uint32_t bits = 0;
   int32_t prev = -1;
   if (DENSE) {
-    if (live) bits = summarize_dense<LB>(p.level, base, c_lo, c_hi);
+    if (live) bits = summarize_dense<LB>(tab, lwb, c_lo, c_hi);
   } else {
     LaneSummary s{0u, -1, -1};
-    if (live) s = summarize_sparse<LB>(p.level, base, c_lo, c_hi);
-    prev = prev_nonzero_before_lane(s.last, tl, p.lpb);
-    bits = s.bits + (s.first >= 0 ? elias_len((uint32_t)(s.first - prev)) : 0u);
+    if (live) s = summarize_sparse<LB>(tab, lwb, c_lo, c_hi);
+    prev = prev_nonzero_before_lane(s.last, tl, lpb);
+    bits = s.bits + (s.first >= 0 ? tab_len(tab, (uint32_t)(s.first - prev)) : 0u);
   }
   if (live && tl == 0) bits += 32u;
   *prev_out = prev;
@@ -185,6 +266,9 @@ __global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketPara
                                                                 uint32_t* __restrict__ len,
                                                                 uint64_t* __restrict__ cta_sums) {
   __shared__ uint32_t warp_sum[kWarps];
+  __shared__ uint32_t tab[17];
+  fill_code_table(tab);
+  __syncthreads();
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t tl = lane & (p.lpb - 1), team = lane / p.lpb, bpw = 32 / p.lpb;
   const uint64_t b = (uint64_t)blockIdx.x * p.nbc + warp * bpw + team;
@@ -192,8 +276,9 @@ __global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketPara
   const uint64_t base = live ? b * p.d : 0;
   const uint32_t db = live ? (uint32_t)min((uint64_t)p.d, p.n - base) : 0;
   const uint32_t c_lo = min(tl * p.seg, db), c_hi = min(c_lo + p.seg, db);
+  const uint32_t* lwb = p.level + ((base * LB) >> 5);            // the bucket's first level word
   int32_t prev;
-  const uint32_t bits = lane_bits<LB, DENSE>(p, base, c_lo, c_hi, tl, live, &prev);
+  const uint32_t bits = lane_bits<LB, DENSE>(tab, lwb, p.lpb, c_lo, c_hi, tl, live, &prev);
   const uint32_t L = team_sum(bits, p.lpb);
   if (live && tl == 0) len[b] = L;
   uint32_t w = (tl == 0) ? L : 0u;                 // one contribution per bucket
@@ -319,7 +404,9 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
                                                                  uint8_t* __restrict__ out) {
   extern __shared__ uint32_t stage[];
   __shared__ uint32_t warp_sum[kWarps];
+  __shared__ uint32_t tab[17];
   if (!ctrl->ok) return;
+  fill_code_table(tab);
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t tl = lane & (p.lpb - 1), team = lane / p.lpb, bpw = 32 / p.lpb;
   const uint64_t b = (uint64_t)blockIdx.x * p.nbc + warp * bpw + team;
@@ -358,7 +445,9 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
 
   // this lane's first bit inside its bucket: scan of the lane lengths over the team
   int32_t prev;
-  const uint32_t bits = lane_bits<LB, DENSE>(p, base, c_lo, c_hi, tl, live, &prev);
+  const uint32_t* lwb = p.level + ((base * LB) >> 5);            // the bucket's first level word
+  const uint32_t* swb = p.sign + (base >> 5);                    // ... and first sign word
+  const uint32_t bits = lane_bits<LB, DENSE>(tab, lwb, p.lpb, c_lo, c_hi, tl, live, &prev);
   uint32_t linc = bits;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -371,20 +460,18 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
     if (tl == 0) bw.put(__float_as_uint(__ldg(p.A + b)), 32);
     if (DENSE) {
       for (uint32_t c = c_lo; c < c_hi; ++c) {
-        const uint64_t i = base + c;
-        const uint32_t sg = (__ldg(p.sign + (i >> 5)) >> (i & 31)) & 1u;
+        const uint32_t sg = (__ldg(swb + (c >> 5)) >> (c & 31)) & 1u;
         uint32_t ln;
-        const uint32_t code = elias_code(level_at<LB>(p.level, i) + 1u, &ln);
+        const uint32_t code = tab_code(tab, level_at<LB>(lwb, c) + 1u, &ln);
         bw.put((sg << ln) | code, ln + 1);
       }
     } else {
-      for_each_nonzero<LB>(p.level, base, c_lo, c_hi, [&](uint32_t pos, uint32_t level) {
+      for_each_nonzero<LB>(lwb, c_lo, c_hi, [&](uint32_t pos, uint32_t level) {
         uint32_t ln;
-        uint32_t code = elias_code(pos - (uint32_t)prev, &ln);
+        uint32_t code = tab_code(tab, pos - (uint32_t)prev, &ln);
         bw.put(code, ln);
-        const uint64_t i = base + pos;
-        const uint32_t sg = (__ldg(p.sign + (i >> 5)) >> (i & 31)) & 1u;
-        code = elias_code(level, &ln);
+        const uint32_t sg = (__ldg(swb + (pos >> 5)) >> (pos & 31)) & 1u;
+        code = tab_code(tab, level, &ln);
         bw.put((sg << ln) | code, ln + 1);
         prev = (int32_t)pos;
       });
