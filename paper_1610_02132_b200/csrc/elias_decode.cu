@@ -219,35 +219,42 @@ struct FieldParams {
   uint32_t bucket_words;  // K rows + K scales, padded to 4
 };
 
-// Bit source over the payload: 64-bit left-aligned window, one word prefetched.
+// Bit source over the payload: a 64-bit left-aligned window held as two 32-bit halves (all
+// shifts are single funnel-shift instructions), with the next payload word prefetched.
 struct BitSrc {
-  const uint32_t* words;
-  uint64_t widx;     // index of `nextw`
+  const uint32_t* wp;   // payload word the window started in
+  uint32_t idx;         // index (from wp) of `nextw`
   uint32_t nextw;
-  uint64_t win;
-  uint32_t avail;
-  __device__ __forceinline__ void open(const uint32_t* w, uint64_t bit) {
-    words = w;
-    widx = bit >> 5;
-    const uint32_t w0 = __ldg(words + widx), w1 = __ldg(words + widx + 1);
-    nextw = __ldg(words + widx + 2);
+  uint32_t hi, lo;      // window, most significant bit first
+  uint32_t avail;       // valid bits in the window
+  __device__ __forceinline__ void open(const uint32_t* words, uint64_t bit) {
+    wp = words + (bit >> 5);
+    const uint32_t w0 = __ldg(wp), w1 = __ldg(wp + 1);
+    nextw = __ldg(wp + 2);
+    idx = 2;
     const uint32_t sh = (uint32_t)(bit & 31);
-    win = (((uint64_t)w0 << 32) | w1) << sh;
+    hi = __funnelshift_l(w1, w0, sh);
+    lo = w1 << sh;
     avail = 64 - sh;
-    widx += 2;
   }
   __device__ __forceinline__ void refill() {          // afterwards at least 33 valid bits
     if (avail <= 32) {
-      win |= (uint64_t)nextw << (32 - avail);
+      const uint32_t s = 32 - avail;                  // the new word lands s bits above bit 0
+      hi |= __funnelshift_lc(nextw, 0u, s);
+      lo = __funnelshift_lc(0u, nextw, s);
       avail += 32;
-      ++widx;
-      nextw = __ldg(words + widx);
+      ++idx;
+      nextw = __ldg(wp + idx);
     }
   }
-  __device__ __forceinline__ uint32_t take(uint32_t nb) {   // nb in [1, 32]
-    const uint32_t v = (uint32_t)(win >> (64 - nb));
-    win <<= nb;
+  __device__ __forceinline__ void drop(uint32_t nb) {  // nb in [1, 32]
+    hi = __funnelshift_lc(lo, hi, nb);
+    lo = __funnelshift_lc(0u, lo, nb);
     avail -= nb;
+  }
+  __device__ __forceinline__ uint32_t take(uint32_t nb) {   // nb in [1, 32]
+    const uint32_t v = hi >> (32 - nb);
+    drop(nb);
     return v;
   }
   // Definition A.1 decoder on the window; at most three groups (values < 2^16).
@@ -255,40 +262,62 @@ struct BitSrc {
     uint32_t N = 1;
 #pragma unroll
     for (int it = 0; it < 3; ++it) {
-      if (!(win >> 63)) break;
+      if ((int32_t)hi >= 0) break;
       const uint32_t nb = N + 1;
       N = take(nb);
       used += nb;
     }
-    if (win >> 63) return false;
-    take(1);
+    if ((int32_t)hi < 0) return false;
+    drop(1);
     used += 1;
     value = N;
     return true;
   }
 };
 
-// Accumulates field bits for ascending positions and stores a word when the position moves on.
-struct FieldWriter {
-  uint32_t* row;
-  uint32_t cur_idx, cur_val;
-  __device__ __forceinline__ void begin(uint32_t* r) { row = r; cur_idx = 0xFFFFFFFFu; cur_val = 0; }
-  __device__ __forceinline__ void put(uint32_t idx, uint32_t bits) {
-    if (idx != cur_idx) {
-      if (cur_idx != 0xFFFFFFFFu) row[cur_idx] = cur_val;
-      cur_idx = idx;
-      cur_val = 0;
+// Lookup table for the recursive Elias code: entry i (the next 12 stream bits) holds
+// value | length << 8 when those bits start with a complete code of at most 12 bits (every value
+// below 64), else 0. Built once per CTA with the definition's decoder.
+constexpr uint32_t kLutBits = 12;
+
+__device__ __forceinline__ void fill_elias_lut(uint16_t* lut) {
+  for (uint32_t i = threadIdx.x; i < (1u << kLutBits); i += blockDim.x) {
+    uint32_t w = i << (32 - kLutBits), N = 1, used = 0;
+    bool ok = true;
+    for (int it = 0; it < 3 && (w >> 31); ++it) {
+      const uint32_t nb = N + 1;
+      if (used + nb > kLutBits) { ok = false; break; }
+      N = w >> (32 - nb);
+      w <<= nb;
+      used += nb;
     }
-    cur_val |= bits;
+    ok = ok && !(w >> 31) && used + 1 <= kLutBits;
+    lut[i] = ok ? (uint16_t)(N | ((used + 1) << 8)) : (uint16_t)0;
   }
-  __device__ __forceinline__ void end() { if (cur_idx != 0xFFFFFFFFu) row[cur_idx] = cur_val; }
-};
+}
+
+// One Elias integer from the window: table hit in the common case, group loop otherwise.
+__device__ __forceinline__ bool read_int(BitSrc& src, const uint16_t* lut, uint32_t skip, uint32_t& value,
+                                         uint32_t& used) {
+  // `skip` (0 or 1) bits in front of the code are dropped together with it
+  const uint32_t e = lut[(src.hi << skip) >> (32 - kLutBits)];
+  if (e) {
+    const uint32_t nb = (e >> 8) + skip;
+    value = e & 0xFFu;
+    src.drop(nb);
+    used += nb;
+    return true;
+  }
+  if (skip) { src.drop(1); used += 1; }
+  return src.elias(value, used);
+}
 
 template <int LB, bool DENSE>
 __device__ __forceinline__ uint32_t parse_to_fields(const uint32_t* __restrict__ words,
                                                     const uint64_t* __restrict__ table, uint64_t b,
                                                     uint64_t B, uint32_t db, uint32_t d, uint32_t s,
-                                                    uint32_t* __restrict__ row, float* A_out) {
+                                                    const uint16_t* lut, uint32_t* __restrict__ row,
+                                                    float* A_out) {
   const uint64_t lo = __ldg(table + b), hi = __ldg(table + b + 1), all = __ldg(table + B);
   *A_out = 0.f;
   if (hi < lo || hi - lo < 32 || hi > all) return QSGD_DEV_TABLE;
@@ -299,44 +328,39 @@ __device__ __forceinline__ uint32_t parse_to_fields(const uint32_t* __restrict__
   BitSrc src;
   src.open(words, lo);
   *A_out = __uint_as_float(src.take(32));
-  FieldWriter lv, sg;
-  lv.begin(row);
-  sg.begin(row + (d * LB >> 5));
+  uint32_t* srow = row + ((d * LB) >> 5);            // sign bitmap of this peer row
   uint32_t used = 0, err = 0;
+  // The row is zero and only this lane writes it, so fields are OR-ed in place.
   if (DENSE) {
     for (uint32_t c = 0; c < db; ++c) {
       src.refill();
-      const uint32_t neg = src.take(1);
+      const uint32_t neg = src.hi >> 31;
       uint32_t v;
-      if (!src.elias(v, used)) { err = QSGD_DEV_OVERRUN; break; }
-      used += 1;
+      if (!read_int(src, lut, 1u, v, used)) { err = QSGD_DEV_OVERRUN; break; }
       if (used > total) { err = QSGD_DEV_OVERRUN; break; }
       if (v - 1u > s) { err = QSGD_DEV_LEVEL; break; }
       if (v > 1u) {
-        lv.put((c * LB) >> 5, (v - 1u) << ((c * LB) & 31));
-        if (neg) sg.put(c >> 5, 1u << (c & 31));
+        row[(c * LB) >> 5] |= (v - 1u) << ((c * LB) & 31);
+        if (neg) srow[c >> 5] |= 1u << (c & 31);
       }
     }
     if (!err && used != total) err = QSGD_DEV_OVERRUN;
   } else {
-    int32_t at = -1;
+    uint32_t at = 0xFFFFFFFFu;                        // position of the previous nonzero (-1)
     while (used < total) {
       uint32_t gap, level;
       src.refill();
-      if (!src.elias(gap, used) || used >= total) { err = QSGD_DEV_OVERRUN; break; }
-      at += (int32_t)gap;
-      if (at >= (int32_t)db) { err = QSGD_DEV_POSITION; break; }
-      const uint32_t neg = src.take(1);
-      used += 1;
+      if (!read_int(src, lut, 0u, gap, used) || used >= total) { err = QSGD_DEV_OVERRUN; break; }
+      at += gap;
+      if (at >= db) { err = QSGD_DEV_POSITION; break; }
       src.refill();
-      if (!src.elias(level, used) || used > total) { err = QSGD_DEV_OVERRUN; break; }
+      const uint32_t neg = src.hi >> 31;
+      if (!read_int(src, lut, 1u, level, used) || used > total) { err = QSGD_DEV_OVERRUN; break; }
       if (level < 1u || level > s) { err = QSGD_DEV_LEVEL; break; }
-      lv.put(((uint32_t)at * LB) >> 5, level << (((uint32_t)at * LB) & 31));
-      if (neg) sg.put((uint32_t)at >> 5, 1u << ((uint32_t)at & 31));
+      row[(at * LB) >> 5] |= level << ((at * LB) & 31);
+      if (neg) srow[at >> 5] |= 1u << (at & 31);
     }
   }
-  lv.end();
-  sg.end();
   return err;
 }
 
@@ -344,13 +368,16 @@ template <int LB, bool DENSE, bool FUSED, bool SINGLE>
 __global__ void __launch_bounds__(128) decode_elias_fields_kernel(const __grid_constant__ FieldParams p) {
   extern __shared__ __align__(16) uint32_t fsm[];
   __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
+  __shared__ uint16_t elias_lut[1u << kLutBits];
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const float sf = (float)p.s;
   float lut0 = 0.f;
+  fill_elias_lut(elias_lut);
   if (LB == 8) {
     for (uint32_t i = tid; i < 256 * 32; i += blockDim.x) xi_tab[i] = __fdiv_rn((float)(i >> 5), sf);
-    __syncthreads();
-  } else {
+  }
+  __syncthreads();
+  if (LB != 8) {
     const uint32_t level = lane & ((1u << LB) - 1u), neg = (lane >> LB) & 1u;
     const float q = __fdiv_rn((float)level, sf);
     lut0 = neg ? -q : q;
@@ -378,7 +405,7 @@ __global__ void __launch_bounds__(128) decode_elias_fields_kernel(const __grid_c
         const uint32_t db = (uint32_t)min((uint64_t)p.d, p.n - base);
         float A;
         const uint32_t st = parse_to_fields<LB, DENSE>(p.peers.payload[k], p.peers.table[k], b, p.B, db, p.d,
-                                                       p.s, bucket + k * p.row_words, &A);
+                                                       p.s, elias_lut, bucket + k * p.row_words, &A);
         reinterpret_cast<float*>(bucket + p.K * p.row_words)[k] = A;
         if (st) atomicOr(p.status, st);
       }
@@ -445,7 +472,7 @@ int launch_fields(FieldParams& p, bool fused, cudaStream_t stream, bool* handled
   while (G > 1 && (size_t)G * p.bucket_words * 4 > (16u << 10)) G >>= 1;
   p.G = G;
   const size_t per_warp = (size_t)G * p.bucket_words * 4;
-  const size_t budget = (size_t)max_smem - (LB == 8 ? 32768 : 128) - 1024;
+  const size_t budget = (size_t)max_smem - (LB == 8 ? 32768 : 128) - 8192 - 1024;
   int warps = 4;
   while (warps > 1 && (size_t)warps * per_warp > (warps == 4 ? (96u << 10) : budget)) warps >>= 1;
   if ((size_t)warps * per_warp > budget) return 0;               // caller falls back to the slow kernel
