@@ -163,7 +163,7 @@ uint64_t qsgd_launch_count(void);
  *   - code_kind must be QSGD_CODE_ELIAS or QSGD_CODE_ELIAS_DENSE (fixed-width needs no scratch:
  *     use qsgd_encode). Results are bit-identical to qsgd_encode with the same arguments.
  *   - Limit: qsgd_workspace_bytes(n, bucket, s, code_kind) must not exceed
- *     qsgd_static_scratch_bytes(); e.g. bucket 512, s = 15 fits up to about 51 million
+ *     qsgd_static_scratch_bytes(); e.g. bucket 512, s = 15 fits up to about 47 million
  *     coordinates. Larger problems are rejected with QSGD_ERR_SCRATCH and nothing is launched.
  *   - The first call on each device looks up the device address of the built-in array (a host
  *     side query, done with that device current and cached per device). Make that first call

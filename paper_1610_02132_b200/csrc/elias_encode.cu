@@ -50,6 +50,7 @@ Teams make_teams(uint32_t d) {
 struct EliasWs {
   uint8_t* fixed;             // fixed-width intermediate
   uint32_t* len;              // L_b
+  uint32_t* lane_rec;         // per lane of every bucket team: its bits | (previous nonzero + 1) << 16
   uint64_t* cta_sums;         // per scatter CTA: sum of its buckets' lengths, then exclusive prefix
   Ctrl* ctrl;
   size_t bytes;
@@ -62,6 +63,7 @@ EliasWs carve(uint8_t* ws, uint64_t n, uint32_t d, uint32_t s) {
   size_t o = 0;
   w.fixed = ws + o; o += align16(L.total);
   w.len = reinterpret_cast<uint32_t*>(ws + o); o += align16(4 * L.B);
+  w.lane_rec = reinterpret_cast<uint32_t*>(ws + o); o += align16(4 * L.B * tm.lpb);
   const uint64_t ctas = (L.B + tm.nbc - 1) / tm.nbc;
   w.cta_sums = reinterpret_cast<uint64_t*>(ws + o); o += align16(8 * (ctas + 1));
   w.ctrl = reinterpret_cast<Ctrl*>(ws + o); o += align16(sizeof(Ctrl));
@@ -264,6 +266,7 @@ __device__ __forceinline__ uint32_t team_sum(uint32_t v, uint32_t lpb) {
 template <int LB, bool DENSE>
 __global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketParams p,
                                                                 uint32_t* __restrict__ len,
+                                                                uint32_t* __restrict__ lane_rec,
                                                                 uint64_t* __restrict__ cta_sums) {
   __shared__ uint32_t warp_sum[kWarps];
   __shared__ uint32_t tab[17];
@@ -279,6 +282,7 @@ __global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketPara
   const uint32_t* lwb = p.level + ((base * LB) >> 5);            // the bucket's first level word
   int32_t prev;
   const uint32_t bits = lane_bits<LB, DENSE>(tab, lwb, p.lpb, c_lo, c_hi, tl, live, &prev);
+  if (live) lane_rec[b * p.lpb + tl] = bits | ((uint32_t)(prev + 1) << 16);   // reused by the scatter
   const uint32_t L = team_sum(bits, p.lpb);
   if (live && tl == 0) len[b] = L;
   uint32_t w = (tl == 0) ? L : 0u;                 // one contribution per bucket
@@ -399,6 +403,7 @@ struct StageWriter {
 template <int LB, bool DENSE>
 __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketParams p,
                                                                  const uint32_t* __restrict__ len,
+                                                                 const uint32_t* __restrict__ lane_rec,
                                                                  const uint64_t* __restrict__ cta_start,
                                                                  const Ctrl* __restrict__ ctrl,
                                                                  uint8_t* __restrict__ out) {
@@ -447,7 +452,10 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
   int32_t prev;
   const uint32_t* lwb = p.level + ((base * LB) >> 5);            // the bucket's first level word
   const uint32_t* swb = p.sign + (base >> 5);                    // ... and first sign word
-  const uint32_t bits = lane_bits<LB, DENSE>(tab, lwb, p.lpb, c_lo, c_hi, tl, live, &prev);
+  // this lane's share of the string and the nonzero before it were counted by the length kernel
+  const uint32_t rec = live ? __ldg(lane_rec + b * p.lpb + tl) : 0u;
+  const uint32_t bits = rec & 0xFFFFu;
+  prev = (int32_t)(rec >> 16) - 1;
   uint32_t linc = bits;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -509,7 +517,7 @@ int run_pipeline(BucketParams& bp, const EliasWs& w, uint32_t s, uint8_t* out, s
   const uint64_t ctas = (bp.B + tm.nbc - 1) / tm.nbc;
   {
     ScopedKernel sk(kKernEliasLength, stream);
-    elias_length_kernel<LB, DENSE><<<(uint32_t)ctas, kThreads, 0, stream>>>(bp, w.len, w.cta_sums);
+    elias_length_kernel<LB, DENSE><<<(uint32_t)ctas, kThreads, 0, stream>>>(bp, w.len, w.lane_rec, w.cta_sums);
   }
   {
     ScopedKernel sk(kKernScanSums, stream);
@@ -527,7 +535,7 @@ int run_pipeline(BucketParams& bp, const EliasWs& w, uint32_t s, uint8_t* out, s
       if (e != cudaSuccess) return (int)e;
     }
     ScopedKernel sk(kKernEliasScatter, stream);
-    kern<<<(uint32_t)ctas, kThreads, smem, stream>>>(bp, w.len, w.cta_sums, w.ctrl, out);
+    kern<<<(uint32_t)ctas, kThreads, smem, stream>>>(bp, w.len, w.lane_rec, w.cta_sums, w.ctrl, out);
   }
   return (int)cudaGetLastError();
 }
