@@ -134,7 +134,7 @@ int qsgd_encode(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int nor
     const FixedLayout L = make_fixed_layout(n, bucket, s);
     if (out_capacity < L.total) return QSGD_ERR_CAPACITY;
     return launch_quantize_fixed(g, n, bucket, s, norm_kind, seed, step, worker,
-                                 static_cast<uint8_t*>(out), status_dev, out_bits, cs);
+                                 static_cast<uint8_t*>(out), status_dev, out_bits, nullptr, cs);
   }
   if (!workspace) return QSGD_ERR_NULL;
   if (!aligned16(workspace)) return QSGD_ERR_ALIGN;

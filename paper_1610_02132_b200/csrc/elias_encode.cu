@@ -3,8 +3,9 @@
 //   1. quantize into the fixed-width layout held in the workspace (quantize_fixed.cu);
 //   2. string length L_b of every bucket, and the sum of the lengths of each CTA's run of
 //      consecutive buckets (elias_length_kernel);
-//   3. one CTA scans the per-CTA sums, fixes the message geometry, checks the capacity and clears
-//      the few payload words that two CTAs will share (scan_sums_kernel);
+//   3. the CTA of the length kernel that publishes its sum last (an arrival counter, no waiting)
+//      scans the per-CTA sums, fixes the message geometry, checks the capacity and clears the few
+//      payload words that two scatter CTAs will share;
 //   4. each CTA of the scatter kernel derives the bit offsets of its own buckets, writes their
 //      offset-table entries, assembles its run of strings in shared memory (lanes own
 //      consecutive sub-ranges of a bucket; bits of neighbouring lanes and buckets meet inside
@@ -28,7 +29,7 @@ struct Ctrl {                 // control block at the end of the workspace
   uint64_t total_bits;
   uint64_t payload_bytes;
   uint32_t ok;                // 1 when the message fits out_capacity
-  uint32_t pad;
+  uint32_t arrived;           // CTAs of the length kernel that have published their sum
 };
 
 struct Teams {
@@ -222,6 +223,15 @@ __device__ __forceinline__ int32_t prev_nonzero_before_lane(int32_t last, uint32
   return tl == 0 ? -1 : excl;
 }
 
+struct ScanArgs {              // what the last CTA of the length kernel needs for the scan
+  uint64_t ctas;
+  size_t out_capacity;
+  Ctrl* ctrl;
+  uint64_t* out_bits;
+  uint32_t* status_dev;
+  uint8_t* out;
+};
+
 struct BucketParams {
   const float* A;
   const uint32_t* sign;
@@ -262,13 +272,80 @@ __device__ __forceinline__ uint32_t team_sum(uint32_t v, uint32_t lpb) {
   return v;
 }
 
+// ---- scan of the per-CTA sums, run by the CTA of the length kernel that finishes last ------------
+__device__ __forceinline__ uint64_t block_exclusive_scan(uint64_t v, uint64_t* total) {
+  __shared__ uint64_t warp_sums[32];
+  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  uint64_t inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint64_t t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= (uint32_t)o) inc += t;
+  }
+  if (lane == 31) warp_sums[warp] = inc;
+  __syncthreads();
+  uint64_t before = 0, all = 0;
+  for (uint32_t w = 0; w < nwarps; ++w) {
+    const uint64_t t = warp_sums[w];
+    if (w < warp) before += t;
+    all += t;
+  }
+  __syncthreads();
+  *total = all;
+  return before + inc - v;
+}
+
+// In place: cta_sums[c] becomes the first payload bit of CTA c's run, cta_sums[ctas] the payload
+// length. Also: message geometry, capacity check, and zeroes in every payload word that two
+// scatter CTAs share (they OR into those; all other words are stored whole) plus the padding.
+// Called by all threads of one CTA.
+__device__ __forceinline__ void scan_cta_sums(uint64_t* cta_sums, uint64_t ctas, uint64_t B, size_t out_capacity,
+                                              Ctrl* ctrl, uint64_t* out_bits, uint32_t* status_dev, uint8_t* out) {
+  __shared__ uint32_t ok_s;
+  __shared__ uint64_t pay_s;
+  // every thread owns a contiguous chunk of the sums: one block-wide scan in total
+  const uint64_t chunk = (ctas + blockDim.x - 1) / blockDim.x;
+  const uint64_t lo = min((uint64_t)threadIdx.x * chunk, ctas), hi = min(lo + chunk, ctas);
+  uint64_t mine = 0;
+#pragma unroll 8
+  for (uint64_t i = lo; i < hi; ++i) mine += __ldcg(cta_sums + i);
+  uint64_t total;
+  uint64_t run = block_exclusive_scan(mine, &total);
+  if (threadIdx.x == 0) {
+    const uint64_t pay = align16((total + 7) / 8);
+    const uint64_t total_bytes = pay + 8 * (B + 1);
+    const bool ok = total_bytes <= out_capacity;
+    ctrl->total_bits = total;
+    ctrl->payload_bytes = pay;
+    ctrl->ok = ok ? 1u : 0u;
+    out_bits[0] = total; out_bits[1] = pay; out_bits[2] = total_bytes; out_bits[3] = 0;
+    if (!ok) atomicOr(status_dev, QSGD_DEV_CAPACITY);
+    ok_s = ok ? 1u : 0u;
+    pay_s = pay;
+    cta_sums[ctas] = total;
+  }
+  __syncthreads();
+  const bool ok = ok_s != 0;
+  uint32_t* words = reinterpret_cast<uint32_t*>(out);
+#pragma unroll 8
+  for (uint64_t i = lo; i < hi; ++i) {
+    const uint64_t v = __ldcg(cta_sums + i);
+    cta_sums[i] = run;
+    if (ok && (run & 31)) words[run >> 5] = 0u;
+    run += v;
+  }
+  if (ok && threadIdx.x == 0)
+    for (uint64_t w = total >> 5; w < pay_s / 4; ++w) words[w] = 0u;        // tail word + padding
+}
+
 // ---- 2. string length per bucket, sum per CTA ------------------------------------------------------
 template <int LB, bool DENSE>
 __global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketParams p,
                                                                 uint32_t* __restrict__ len,
                                                                 uint32_t* __restrict__ lane_rec,
-                                                                uint64_t* __restrict__ cta_sums) {
+                                                                uint64_t* cta_sums, const ScanArgs sa) {
   __shared__ uint32_t warp_sum[kWarps];
+  __shared__ uint32_t is_last;
   __shared__ uint32_t tab[17];
   fill_code_table(tab);
   __syncthreads();
@@ -295,86 +372,15 @@ __global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketPara
 #pragma unroll
     for (int i = 0; i < kWarps; ++i) s += warp_sum[i];
     cta_sums[blockIdx.x] = s;
-  }
-}
-
-// ---- 3. scan of the per-CTA sums (one CTA) -------------------------------------------------------
-constexpr int kScanThreads = 1024;
-
-__device__ __forceinline__ uint64_t block_exclusive_scan(uint64_t v, uint64_t* total) {
-  __shared__ uint64_t warp_sums[32];
-  const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-  uint64_t inc = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const uint64_t t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= (uint32_t)o) inc += t;
-  }
-  if (lane == 31) warp_sums[warp] = inc;
-  __syncthreads();
-  uint64_t before = 0, all = 0;
-  for (uint32_t w = 0; w < nwarps; ++w) {
-    const uint64_t t = warp_sums[w];
-    if (w < warp) before += t;
-    all += t;
+    // publish, then take a ticket: whoever draws the last one sees every CTA's sum
+    __threadfence();
+    is_last = atomicAdd(&sa.ctrl->arrived, 1u) == gridDim.x - 1u ? 1u : 0u;
   }
   __syncthreads();
-  *total = all;
-  return before + inc - v;
-}
-
-// In place: cta_sums[c] becomes the first payload bit of CTA c's run, cta_sums[ctas] the payload
-// length. Also: message geometry, capacity check, and zeroes in every payload word that two
-// scatter CTAs share (they OR into those; all other words are stored whole) plus the padding.
-__global__ void __launch_bounds__(kScanThreads) scan_sums_kernel(uint64_t* __restrict__ cta_sums,
-                                                                 uint64_t ctas, uint64_t B,
-                                                                 size_t out_capacity, Ctrl* ctrl,
-                                                                 uint64_t* __restrict__ out_bits,
-                                                                 uint32_t* __restrict__ status_dev,
-                                                                 uint8_t* __restrict__ out) {
-  __shared__ uint64_t carry_s;
-  __shared__ uint32_t ok_s;
-  // pass 1: payload length
-  uint64_t mine = 0;
-  for (uint64_t i = threadIdx.x; i < ctas; i += kScanThreads) mine += cta_sums[i];
-  uint64_t total;
-  block_exclusive_scan(mine, &total);
-  if (threadIdx.x == 0) {
-    const uint64_t pay = align16((total + 7) / 8);
-    const uint64_t total_bytes = pay + 8 * (B + 1);
-    const bool ok = total_bytes <= out_capacity;
-    ctrl->total_bits = total;
-    ctrl->payload_bytes = pay;
-    ctrl->ok = ok ? 1u : 0u;
-    out_bits[0] = total; out_bits[1] = pay; out_bits[2] = total_bytes; out_bits[3] = 0;
-    if (!ok) atomicOr(status_dev, QSGD_DEV_CAPACITY);
-    ok_s = ok ? 1u : 0u;
-    carry_s = 0;
-    if (ok) {
-      uint32_t* words = reinterpret_cast<uint32_t*>(out);
-      for (uint64_t w = total >> 5; w < pay / 4; ++w) words[w] = 0u;      // tail word + padding
-    }
+  if (is_last) {
+    __threadfence();
+    scan_cta_sums(cta_sums, sa.ctas, p.B, sa.out_capacity, sa.ctrl, sa.out_bits, sa.status_dev, sa.out);
   }
-  __syncthreads();
-  const bool ok = ok_s != 0;
-  uint32_t* words = reinterpret_cast<uint32_t*>(out);
-  // pass 2: exclusive prefix, in place
-  for (uint64_t base = 0; base < ctas; base += kScanThreads) {
-    const uint64_t i = base + threadIdx.x;
-    const uint64_t v = i < ctas ? cta_sums[i] : 0;
-    uint64_t chunk;
-    const uint64_t ex = block_exclusive_scan(v, &chunk);
-    const uint64_t carry = carry_s;
-    if (i < ctas) {
-      const uint64_t start = carry + ex;
-      cta_sums[i] = start;
-      if (ok && (start & 31)) words[start >> 5] = 0u;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) carry_s = carry + chunk;
-    __syncthreads();
-  }
-  if (threadIdx.x == 0) cta_sums[ctas] = carry_s;
 }
 
 // ---- 4. scatter ----------------------------------------------------------------------------------
@@ -516,13 +522,11 @@ int run_pipeline(BucketParams& bp, const EliasWs& w, uint32_t s, uint8_t* out, s
   bp.lpb = tm.lpb; bp.seg = tm.seg; bp.nbc = tm.nbc;
   const uint64_t ctas = (bp.B + tm.nbc - 1) / tm.nbc;
   {
+    ScanArgs sa;
+    sa.ctas = ctas; sa.out_capacity = out_capacity; sa.ctrl = w.ctrl; sa.out_bits = out_bits;
+    sa.status_dev = status_dev; sa.out = out;
     ScopedKernel sk(kKernEliasLength, stream);
-    elias_length_kernel<LB, DENSE><<<(uint32_t)ctas, kThreads, 0, stream>>>(bp, w.len, w.lane_rec, w.cta_sums);
-  }
-  {
-    ScopedKernel sk(kKernScanSums, stream);
-    scan_sums_kernel<<<1, kScanThreads, 0, stream>>>(w.cta_sums, ctas, bp.B, out_capacity, w.ctrl, out_bits,
-                                                     status_dev, out);
+    elias_length_kernel<LB, DENSE><<<(uint32_t)ctas, kThreads, 0, stream>>>(bp, w.len, w.lane_rec, w.cta_sums, sa);
   }
   {
     // staging: the longest legal strings of a CTA's buckets, plus the shared lead-in word
@@ -551,7 +555,8 @@ int launch_elias_encode(const float* g, uint64_t n, uint32_t d, uint32_t s, int 
                         size_t out_capacity, uint64_t* out_bits, uint8_t* workspace,
                         uint32_t* status_dev, cudaStream_t stream) {
   const EliasWs w = carve(workspace, n, d, s);
-  int st = launch_quantize_fixed(g, n, d, s, norm_kind, seed, step, worker, w.fixed, status_dev, nullptr, stream);
+  int st = launch_quantize_fixed(g, n, d, s, norm_kind, seed, step, worker, w.fixed, status_dev, nullptr,
+                                 &w.ctrl->arrived, stream);
   if (st) return st;
   const FixedLayout L = make_fixed_layout(n, d, s);
   BucketParams bp;

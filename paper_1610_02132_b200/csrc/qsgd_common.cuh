@@ -94,7 +94,7 @@ struct PeerSet {                 // K messages, resolved to region pointers on t
 
 int launch_quantize_fixed(const float* g, uint64_t n, uint32_t d, uint32_t s, int norm_kind,
                           uint64_t seed, uint32_t step, uint32_t worker, uint8_t* out,
-                          uint32_t* status_dev, uint64_t* info, cudaStream_t stream);
+                          uint32_t* status_dev, uint64_t* info, uint32_t* clear_word, cudaStream_t stream);
 
 int launch_decode_fixed(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s,
                         float* acc_or_x, bool fused, float eta, cudaStream_t stream);

@@ -44,6 +44,7 @@ struct QuantizeParams {
   uint32_t* status;
   uint64_t* info;         // optional: the four message-info words of a fixed-width message
   uint64_t total_bytes;
+  uint32_t* clear_word;   // optional: a word the kernel sets to zero (arrival counter of a later kernel)
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -172,10 +173,19 @@ struct FastParams {
   uint32_t* status;
   uint64_t* info;           // optional message-info words, written by CTA 0
   uint64_t total_bytes;
+  uint32_t* clear_word;     // optional word set to zero by CTA 0
   PhiloxConsts pc;
+  uint32_t main_ctas;       // CTAs that stream complete tiles
+  QuantizeParams tail;      // parameters of the extra CTA (used when gridDim.x > main_ctas)
 };
 
+template <int LB, int NORM>
+__device__ __forceinline__ void quantize_generic_tile(const QuantizeParams& p, uint32_t block, uint32_t nblocks,
+                                                      float* tile, float* part, float* s_rcp);
+
 // CROSS: a bucket spans several warps (d >= 1024); otherwise a bucket is d / 16 <= 32 lanes.
+// CTAs 0 .. main_ctas - 1 stream the complete tiles; one optional extra CTA runs the ragged last
+// tile and the region padding through the generic tile code (its operands alias the tile ring).
 template <int LB, int NORM, bool CROSS>
 __global__ void __launch_bounds__(kThreads, 4)
 quantize_pow2_kernel(const __grid_constant__ FastParams p) {
@@ -183,7 +193,11 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
   TileSmem& sm = *reinterpret_cast<TileSmem*>(smem_raw);
 
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint32_t grid = gridDim.x;
+  const uint32_t grid = p.main_ctas;
+  if (blockIdx.x >= grid) {                     // the extra CTA: ragged tail + padding
+    quantize_generic_tile<LB, NORM>(p.tail, 0u, 1u, sm.tile[0], sm.tile[1], sm.tile[1] + 1024);
+    return;
+  }
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(&sm.full[s], 1);
@@ -196,6 +210,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
     if (blockIdx.x == 0 && p.info) {
       p.info[0] = 8 * p.total_bytes; p.info[1] = 0; p.info[2] = p.total_bytes; p.info[3] = 0;
     }
+    if (blockIdx.x == 0 && p.clear_word) *p.clear_word = 0u;
     for (int s = 0; s < kStages; ++s) {
       const uint32_t t = blockIdx.x + (uint32_t)s * grid;
       if (t < p.full_tiles) {
@@ -380,17 +395,17 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
 constexpr int kGroupsPerThread = kTile / 8 / kThreads;  // 2
 constexpr int kMaxBucketsPerTile = kTile / 32;          // 128
 
+// One tile of the generic path. `block` / `nblocks` play the role of blockIdx / gridDim so that the
+// main kernel can run the ragged last tile in one extra CTA of its own grid.
 template <int LB, int NORM>
-__global__ void __launch_bounds__(kThreads) quantize_generic_kernel(const QuantizeParams p) {
-  __shared__ __align__(16) float tile[kTile];
-  __shared__ float part[kTile / 8];
-  __shared__ float s_rcp[kMaxBucketsPerTile];
-
+__device__ __forceinline__ void quantize_generic_tile(const QuantizeParams& p, uint32_t block, uint32_t nblocks,
+                                                      float* tile, float* part, float* s_rcp) {
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const uint64_t t0 = p.coord_base + (uint64_t)blockIdx.x * p.tile_coords;   // first coordinate
-  if (blockIdx.x == 0 && tid == 0 && p.info) {
+  const uint64_t t0 = p.coord_base + (uint64_t)block * p.tile_coords;   // first coordinate
+  if (block == 0 && tid == 0 && p.info) {
     p.info[0] = 8 * p.total_bytes; p.info[1] = 0; p.info[2] = p.total_bytes; p.info[3] = 0;
   }
+  if (block == 0 && tid == 0 && p.clear_word) *p.clear_word = 0u;
   const uint64_t left = p.n - t0;
   const uint32_t valid = left < p.tile_coords ? (uint32_t)left : p.tile_coords;
   if (valid == 0) {                            // nothing left to encode: only the padding
@@ -535,11 +550,19 @@ __global__ void __launch_bounds__(kThreads) quantize_generic_kernel(const Quanti
     }
   }
 
-  if (blockIdx.x == gridDim.x - 1 && tid < 4) {
+  if (block == nblocks - 1 && tid < 4) {
     if (p.B + tid < ((p.B + 3) & ~3ull)) p.A_out[p.B + tid] = 0.f;
     if (p.sign_words + tid < ((p.sign_words + 3) & ~3ull)) p.sign_out[p.sign_words + tid] = 0u;
     if (p.level_words + tid < ((p.level_words + 3) & ~3ull)) p.level_out[p.level_words + tid] = 0u;
   }
+}
+
+template <int LB, int NORM>
+__global__ void __launch_bounds__(kThreads) quantize_generic_kernel(const QuantizeParams p) {
+  __shared__ __align__(16) float tile[kTile];
+  __shared__ float part[kTile / 8];
+  __shared__ float s_rcp[kMaxBucketsPerTile];
+  quantize_generic_tile<LB, NORM>(p, blockIdx.x, gridDim.x, tile, part, s_rcp);
 }
 
 PhiloxConsts make_philox_consts(uint64_t seed, uint32_t step, uint32_t worker) {
@@ -560,7 +583,7 @@ PhiloxConsts make_philox_consts(uint64_t seed, uint32_t step, uint32_t worker) {
 }
 
 template <int LB, int NORM, bool CROSS>
-int launch_fast(const FastParams& fp, cudaStream_t stream) {
+int launch_fast(FastParams& fp, bool with_tail, cudaStream_t stream) {
   static int ctas_per_sm = 0, sms = 0;
   auto kern = quantize_pow2_kernel<LB, NORM, CROSS>;
   const size_t smem = sizeof(TileSmem) + 128;
@@ -576,9 +599,9 @@ int launch_fast(const FastParams& fp, cudaStream_t stream) {
     ctas_per_sm = occ > 0 ? occ : 1;
   }
   const uint32_t cap = (uint32_t)(sms * ctas_per_sm);
-  const uint32_t grid = fp.full_tiles < cap ? fp.full_tiles : cap;
+  fp.main_ctas = fp.full_tiles < cap ? fp.full_tiles : cap;
   ScopedKernel sk(kKernQuantize, stream);
-  kern<<<grid, kThreads, smem, stream>>>(fp);
+  kern<<<fp.main_ctas + (with_tail ? 1u : 0u), kThreads, smem, stream>>>(fp);
   return (int)cudaGetLastError();
 }
 
@@ -594,17 +617,22 @@ int launch_one(QuantizeParams& p, uint64_t seed, cudaStream_t stream) {
     fp.log2d = 0;
     while ((1u << fp.log2d) < d) ++fp.log2d;
     fp.A_out = p.A_out; fp.sign_out = p.sign_out; fp.level_out = p.level_out; fp.status = p.status;
-    fp.info = p.info; fp.total_bytes = p.total_bytes;
+    fp.info = p.info; fp.total_bytes = p.total_bytes; fp.clear_word = p.clear_word;
     fp.pc = make_philox_consts(seed, p.step, p.worker);
-    const int st = d >= 1024 ? launch_fast<LB, NORM, true>(fp, stream) : launch_fast<LB, NORM, false>(fp, stream);
-    if (st) return st;
+    // the ragged tail (fewer than 4096 coordinates) and the zero padding of the three regions go
+    // to one extra CTA of the same launch; nothing to do when n is a multiple of the tile and
+    // every region already ends on a 16-byte boundary
+    p.coord_base = (uint64_t)full_tiles * kTile;
+    const bool with_tail = !(p.n == p.coord_base && ((p.B | p.sign_words | p.level_words) & 3ull) == 0);
+    fp.tail = p;
+    fp.tail.info = nullptr;
+    fp.tail.clear_word = nullptr;
+    return d >= 1024 ? launch_fast<LB, NORM, true>(fp, with_tail, stream)
+                     : launch_fast<LB, NORM, false>(fp, with_tail, stream);
   }
-  // whatever is left (a ragged tail, or everything when the fast path does not apply), and the
-  // zero padding of the three regions
-  p.coord_base = (uint64_t)full_tiles * kTile;
-  const uint64_t rem = p.n - p.coord_base;
-  if (full_tiles > 0 && rem == 0 && ((p.B | p.sign_words | p.level_words) & 3ull) == 0)
-    return (int)cudaGetLastError();                 // no ragged tail and no padding to write
+  // the fast path does not apply: everything through the generic kernel
+  p.coord_base = 0;
+  const uint64_t rem = p.n;
   uint64_t tiles = (rem + p.tile_coords - 1) / p.tile_coords;
   if (tiles == 0) tiles = 1;
   {
@@ -624,7 +652,7 @@ int launch_lb(QuantizeParams& p, int norm_kind, uint64_t seed, cudaStream_t stre
 
 int launch_quantize_fixed(const float* g, uint64_t n, uint32_t d, uint32_t s, int norm_kind,
                           uint64_t seed, uint32_t step, uint32_t worker, uint8_t* out,
-                          uint32_t* status_dev, uint64_t* info, cudaStream_t stream) {
+                          uint32_t* status_dev, uint64_t* info, uint32_t* clear_word, cudaStream_t stream) {
   const FixedLayout L = make_fixed_layout(n, d, s);
   QuantizeParams p;
   p.g = g; p.n = n; p.d = d; p.s = s;
@@ -639,6 +667,7 @@ int launch_quantize_fixed(const float* g, uint64_t n, uint32_t d, uint32_t s, in
   p.status = status_dev;
   p.info = info;
   p.total_bytes = L.total;
+  p.clear_word = clear_word;
   switch (L.lb) {
     case 1: return launch_lb<1>(p, norm_kind, seed, stream);
     case 2: return launch_lb<2>(p, norm_kind, seed, stream);
