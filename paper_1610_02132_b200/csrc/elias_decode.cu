@@ -347,18 +347,38 @@ __device__ __forceinline__ uint32_t parse_to_fields(const uint32_t* __restrict__
     if (!err && used != total) err = QSGD_DEV_OVERRUN;
   } else {
     uint32_t at = 0xFFFFFFFFu;                        // position of the previous nonzero (-1)
-    while (used < total) {
-      uint32_t gap, level;
+    while (used < total && err == 0u) {
+      // One refill leaves >= 33 bits: enough for a table-decoded triple (<= 12 + 1 + 12 bits).
       src.refill();
-      if (!read_int(src, lut, 0u, gap, used) || used >= total) { err = QSGD_DEV_OVERRUN; break; }
+      uint32_t gap, level, neg;
+      const uint32_t e1 = lut[src.hi >> (32 - kLutBits)];
+      if (e1) {
+        gap = e1 & 0xFFu;
+        src.drop(e1 >> 8);
+        used += e1 >> 8;
+      } else {
+        if (!src.elias(gap, used)) { err = QSGD_DEV_OVERRUN; break; }
+        src.refill();
+      }
+      neg = src.hi >> 31;
+      const uint32_t e2 = lut[(src.hi << 1) >> (32 - kLutBits)];
+      if (e2) {
+        level = e2 & 0xFFu;
+        src.drop((e2 >> 8) + 1u);
+        used += (e2 >> 8) + 1u;
+      } else {
+        src.drop(1);
+        used += 1;
+        if (!src.elias(level, used)) { err = QSGD_DEV_OVERRUN; break; }
+      }
       at += gap;
-      if (at >= db) { err = QSGD_DEV_POSITION; break; }
-      src.refill();
-      const uint32_t neg = src.hi >> 31;
-      if (!read_int(src, lut, 1u, level, used) || used > total) { err = QSGD_DEV_OVERRUN; break; }
-      if (level < 1u || level > s) { err = QSGD_DEV_LEVEL; break; }
-      row[(at * LB) >> 5] |= level << ((at * LB) & 31);
-      if (neg) srow[at >> 5] |= 1u << (at & 31);
+      err |= at >= db ? QSGD_DEV_POSITION : 0u;
+      err |= (level < 1u || level > s) ? QSGD_DEV_LEVEL : 0u;
+      err |= used > total ? QSGD_DEV_OVERRUN : 0u;
+      if (err == 0u) {
+        row[(at * LB) >> 5] |= level << ((at * LB) & 31);
+        srow[at >> 5] |= neg << (at & 31);
+      }
     }
   }
   return err;
