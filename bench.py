@@ -228,9 +228,9 @@ def kernel_algorithmic_bytes(hp, code_name):
         info = hp.info[1]
         msg = float(np.mean(info[:, 2].astype(np.float64)))
         pay = float(np.mean(info[:, 1].astype(np.float64)))
-        out.update({"decode_elias": K * msg + 8 * n, "elias_scatter": MF + pay,
-                    "elias_length": MF - 4 * ((n + 31) // 32) + 4 * B, "zero_payload": pay,
-                    "scan_block_sums": 4 * B, "scan_downsweep": 4 * B + 16 * (B + 1)})
+        out.update({"decode_elias": K * msg + 8 * n, "decode_elias_sparse": K * msg + 8 * n,
+                    "elias_scatter": MF + pay + 8 * (B + 1),
+                    "elias_length": MF - 4 * ((n + 31) // 32) + 4 * B})
     return out
 
 

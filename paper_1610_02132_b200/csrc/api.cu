@@ -33,9 +33,8 @@ ScopedKernel::~ScopedKernel() {
 }
 
 static const char* const kKernelNames[kKernCount] = {
-    "quantize_fixed", "quantize_tail", "fixed_info", "decode_fixed", "sgd_step", "elias_length",
-    "scan_block_sums", "scan_sums", "scan_downsweep", "zero_payload", "elias_scatter",
-    "decode_elias"};
+    "quantize_fixed", "quantize_tail", "decode_fixed", "sgd_step", "elias_length",
+    "elias_scatter", "decode_elias", "decode_elias_sparse"};
 
 namespace {
 

@@ -33,7 +33,42 @@ struct EliasDecodeParams {
   float c;             // eta / K
   uint32_t* status;
   uint32_t warp_bytes; // shared memory per warp
+  uint32_t defer_sparse;  // a sparse-regime kernel was launched beside this one
 };
+
+// Work split of the sparse-regime decoder (defined further down): a warp owns G = 32 / Kpad buckets
+// and walks each in ranges of R positions; a (bucket, peer) list holds the C entries of one range.
+struct SparseShape {
+  uint32_t Kpad;      // lanes per bucket: K rounded up to a power of two
+  uint32_t G;         // buckets per warp
+  uint32_t R;         // positions per range; G * R <= 2048 sums per warp
+  uint32_t C;         // entries per list and range
+  uint32_t ranges;    // ceil(d / R)
+};
+
+__host__ __device__ inline SparseShape sparse_shape(uint32_t K, uint32_t d) {
+  SparseShape sh;
+  sh.Kpad = 1;
+  while (sh.Kpad < K && sh.Kpad < 32u) sh.Kpad <<= 1;
+  sh.G = 32u / sh.Kpad;
+  sh.R = 2048u / sh.G;                     // a power of two, >= 64
+  if (d <= sh.R) sh.R = d;                 // whole bucket in one range
+  sh.C = sh.R / 32u > 16u ? sh.R / 32u : 16u;
+  sh.ranges = (d + sh.R - 1) / sh.R;
+  return sh;
+}
+
+// Strings short enough for the entry-list decoder? True when the average string carries fewer than
+// 8 bits per list slot beyond its scale: an entry of a sparse bucket costs 11 to 14 bits, so lists
+// then fill to about 60 % on average and rarely overflow. Same answer in every thread of every
+// kernel that asks.
+__device__ __forceinline__ bool sparse_regime(const PeerSet& peers, uint32_t K, uint64_t B, uint32_t d) {
+  if (K > 32u) return false;
+  const SparseShape sh = sparse_shape(K, d);
+  uint64_t bits = 0;
+  for (uint32_t k = 0; k < K; ++k) bits += __ldg(peers.table[k] + B);
+  return bits < (uint64_t)K * B * (32ull + 8ull * sh.C * sh.ranges);
+}
 
 template <typename CodeT> struct CodeTraits;
 template <> struct CodeTraits<uint8_t> { static constexpr uint32_t kSignBit = 0x80u; };
@@ -85,6 +120,7 @@ template <typename CodeT, bool DENSE, bool FUSED>
 __global__ void __launch_bounds__(kThreads) decode_elias_slow_kernel(const __grid_constant__ EliasDecodeParams p) {
   extern __shared__ __align__(16) uint8_t smem[];
   __shared__ float xi[256];
+  if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const float sf = (float)p.s;
   for (uint32_t l = threadIdx.x; l < 256; l += kThreads) xi[l] = __fdiv_rn((float)l, sf);
   __syncthreads();
@@ -217,6 +253,7 @@ struct FieldParams {
   uint32_t* status;
   uint32_t row_words;   // per peer row: d * lb / 32 level words, then d / 32 sign words (padded to 4)
   uint32_t bucket_words;  // K rows + K scales, padded to 4
+  uint32_t defer_sparse;  // a sparse-regime kernel was launched beside this one
 };
 
 // Bit source over the payload: a 64-bit left-aligned window held as two 32-bit halves (all
@@ -384,11 +421,303 @@ __device__ __forceinline__ uint32_t parse_to_fields(const uint32_t* __restrict__
   return err;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Sparse-regime decoder (Section 3.1, "Sparse Regime": few nonzeros per bucket). When the strings
+// are short the work should follow the nonzeros, not the coordinates. A warp owns G buckets; lane
+// (bucket, peer) walks that peer's string of that bucket once, range by range: for each range of
+// R positions it lists the (position, sign, level) entries that fall into it, the K lists of a
+// bucket are then added in ascending k into a tile of R sums by the bucket's lanes (entries of one
+// list hit distinct positions), and the tile is written out and re-zeroed. An entry past the range
+// waits in a register for its range; a list that overflows is continued by its own lane at its
+// turn in the k order, adding straight into the tile. In the fused step, groups of four
+// coordinates whose sums are all +0 are left untouched: for c >= 0, x - c * (+0) is x bit for bit.
+//
+// The regime is decided on the device from the payload lengths (no host synchronisation): this
+// kernel and the field-rebuilding kernel are launched back to back, each evaluates the same
+// predicate, and exactly one of them does the work.
+// ------------------------------------------------------------------------------------------------
+struct SparseParams {
+  PeerSet peers;
+  uint32_t K;
+  SparseShape sh;
+  uint64_t n;
+  uint32_t d;
+  uint32_t s;
+  uint64_t B;
+  float* out;
+  float c;
+  uint32_t* status;
+  uint32_t warp_words;   // shared-memory words per warp: G * R sums, 64 of scales and counts, 32 lists
+  uint32_t quad_shift;   // log2(R / 4) when R is a power of two, else 32
+};
+
+// The recursive Elias code (Definition A.1) of one integer below 2^16, decoded without branches
+// from the next 32 stream bits (most significant first): "0" is 1; otherwise up to three groups
+// follow, each one bit longer than the value of the one before and starting with a 1, closed by a
+// 0. Returns false when a fourth group starts.
+__device__ __forceinline__ bool elias_from_window(uint32_t w, uint32_t& value, uint32_t& len) {
+  const uint32_t c0 = w >> 31;
+  const uint32_t n1 = w >> 30;                       // first group: 2 bits
+  uint32_t r = w << 2;
+  const uint32_t c1 = r >> 31;
+  const uint32_t l2 = n1 + 1u;                       // second group: 3 or 4 bits
+  const uint32_t n2 = r >> (32u - l2);
+  r <<= l2;
+  const uint32_t c2 = r >> 31;
+  const uint32_t l3 = n2 + 1u;                       // third group: up to 16 bits
+  const uint32_t n3 = r >> (32u - l3);
+  r <<= l3;
+  const uint32_t c3 = r >> 31;
+  value = c0 ? (c1 ? (c2 ? n3 : n2) : n1) : 1u;
+  len = c0 ? (c1 ? (c2 ? 3u + l2 + l3 : 3u + l2) : 3u) : 1u;
+  return !(c0 & c1 & c2 & c3);
+}
+
+constexpr uint32_t kNoEntry = 0xFFFFFFFFu;           // entries are position | level << 16 | negative << 31
+
+struct LaneParse {           // one peer's string of one bucket, mid-parse
+  BitSrc src;
+  uint32_t used, total;      // bits consumed / bits of the string after its scale
+  uint32_t at;               // position of the last decoded nonzero (-1 before the first)
+  uint32_t err;
+  uint32_t pend;             // decoded entry that has not been delivered yet, or kNoEntry
+};
+
+// Delivers, in order, the entries with position < rend, at most `limit` of them; sink(index within
+// this call, entry). Stops early at the end of the string or at an error. Every decode consumes at
+// least three bits of a string whose length is known, so the loop is bounded.
+template <typename F>
+__device__ __forceinline__ uint32_t advance(LaneParse& st, uint32_t rend, uint32_t limit, uint32_t db, uint32_t s,
+                                            F&& sink) {
+  uint32_t n = 0;
+  for (;;) {
+    if (st.pend != kNoEntry) {
+      if ((st.pend & 0xFFFFu) >= rend || n >= limit) break;
+      sink(n, st.pend);
+      ++n;
+      st.pend = kNoEntry;
+    }
+    if (st.used >= st.total || st.err != 0u) break;
+    uint32_t gap, level, len;
+    st.src.refill();                                  // >= 33 valid bits: a code takes at most 23
+    bool ok = elias_from_window(st.src.hi, gap, len);
+    st.src.drop(len);
+    st.used += len;
+    st.src.refill();
+    const uint32_t neg = st.src.hi >> 31;
+    ok &= elias_from_window(st.src.hi << 1, level, len);
+    st.src.drop(len + 1u);
+    st.used += len + 1u;
+    st.at += gap;
+    st.err |= ok ? 0u : QSGD_DEV_OVERRUN;
+    st.err |= st.at >= db ? QSGD_DEV_POSITION : 0u;
+    st.err |= level > s ? QSGD_DEV_LEVEL : 0u;
+    st.err |= st.used > st.total ? QSGD_DEV_OVERRUN : 0u;
+    if (st.err == 0u) st.pend = st.at | (level << 16) | (neg << 31);
+  }
+  return n;
+}
+
+template <bool FUSED>
+__global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __grid_constant__ SparseParams p) {
+  extern __shared__ __align__(16) uint32_t ssm[];
+  __shared__ float xi[256];
+  if (!sparse_regime(p.peers, p.K, p.B, p.d)) return;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const uint32_t G = p.sh.G, Kpad = p.sh.Kpad, R = p.sh.R, C = p.sh.C;
+  for (uint32_t i = tid; i < 256; i += blockDim.x) xi[i] = __fdiv_rn((float)i, (float)p.s);
+  // per warp: G tiles of R sums | 32 scales | 32 counts | 32 lists of C entries
+  uint32_t* mine = ssm + (size_t)warp * p.warp_words;
+  float* tile = reinterpret_cast<float*>(mine);
+  float4* tile4 = reinterpret_cast<float4*>(mine);
+  float* scales = reinterpret_cast<float*>(mine + G * R);
+  uint32_t* counts = mine + G * R + 32;
+  uint32_t* lists = mine + G * R + 64;
+  for (uint32_t q = lane; q < ((G * R) >> 2); q += 32) tile4[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+  __syncthreads();
+
+  const uint32_t pg = lane / Kpad, pk = lane % Kpad;           // this lane's bucket in the group and peer
+  float* sums = tile + pg * R;                                 // its bucket's tile
+  uint32_t* list = lists + lane * C;
+  const bool skip_zero = FUSED && p.c >= 0.f;                  // x - c * (+0) == x
+  const uint64_t groups = (p.B + G - 1) / G;
+  const uint32_t tile_quads = R >> 2;
+  constexpr uint32_t kMore = 0x80000000u;
+  constexpr int kU = 8;                                        // quads per lane in flight when writing out
+
+  for (uint64_t grp = (uint64_t)blockIdx.x * nwarps + warp; grp < groups; grp += (uint64_t)gridDim.x * nwarps) {
+    const uint64_t b0 = grp * G;
+    // ---- open this lane's string ---------------------------------------------------------------
+    LaneParse st;
+    st.used = st.total = st.err = 0u;
+    st.at = 0xFFFFFFFFu;
+    st.pend = kNoEntry;
+    uint32_t db = 0;                                           // coordinates of this lane's bucket
+    float A = 0.f;
+    if (b0 + pg < p.B) db = (uint32_t)min((uint64_t)p.d, p.n - (b0 + pg) * p.d);
+    const bool parsing = db != 0u && pk < p.K;
+    if (parsing) {
+      const uint64_t b = b0 + pg;
+      const uint32_t* words = p.peers.payload[pk];
+      const uint64_t* table = p.peers.table[pk];
+      const uint64_t lo = __ldg(table + b), hi = __ldg(table + b + 1), all = __ldg(table + p.B);
+      const uint64_t cap_bits = (uint64_t)((const uint8_t*)table - (const uint8_t*)words) * 8ull;
+      if (hi < lo || hi - lo < 32 || hi > all) st.err = QSGD_DEV_TABLE;
+      else if ((const uint8_t*)table > (const uint8_t*)words && all > cap_bits) st.err = QSGD_DEV_TABLE;
+      else if (hi - lo > 32ull + (uint64_t)db * 40ull) st.err = QSGD_DEV_OVERRUN;   // longer than any legal string
+      else {
+        st.total = (uint32_t)(hi - lo) - 32u;
+        st.src.open(words, lo);
+        A = __uint_as_float(st.src.take(32));
+      }
+    }
+    scales[lane] = A;
+
+    for (uint32_t rbeg = 0; rbeg < p.d; rbeg += R) {
+      const uint32_t rend = min(rbeg + R, p.d);
+      // ---- phase 1: list the entries of this range -------------------------------------------
+      uint32_t mycnt = 0;
+      if (parsing) {
+        mycnt = advance(st, rend, C, db, p.s, [&](uint32_t e, uint32_t en) { list[e] = en; });
+        if (st.pend != kNoEntry && (st.pend & 0xFFFFu) < rend) mycnt |= kMore;
+      }
+      counts[lane] = mycnt;
+      __syncwarp();
+      // ---- phase 2: each bucket's lanes add its lists in ascending k -------------------------
+      for (uint32_t k = 0; k < p.K; ++k) {
+        const uint32_t owner = pg * Kpad + k;
+        const float Ak = scales[owner];
+        const uint32_t cnt = counts[owner];
+        const bool bad = !(fabsf(Ak) <= 3.402823466e+38f);    // inf or NaN scale: A * 0 is NaN everywhere
+        const bool odd = __any_sync(0xffffffffu, bad || (cnt & kMore) != 0u);   // warp-uniform
+        if (odd) {
+          if (bad) {
+            const float z = __fmul_rn(Ak, 0.f);
+            for (uint32_t i = rbeg + pk; i < min(rend, db); i += Kpad) sums[i - rbeg] = __fadd_rn(sums[i - rbeg], z);
+          }
+          __syncwarp();
+        }
+        const uint32_t* lk = lists + owner * C;
+        for (uint32_t e = pk; e < (cnt & ~kMore); e += Kpad) {
+          const uint32_t en = lk[e];
+          const float v = __fmul_rn(Ak, xi[(en >> 16) & 0xFFu]);
+          float* cell = sums + ((en & 0xFFFFu) - rbeg);
+          *cell = __fadd_rn(*cell, (int32_t)en < 0 ? -v : v);
+        }
+        __syncwarp();
+        if (odd) {                                           // rest of a long list, by its own lane
+          if (lane == owner && (cnt & kMore)) {
+            advance(st, rend, 0xFFFFFFFFu, db, p.s, [&](uint32_t, uint32_t en) {
+              const float v = __fmul_rn(A, xi[(en >> 16) & 0xFFu]);
+              float* cell = sums + ((en & 0xFFFFu) - rbeg);
+              *cell = __fadd_rn(*cell, (int32_t)en < 0 ? -v : v);
+            });
+          }
+          __syncwarp();
+        }
+      }
+      // ---- phase 3: write the G ranges out (each contiguous in memory) and re-zero the tiles ---
+      const uint32_t range_quads = (rend - rbeg) >> 2;
+      for (uint32_t q0 = 0; q0 < G * tile_quads; q0 += 32 * kU) {
+        float4 t[kU], x[kU];
+        uint64_t at[kU];
+        uint32_t need = 0, full = 0;
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+          const uint32_t q = q0 + u * 32 + lane;
+          const uint32_t g = p.quad_shift < 32u ? q >> p.quad_shift : q / tile_quads;
+          const uint32_t j = q - g * tile_quads;
+          at[u] = (b0 + g) * p.d + rbeg + 4u * j;
+          t[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (q < G * tile_quads && j < range_quads && b0 + g < p.B && at[u] < p.n) {
+            t[u] = tile4[q];
+            const bool any = ((__float_as_uint(t[u].x) | __float_as_uint(t[u].y) | __float_as_uint(t[u].z) | __float_as_uint(t[u].w)) != 0u);
+            if (any) tile4[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (any || !skip_zero) {
+              need |= 1u << u;
+              if (at[u] + 4 <= p.n) full |= 1u << u;
+            }
+          }
+        }
+        if (FUSED) {
+#pragma unroll
+          for (int u = 0; u < kU; ++u)
+            if ((full >> u) & 1u) x[u] = *reinterpret_cast<const float4*>(p.out + at[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+          if (!((need >> u) & 1u)) continue;
+          float* o = p.out + at[u];
+          if ((full >> u) & 1u) {
+            float4 r = t[u];
+            if (FUSED) {
+              r.x = __fsub_rn(x[u].x, __fmul_rn(p.c, r.x)); r.y = __fsub_rn(x[u].y, __fmul_rn(p.c, r.y));
+              r.z = __fsub_rn(x[u].z, __fmul_rn(p.c, r.z)); r.w = __fsub_rn(x[u].w, __fmul_rn(p.c, r.w));
+            }
+            *reinterpret_cast<float4*>(o) = r;
+          } else {                                            // the quad that straddles n
+            if (at[u] + 0 < p.n) o[0] = FUSED ? __fsub_rn(o[0], __fmul_rn(p.c, t[u].x)) : t[u].x;
+            if (at[u] + 1 < p.n) o[1] = FUSED ? __fsub_rn(o[1], __fmul_rn(p.c, t[u].y)) : t[u].y;
+            if (at[u] + 2 < p.n) o[2] = FUSED ? __fsub_rn(o[2], __fmul_rn(p.c, t[u].z)) : t[u].z;
+          }
+        }
+      }
+      __syncwarp();
+    }
+    // a string must end exactly where the table says
+    if (parsing && st.err == 0u && (st.used != st.total || st.pend != kNoEntry)) st.err = QSGD_DEV_OVERRUN;
+    if (st.err) atomicOr(p.status, st.err);
+    __syncwarp();
+  }
+}
+
+// Launches the sparse-regime kernel when the configuration allows one (K <= 32, Code_s); the
+// caller then tells the other decoders to stand down when the predicate holds.
+int launch_sparse(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s, float* out, bool fused,
+                  float c, uint32_t* status, cudaStream_t stream, bool* launched) {
+  *launched = false;
+  if (K > 32u) return 0;
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  SparseParams p;
+  p.peers = peers; p.K = K; p.n = n; p.d = d; p.s = s;
+  p.sh = sparse_shape(K, d);
+  p.B = (n + d - 1) / d;
+  p.out = out; p.c = c; p.status = status;
+  p.warp_words = p.sh.G * p.sh.R + 64u + 32u * p.sh.C;
+  p.quad_shift = 32;
+  const uint32_t tile_quads = p.sh.R >> 2;
+  if ((tile_quads & (tile_quads - 1)) == 0)
+    for (p.quad_shift = 0; (1u << p.quad_shift) < tile_quads; ++p.quad_shift) {}
+  const size_t per_warp = (size_t)p.warp_words * 4;              // at most 16.3 KB
+  const int warps = 8 * per_warp <= (100u << 10) ? 8 : 4;
+  auto kern = fused ? decode_elias_sparse_kernel<true> : decode_elias_sparse_kernel<false>;
+  const size_t smem = (size_t)warps * per_warp;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return (int)e;
+  int occ = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, warps * 32, smem);
+  if (e != cudaSuccess) return (int)e;
+  if (occ < 1) occ = 1;
+  const uint64_t groups = (p.B + p.sh.G - 1) / p.sh.G;
+  const uint64_t want = (groups + warps - 1) / warps;
+  const uint64_t cap = (uint64_t)sms * occ;
+  const uint32_t grid = (uint32_t)(want < cap ? want : cap);
+  {
+    ScopedKernel sk(kKernDecodeEliasSparse, stream);
+    kern<<<grid, warps * 32, smem, stream>>>(p);
+  }
+  *launched = true;
+  return (int)cudaGetLastError();
+}
+
 template <int LB, bool DENSE, bool FUSED, bool SINGLE>
 __global__ void __launch_bounds__(128) decode_elias_fields_kernel(const __grid_constant__ FieldParams p) {
   extern __shared__ __align__(16) uint32_t fsm[];
   __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
   __shared__ uint16_t elias_lut[1u << kLutBits];
+  if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const float sf = (float)p.s;
   float lut0 = 0.f;
@@ -529,13 +858,16 @@ int launch_fields_lb(FieldParams& p, bool dense, bool fused, cudaStream_t stream
 int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s,
                         bool dense, float* acc_or_x, bool fused, float eta, uint32_t* status_dev,
                         cudaStream_t stream) {
+  bool sparse = false;
   {
     FieldParams f;
     f.peers = peers; f.K = K; f.n = n; f.d = d; f.s = s;
     f.B = (n + d - 1) / d;
     f.out = acc_or_x; f.c = eta / (float)K; f.status = status_dev;
     bool handled = false;
-    int st;
+    int st = dense ? 0 : launch_sparse(peers, K, n, d, s, acc_or_x, fused, f.c, status_dev, stream, &sparse);
+    if (st) return st;
+    f.defer_sparse = sparse ? 1u : 0u;
     switch (level_bits_for(s)) {
       case 1: st = launch_fields_lb<1>(f, dense, fused, stream, &handled); break;
       case 2: st = launch_fields_lb<2>(f, dense, fused, stream, &handled); break;
@@ -548,6 +880,7 @@ int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d
   p.peers = peers; p.K = K; p.Kc = K; p.n = n; p.d = d; p.s = s;
   p.B = (n + d - 1) / d;
   p.out = acc_or_x; p.c = eta / (float)K; p.status = status_dev; p.warp_bytes = 0;
+  p.defer_sparse = sparse ? 1u : 0u;
   if (s <= 127) return dense ? launch_slow<uint8_t, true>(p, fused, stream) : launch_slow<uint8_t, false>(p, fused, stream);
   return dense ? launch_slow<uint16_t, true>(p, fused, stream) : launch_slow<uint16_t, false>(p, fused, stream);
 }

@@ -117,9 +117,8 @@ int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d
 // timing is switched on (qsgd_profile_enable), records a CUDA event before and after it on the
 // launching stream.
 enum KernelId {
-  kKernQuantize = 0, kKernQuantizeTail, kKernFixedInfo, kKernDecodeFixed, kKernSgdStep, kKernEliasLength,
-  kKernScanBlockSums, kKernScanSums, kKernScanDownsweep, kKernZeroPayload, kKernEliasScatter,
-  kKernDecodeElias, kKernCount
+  kKernQuantize = 0, kKernQuantizeTail, kKernDecodeFixed, kKernSgdStep, kKernEliasLength,
+  kKernEliasScatter, kKernDecodeElias, kKernDecodeEliasSparse, kKernCount
 };
 
 struct ScopedKernel {

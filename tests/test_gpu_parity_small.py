@@ -111,3 +111,53 @@ def test_elias_bucket_shapes(d, s):
             msgs.append(m)
             infos.append(info)
         decode_parity(msgs, infos, n, d, s, code_kind)
+
+
+def sparse_regime_bits(K, d):
+    """Bits per string below which the decoder takes its entry-list path (mirrors the kernel's
+    work split: G = 32 / Kpad buckets per warp, ranges of R positions, lists of C entries)."""
+    kpad = 1
+    while kpad < K and kpad < 32:
+        kpad *= 2
+    R = min(d, 2048 // (32 // kpad))
+    C = max(16, R // 32)
+    return 32 + 8 * C * ((d + R - 1) // R)
+
+
+# Short strings (Section 3.1, sparse regime) take the entry-list decoder; these cases sit on
+# that side of its switch, which is decided on the device from the payload lengths.
+@pytest.mark.parametrize("n,d,s,K", [(5 * 4096 + 123, 4096, 1, 8), (9 * 1024 + 77, 1024, 1, 5), (11 * 3008 + 5, 3008, 1, 3),
+                                     (4 * 2048, 2048, 1, 32), (3 * 4096 + 1, 4096, 1, 1),
+                                     (70 * 64 + 9, 64, 1, 16)])
+@pytest.mark.parametrize("eta", [0.1, -0.25])
+def test_elias_sparse_regime(n, d, s, K, eta):
+    msgs, infos = [], []
+    for w in range(K):
+        g = make(n, "sparse", seed=300 + w)
+        m, info = encode_parity(g, d, s, O.NORM_L2, O.CODE_ELIAS, seed=5, step=3, worker=w)
+        msgs.append(m)
+        infos.append(info)
+    B = O.n_buckets(n, d)
+    assert sum(i[0] for i in infos) < K * B * sparse_regime_bits(K, d), "case is not in the sparse regime"
+    x0 = I.gaussian(n, 1.0, seed=9)
+    x0[::7] = -0.0                                  # x - c * (+0) must keep the sign of zero
+    decode_parity(msgs, infos, n, d, s, O.CODE_ELIAS, eta=eta, x0=x0)
+
+
+@pytest.mark.parametrize("d,s,Bn", [(512, 15, 80), (4096, 255, 200), (128, 3, 48)])
+def test_elias_sparse_regime_long_lists(d, s, Bn):
+    """Mostly empty buckets keep the payload short while a few buckets hold far more nonzeros
+    than one list has room for."""
+    K = 6
+    n = Bn * d - 17
+    msgs, infos = [], []
+    for w in range(K):
+        g = np.zeros(n, dtype=np.float32)
+        for b in (3 + w % 2, 20, Bn - 1):
+            lo, hi = b * d, min((b + 1) * d, n)
+            g[lo:hi] = make(hi - lo, "gauss", seed=400 + 7 * w + b)
+        m, info = encode_parity(g, d, s, O.NORM_MAX, O.CODE_ELIAS, seed=6, step=0, worker=w)
+        msgs.append(m)
+        infos.append(info)
+    assert sum(i[0] for i in infos) < K * Bn * sparse_regime_bits(K, d), "case is not in the sparse regime"
+    decode_parity(msgs, infos, n, d, s, O.CODE_ELIAS, eta=0.5, x0=I.gaussian(n, 1.0, seed=1))
