@@ -536,7 +536,7 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
   for (uint32_t q = lane; q < ((G * R) >> 2); q += 32) tile4[q] = make_float4(0.f, 0.f, 0.f, 0.f);
   __syncthreads();
 
-  const uint32_t pg = lane / Kpad, pk = lane % Kpad;           // this lane's bucket in the group and peer
+  const uint32_t pg = lane / Kpad, pk = lane % Kpad;           // this lane's bucket in the group (idle if >= G) and peer
   float* sums = tile + pg * R;                                 // its bucket's tile
   uint32_t* list = lists + lane * C;
   const bool skip_zero = FUSED && p.c >= 0.f;                  // x - c * (+0) == x
@@ -554,7 +554,7 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
     st.pend = kNoEntry;
     uint32_t db = 0;                                           // coordinates of this lane's bucket
     float A = 0.f;
-    if (b0 + pg < p.B) db = (uint32_t)min((uint64_t)p.d, p.n - (b0 + pg) * p.d);
+    if (pg < G && b0 + pg < p.B) db = (uint32_t)min((uint64_t)p.d, p.n - (b0 + pg) * p.d);
     const bool parsing = db != 0u && pk < p.K;
     if (parsing) {
       const uint64_t b = b0 + pg;
@@ -572,6 +572,8 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
       }
     }
     scales[lane] = A;
+    const bool bad_scale = !(fabsf(A) <= 3.402823466e+38f);
+    float* xrow = p.out + (b0 + pg) * (uint64_t)p.d;            // this lane's bucket in x (valid when db != 0)
 
     for (uint32_t rbeg = 0; rbeg < p.d; rbeg += R) {
       const uint32_t rend = min(rbeg + R, p.d);
@@ -582,16 +584,16 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
         if (st.pend != kNoEntry && (st.pend & 0xFFFFu) < rend) mycnt |= kMore;
       }
       counts[lane] = mycnt;
+      // Rare cases that need the careful paths below: a list that overflowed, a non-finite scale.
+      const bool odd_range = __any_sync(0xffffffffu, (mycnt & kMore) != 0u || bad_scale);
       __syncwarp();
       // ---- phase 2: each bucket's lanes add its lists in ascending k -------------------------
       for (uint32_t k = 0; k < p.K; ++k) {
         const uint32_t owner = pg * Kpad + k;
         const float Ak = scales[owner];
         const uint32_t cnt = counts[owner];
-        const bool bad = !(fabsf(Ak) <= 3.402823466e+38f);    // inf or NaN scale: A * 0 is NaN everywhere
-        const bool odd = __any_sync(0xffffffffu, bad || (cnt & kMore) != 0u);   // warp-uniform
-        if (odd) {
-          if (bad) {
+        if (odd_range) {
+          if (!(fabsf(Ak) <= 3.402823466e+38f)) {            // inf or NaN scale: A * 0 is NaN everywhere
             const float z = __fmul_rn(Ak, 0.f);
             for (uint32_t i = rbeg + pk; i < min(rend, db); i += Kpad) sums[i - rbeg] = __fadd_rn(sums[i - rbeg], z);
           }
@@ -605,7 +607,7 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
           *cell = __fadd_rn(*cell, (int32_t)en < 0 ? -v : v);
         }
         __syncwarp();
-        if (odd) {                                           // rest of a long list, by its own lane
+        if (odd_range) {                                     // rest of a long list, by its own lane
           if (lane == owner && (cnt & kMore)) {
             advance(st, rend, 0xFFFFFFFFu, db, p.s, [&](uint32_t, uint32_t en) {
               const float v = __fmul_rn(A, xi[(en >> 16) & 0xFFu]);
@@ -616,7 +618,35 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
           __syncwarp();
         }
       }
-      // ---- phase 3: write the G ranges out (each contiguous in memory) and re-zero the tiles ---
+      // ---- phase 3: write the sums out and re-zero the tiles ------------------------------------
+      if (skip_zero && !odd_range) {
+        // Fused step, c >= 0: only listed positions can hold a nonzero sum. Each lane walks its own
+        // list and claims a cell by exchanging it with +0: whoever receives the nonzero sum applies
+        // it to x, so a position listed by several peers is updated once. Eight in flight per lane.
+        const uint32_t cnt = mycnt;
+        for (uint32_t e0 = 0; e0 < cnt; e0 += kU) {
+          float v[kU], x[kU];
+          uint32_t pos[kU];
+#pragma unroll
+          for (int u = 0; u < kU; ++u) {
+            v[u] = 0.f;
+            pos[u] = 0;
+            if (e0 + u < cnt) {
+              pos[u] = list[e0 + u] & 0xFFFFu;
+              v[u] = atomicExch(sums + (pos[u] - rbeg), 0.f);
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < kU; ++u)
+            if (__float_as_uint(v[u]) != 0u) x[u] = xrow[pos[u]];
+#pragma unroll
+          for (int u = 0; u < kU; ++u)
+            if (__float_as_uint(v[u]) != 0u) xrow[pos[u]] = __fsub_rn(x[u], __fmul_rn(p.c, v[u]));
+        }
+        __syncwarp();
+        continue;
+      }
+      // Otherwise scan the G ranges (each contiguous in memory).
       const uint32_t range_quads = (rend - rbeg) >> 2;
       for (uint32_t q0 = 0; q0 < G * tile_quads; q0 += 32 * kU) {
         float4 t[kU], x[kU];
@@ -685,6 +715,9 @@ int launch_sparse(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint
   p.sh = sparse_shape(K, d);
   p.B = (n + d - 1) / d;
   p.out = out; p.c = c; p.status = status;
+  // A small problem is spread over more warps (fewer buckets each, some lanes idle): the parse is
+  // a chain of dependent instructions, so resident warps are what hides its latency.
+  while (p.sh.G > 1u && p.B / p.sh.G < (uint64_t)sms * 12u) p.sh.G >>= 1;
   p.warp_words = p.sh.G * p.sh.R + 64u + 32u * p.sh.C;
   p.quad_shift = 32;
   const uint32_t tile_quads = p.sh.R >> 2;

@@ -128,7 +128,10 @@ def sparse_regime_bits(K, d):
 # that side of its switch, which is decided on the device from the payload lengths.
 @pytest.mark.parametrize("n,d,s,K", [(5 * 4096 + 123, 4096, 1, 8), (9 * 1024 + 77, 1024, 1, 5), (11 * 3008 + 5, 3008, 1, 3),
                                      (4 * 2048, 2048, 1, 32), (3 * 4096 + 1, 4096, 1, 1),
-                                     (70 * 64 + 9, 64, 1, 16)])
+                                     (70 * 64 + 9, 64, 1, 16),
+                                     # enough buckets that a warp takes its full share of them
+                                     (7200 * 64 + 5, 64, 1, 8), (14300 * 32 + 3, 32, 1, 3),
+                                     (57000 * 32 + 31, 32, 1, 1)])
 @pytest.mark.parametrize("eta", [0.1, -0.25])
 def test_elias_sparse_regime(n, d, s, K, eta):
     msgs, infos = [], []
