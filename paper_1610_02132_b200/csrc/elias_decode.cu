@@ -36,38 +36,39 @@ struct EliasDecodeParams {
   uint32_t defer_sparse;  // a sparse-regime kernel was launched beside this one
 };
 
-// Work split of the sparse-regime decoder (defined further down): a warp owns G = 32 / Kpad buckets
-// and walks each in ranges of R positions; a (bucket, peer) list holds the C entries of one range.
+// Work split of the sparse-regime decoder (defined further down): a warp owns G <= 32 / Kpad
+// buckets and walks each in ranges of R positions; a (bucket, peer) list holds the C entries of one
+// range. Fewer buckets per warp (some lanes idle) spread a small problem over more warps: the parse
+// is a chain of dependent instructions, so resident warps are what hides its latency.
 struct SparseShape {
   uint32_t Kpad;      // lanes per bucket: K rounded up to a power of two
   uint32_t G;         // buckets per warp
   uint32_t R;         // positions per range; G * R <= 2048 sums per warp
-  uint32_t C;         // entries per list and range
-  uint32_t ranges;    // ceil(d / R)
+  uint32_t C;         // entries per list and range: one per 32 positions, at least 16
 };
 
-__host__ __device__ inline SparseShape sparse_shape(uint32_t K, uint32_t d) {
+inline SparseShape sparse_shape(uint32_t K, uint32_t d, uint64_t B, uint32_t sms) {
   SparseShape sh;
   sh.Kpad = 1;
   while (sh.Kpad < K && sh.Kpad < 32u) sh.Kpad <<= 1;
   sh.G = 32u / sh.Kpad;
+  while (sh.G > 1u && B / sh.G < (uint64_t)sms * 12u) sh.G >>= 1;
   sh.R = 2048u / sh.G;                     // a power of two, >= 64
+  if (sh.R > 1024u) sh.R = 1024u;
   if (d <= sh.R) sh.R = d;                 // whole bucket in one range
   sh.C = sh.R / 32u > 16u ? sh.R / 32u : 16u;
-  sh.ranges = (d + sh.R - 1) / sh.R;
   return sh;
 }
 
-// Strings short enough for the entry-list decoder? True when the average string carries fewer than
-// 8 bits per list slot beyond its scale: an entry of a sparse bucket costs 11 to 14 bits, so lists
-// then fill to about 60 % on average and rarely overflow. Same answer in every thread of every
-// kernel that asks.
+// Strings short enough for the entry-list decoder? True when the K payloads average less than a
+// quarter of a bit per coordinate beyond the scales: an entry of a sparse bucket costs 11 to 14
+// bits, so a list with room for one entry per 32 positions then fills to about 60 % on average and
+// rarely overflows. Same answer in every thread of every kernel that asks.
 __device__ __forceinline__ bool sparse_regime(const PeerSet& peers, uint32_t K, uint64_t B, uint32_t d) {
   if (K > 32u) return false;
-  const SparseShape sh = sparse_shape(K, d);
   uint64_t bits = 0;
   for (uint32_t k = 0; k < K; ++k) bits += __ldg(peers.table[k] + B);
-  return bits < (uint64_t)K * B * (32ull + 8ull * sh.C * sh.ranges);
+  return bits < (uint64_t)K * B * (32ull + d / 4u);
 }
 
 template <typename CodeT> struct CodeTraits;
@@ -505,15 +506,23 @@ __device__ __forceinline__ uint32_t advance(LaneParse& st, uint32_t rend, uint32
     st.used += len;
     st.src.refill();
     const uint32_t neg = st.src.hi >> 31;
-    ok &= elias_from_window(st.src.hi << 1, level, len);
+    if ((st.src.hi & 0x40000000u) == 0u) {            // level 1, by far the most frequent in this regime
+      level = 1u;
+      len = 1u;
+    } else {
+      ok &= elias_from_window(st.src.hi << 1, level, len);
+    }
     st.src.drop(len + 1u);
     st.used += len + 1u;
     st.at += gap;
-    st.err |= ok ? 0u : QSGD_DEV_OVERRUN;
-    st.err |= st.at >= db ? QSGD_DEV_POSITION : 0u;
-    st.err |= level > s ? QSGD_DEV_LEVEL : 0u;
-    st.err |= st.used > st.total ? QSGD_DEV_OVERRUN : 0u;
-    if (st.err == 0u) st.pend = st.at | (level << 16) | (neg << 31);
+    if (!ok || st.at >= db || level > s || st.used > st.total) {
+      st.err |= ok ? 0u : QSGD_DEV_OVERRUN;
+      st.err |= st.at >= db ? QSGD_DEV_POSITION : 0u;
+      st.err |= level > s ? QSGD_DEV_LEVEL : 0u;
+      st.err |= st.used > st.total ? QSGD_DEV_OVERRUN : 0u;
+    } else {
+      st.pend = st.at | (level << 16) | (neg << 31);
+    }
   }
   return n;
 }
@@ -712,13 +721,10 @@ int launch_sparse(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   SparseParams p;
   p.peers = peers; p.K = K; p.n = n; p.d = d; p.s = s;
-  p.sh = sparse_shape(K, d);
   p.B = (n + d - 1) / d;
+  p.sh = sparse_shape(K, d, p.B, (uint32_t)sms);
   p.out = out; p.c = c; p.status = status;
-  // A small problem is spread over more warps (fewer buckets each, some lanes idle): the parse is
-  // a chain of dependent instructions, so resident warps are what hides its latency.
-  while (p.sh.G > 1u && p.B / p.sh.G < (uint64_t)sms * 12u) p.sh.G >>= 1;
-  p.warp_words = p.sh.G * p.sh.R + 64u + 32u * p.sh.C;
+  p.warp_words = p.sh.G * p.sh.R + 64u + p.sh.G * p.sh.Kpad * p.sh.C;
   p.quad_shift = 32;
   const uint32_t tile_quads = p.sh.R >> 2;
   if ((tile_quads & (tile_quads - 1)) == 0)

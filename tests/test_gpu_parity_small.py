@@ -114,29 +114,23 @@ def test_elias_bucket_shapes(d, s):
 
 
 def sparse_regime_bits(K, d):
-    """Bits per string below which the decoder takes its entry-list path (mirrors the kernel's
-    work split: G = 32 / Kpad buckets per warp, ranges of R positions, lists of C entries)."""
-    kpad = 1
-    while kpad < K and kpad < 32:
-        kpad *= 2
-    R = min(d, 2048 // (32 // kpad))
-    C = max(16, R // 32)
-    return 32 + 8 * C * ((d + R - 1) // R)
+    """Average bits per string below which the decoder takes its entry-list path."""
+    return 32 + d // 4
 
 
 # Short strings (Section 3.1, sparse regime) take the entry-list decoder; these cases sit on
 # that side of its switch, which is decided on the device from the payload lengths.
-@pytest.mark.parametrize("n,d,s,K", [(5 * 4096 + 123, 4096, 1, 8), (9 * 1024 + 77, 1024, 1, 5), (11 * 3008 + 5, 3008, 1, 3),
-                                     (4 * 2048, 2048, 1, 32), (3 * 4096 + 1, 4096, 1, 1),
-                                     (70 * 64 + 9, 64, 1, 16),
-                                     # enough buckets that a warp takes its full share of them
-                                     (7200 * 64 + 5, 64, 1, 8), (14300 * 32 + 3, 32, 1, 3),
-                                     (57000 * 32 + 31, 32, 1, 1)])
+@pytest.mark.parametrize("n,d,s,K,zeros", [(5 * 4096 + 123, 4096, 1, 8, 0.3), (9 * 1024 + 77, 1024, 1, 5, 0.3),
+                                           (11 * 3008 + 5, 3008, 1, 3, 0.3), (4 * 2048, 2048, 1, 32, 0.3),
+                                           (3 * 4096 + 1, 4096, 1, 1, 0.3), (70 * 64 + 9, 64, 3, 16, 0.98),
+                                           # enough buckets that a warp takes its full share of them
+                                           (7200 * 64 + 5, 64, 1, 8, 0.98), (14300 * 128 + 3, 128, 1, 3, 0.95),
+                                           (57000 * 32 + 31, 32, 1, 1, 0.98)])
 @pytest.mark.parametrize("eta", [0.1, -0.25])
-def test_elias_sparse_regime(n, d, s, K, eta):
+def test_elias_sparse_regime(n, d, s, K, zeros, eta):
     msgs, infos = [], []
     for w in range(K):
-        g = make(n, "sparse", seed=300 + w)
+        g = I.sparse_laplace(n, 1e-3, zeros, seed=300 + w)
         m, info = encode_parity(g, d, s, O.NORM_L2, O.CODE_ELIAS, seed=5, step=3, worker=w)
         msgs.append(m)
         infos.append(info)
