@@ -450,6 +450,7 @@ struct SparseParams {
   uint32_t* status;
   uint32_t warp_words;   // shared-memory words per warp: G * R sums, 64 of scales and counts, 32 lists
   uint32_t quad_shift;   // log2(R / 4) when R is a power of two, else 32
+  uint32_t check_regime; // 0: the host already knows that this kernel is the one to run
 };
 
 // The recursive Elias code (Definition A.1) of one integer below 2^16, decoded without branches
@@ -531,7 +532,7 @@ template <bool FUSED>
 __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __grid_constant__ SparseParams p) {
   extern __shared__ __align__(16) uint32_t ssm[];
   __shared__ float xi[256];
-  if (!sparse_regime(p.peers, p.K, p.B, p.d)) return;
+  if (p.check_regime && !sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const uint32_t G = p.sh.G, Kpad = p.sh.Kpad, R = p.sh.R, C = p.sh.C;
   for (uint32_t i = tid; i < 256; i += blockDim.x) xi[i] = __fdiv_rn((float)i, (float)p.s);
@@ -713,7 +714,7 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
 // Launches the sparse-regime kernel when the configuration allows one (K <= 32, Code_s); the
 // caller then tells the other decoders to stand down when the predicate holds.
 int launch_sparse(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s, float* out, bool fused,
-                  float c, uint32_t* status, cudaStream_t stream, bool* launched) {
+                  float c, uint32_t* status, bool check_regime, cudaStream_t stream, bool* launched) {
   *launched = false;
   if (K > 32u) return 0;
   int dev = 0, sms = 0;
@@ -723,7 +724,7 @@ int launch_sparse(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint
   p.peers = peers; p.K = K; p.n = n; p.d = d; p.s = s;
   p.B = (n + d - 1) / d;
   p.sh = sparse_shape(K, d, p.B, (uint32_t)sms);
-  p.out = out; p.c = c; p.status = status;
+  p.out = out; p.c = c; p.status = status; p.check_regime = check_regime ? 1u : 0u;
   p.warp_words = p.sh.G * p.sh.R + 64u + p.sh.G * p.sh.Kpad * p.sh.C;
   p.quad_shift = 32;
   const uint32_t tile_quads = p.sh.R >> 2;
@@ -897,15 +898,34 @@ int launch_fields_lb(FieldParams& p, bool dense, bool fused, cudaStream_t stream
 int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s,
                         bool dense, float* acc_or_x, bool fused, float eta, uint32_t* status_dev,
                         cudaStream_t stream) {
+  // Which decoder? In a message the offset table follows the padded payload, so table - payload is
+  // the payload size and the host can evaluate the regime predicate itself (to within the padding)
+  // and launch one kernel. With tables kept elsewhere the sizes are only known on the device: both
+  // kernels are launched and exactly one does the work. Either decoder is correct on any input;
+  // the choice is about speed only.
+  const uint64_t B = (n + d - 1) / d;
+  bool sizes_known = !dense && K <= 32u;
+  uint64_t payload_bits = 0;
+  for (uint32_t k = 0; k < K && sizes_known; ++k) {
+    const uint8_t* w = reinterpret_cast<const uint8_t*>(peers.payload[k]);
+    const uint8_t* t = reinterpret_cast<const uint8_t*>(peers.table[k]);
+    const uint64_t longest = align16((B * 32ull + n * 40ull + 7ull) / 8ull);   // no legal payload is longer
+    if (t <= w || (uint64_t)(t - w) > longest) sizes_known = false;
+    else payload_bits += 8ull * (uint64_t)(t - w);
+  }
+  const bool host_sparse = sizes_known && payload_bits < (uint64_t)K * B * (32ull + d / 4u);
   bool sparse = false;
   {
     FieldParams f;
     f.peers = peers; f.K = K; f.n = n; f.d = d; f.s = s;
-    f.B = (n + d - 1) / d;
+    f.B = B;
     f.out = acc_or_x; f.c = eta / (float)K; f.status = status_dev;
     bool handled = false;
-    int st = dense ? 0 : launch_sparse(peers, K, n, d, s, acc_or_x, fused, f.c, status_dev, stream, &sparse);
+    int st = 0;
+    if (!dense && (host_sparse || !sizes_known))
+      st = launch_sparse(peers, K, n, d, s, acc_or_x, fused, f.c, status_dev, !sizes_known, stream, &sparse);
     if (st) return st;
+    if (sparse && sizes_known) return 0;                    // the host chose the sparse-regime kernel
     f.defer_sparse = sparse ? 1u : 0u;
     switch (level_bits_for(s)) {
       case 1: st = launch_fields_lb<1>(f, dense, fused, stream, &handled); break;

@@ -74,11 +74,24 @@ def table_view(msg_dev, info, n, d):
     return msg_dev[info[1]: info[1] + 8 * (B + 1)].view(torch.int64)
 
 
-def decode_parity(msgs_dev, infos, n, d, s, code_kind, eta=0.1, x0=None):
-    """GPU decode+aggregate and SGD step (fused and unfused) == oracle, bit for bit."""
+def decode_parity(msgs_dev, infos, n, d, s, code_kind, eta=0.1, x0=None, tables_first=False):
+    """GPU decode+aggregate and SGD step (fused and unfused) == oracle, bit for bit. With
+    tables_first each offset table is handed over in front of its payload instead of behind it, so
+    the library cannot read the payload size off the two pointers."""
     K = len(msgs_dev)
     dev = msgs_dev[0].device
     tables = None if code_kind == O.CODE_FIXED else [table_view(m, i, n, d) for m, i in zip(msgs_dev, infos)]
+    if tables_first and tables is not None:
+        moved_msgs, moved_tables = [], []
+        for m, t, i in zip(msgs_dev, tables, infos):
+            tb = t.numel() * 8
+            front = (tb + 15) // 16 * 16
+            buf = torch.zeros(front + i[1] + 16, dtype=torch.uint8, device=dev)
+            buf[:tb] = t.view(torch.uint8)
+            buf[front: front + i[1]] = m[: i[1]]
+            moved_tables.append(buf[:tb].view(torch.int64))
+            moved_msgs.append(buf[front:])
+        msgs_dev, tables = moved_msgs, moved_tables
     status = Q.new_status(dev)
     acc = torch.full((n + 64,), 7.0, dtype=torch.float32, device=dev)
     Q.qsgd_decode_accumulate(msgs_dev, tables, n, d, s, code_kind, acc[:n], status)

@@ -98,6 +98,7 @@ def test_elias_peer_counts(K, code_kind):
         msgs.append(m)
         infos.append(info)
     decode_parity(msgs, infos, n, d, s, code_kind, eta=0.05, x0=I.gaussian(n, 1.0, seed=9))
+    decode_parity(msgs, infos, n, d, s, code_kind, eta=0.05, x0=I.gaussian(n, 1.0, seed=9), tables_first=True)
 
 
 @pytest.mark.parametrize("d,s", [(4096, 255), (4096, 1), (2048, 15), (1024, 3), (64, 15), (32, 1)])
@@ -139,6 +140,8 @@ def test_elias_sparse_regime(n, d, s, K, zeros, eta):
     x0 = I.gaussian(n, 1.0, seed=9)
     x0[::7] = -0.0                                  # x - c * (+0) must keep the sign of zero
     decode_parity(msgs, infos, n, d, s, O.CODE_ELIAS, eta=eta, x0=x0)
+    if eta > 0:
+        decode_parity(msgs, infos, n, d, s, O.CODE_ELIAS, eta=eta, x0=x0, tables_first=True)
 
 
 @pytest.mark.parametrize("d,s,Bn", [(512, 15, 80), (4096, 255, 200), (128, 3, 48)])
