@@ -273,3 +273,88 @@ def sgd_step(x, acc, eta, K):
     acc = _f32(acc)
     lib().oq_sgd_step(_p(x, C.c_float), _p(acc, C.c_float), eta, K, x.size)
     return x
+
+
+# --------------------------------------------------------------------------------------------------
+# Per-tensor policy (Section 5, "Protocol": tensors below a size threshold are sent in full
+# precision, and buckets are cut so that they fit the tensors). Written on top of the functions
+# above, in numpy, tensor by tensor:
+#   * the flat gradient is a concatenation of T tensors of the given sizes;
+#   * a tensor with fewer than `min_quantized` elements is "raw": its fp32 values travel as they are;
+#   * every other tensor is cut into buckets of d starting at its own first element, the last one
+#     shorter. Its values are laid out in a "compact" vector in which each tensor is padded with
+#     zeros up to a multiple of d, so that the compact vector has uniform buckets and the ordinary
+#     Encode applies to it unchanged (zeros do not change a norm and quantize to level 0). The
+#     uniform of a coordinate is keyed by its compact index.
+# Policy message = raw values (fp32, padded to 16 bytes) followed by the ordinary message of the
+# compact vector. Decode: ordinary decode of the compact part; the raw values of the K messages are
+# summed in ascending k from +0; both are put back at the tensors' positions.
+# --------------------------------------------------------------------------------------------------
+def policy_plan(sizes, d, min_quantized=10000):
+    """Layout of the compact vector and of the raw region for tensors of the given sizes."""
+    sizes = [int(m) for m in sizes]
+    plan = {"d": d, "n": sum(sizes), "large": [], "small": [], "n_compact": 0, "n_raw": 0}
+    off = 0
+    for m in sizes:
+        if m >= min_quantized:
+            padded = (m + d - 1) // d * d
+            plan["large"].append((off, m, plan["n_compact"]))     # flat offset, size, compact offset
+            plan["n_compact"] += padded
+        elif m > 0:
+            plan["small"].append((off, m, plan["n_raw"]))         # flat offset, size, raw offset
+            plan["n_raw"] += m
+        off += m
+    plan["raw_prefix"] = (4 * plan["n_raw"] + 15) // 16 * 16
+    return plan
+
+
+def policy_gather(g, plan):
+    g = _f32(g)
+    assert g.size == plan["n"]
+    compact = np.zeros(plan["n_compact"], dtype=np.float32)
+    raw = np.zeros(plan["n_raw"], dtype=np.float32)
+    for off, m, c0 in plan["large"]:
+        compact[c0:c0 + m] = g[off:off + m]
+    for off, m, r0 in plan["small"]:
+        raw[r0:r0 + m] = g[off:off + m]
+    return compact, raw
+
+
+def policy_scatter(compact, raw, plan):
+    out = np.zeros(plan["n"], dtype=np.float32)
+    for off, m, c0 in plan["large"]:
+        out[off:off + m] = compact[c0:c0 + m]
+    for off, m, r0 in plan["small"]:
+        out[off:off + m] = raw[r0:r0 + m]
+    return out
+
+
+def policy_encode(g, plan, s, norm_kind, code_kind, seed, step, worker, A_ext=None):
+    """Returns (policy message bytes, info[4]): info[0] = information bits (32 per raw value plus
+    the ordinary message's), info[1] = byte offset of the offset table (0 if none), info[2] =
+    message bytes, info[3] = bytes of the raw region in front."""
+    compact, raw = policy_gather(g, plan)
+    prefix = plan["raw_prefix"]
+    head = np.zeros(prefix, dtype=np.uint8)
+    head[:4 * raw.size] = raw.view(np.uint8)
+    if plan["n_compact"] == 0:
+        return head, [32 * raw.size, 0, prefix, prefix]
+    msg, info = encode(compact, plan["d"], s, norm_kind, code_kind, seed, step, worker, A_ext=A_ext)
+    return (np.concatenate([head, msg]),
+            [info[0] + 32 * raw.size, info[1] + prefix if info[1] else 0, info[2] + prefix, prefix])
+
+
+def policy_decode_accumulate(msgs, infos, plan, s, code_kind):
+    """Sum of the K decoded policy messages, ascending k from +0, at the tensors' positions."""
+    d, prefix, nc, nr = plan["d"], plan["raw_prefix"], plan["n_compact"], plan["n_raw"]
+    st, acc_c = 0, np.zeros(0, dtype=np.float32)
+    if nc:
+        parts = [np.ascontiguousarray(m[prefix:]) for m in msgs]
+        tabs = None
+        if code_kind != CODE_FIXED:
+            tabs = [message_table(p, [i[0], i[1] - prefix, i[2] - prefix, 0], nc, d) for p, i in zip(parts, infos)]
+        st, acc_c = decode_accumulate(parts, tabs, nc, d, s, code_kind)
+    acc_r = np.zeros(nr, dtype=np.float32)
+    for m in msgs:
+        acc_r = acc_r + np.ascontiguousarray(m[:4 * nr]).view(np.float32)     # fp32 adds, ascending k
+    return st, policy_scatter(acc_c, acc_r, plan)
