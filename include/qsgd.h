@@ -180,6 +180,76 @@ int qsgd_encode_elias_static(const float* g, uint64_t n, uint32_t bucket, uint32
                              qsgd_stream_t stream);
 
 /*
+ * Per-tensor policy (Section 5, "Protocol": tensors with fewer than 10K elements are not
+ * quantized, and buckets are cut so that they fit the tensors).
+ *
+ * The flat gradient g[n] is the concatenation of T tensors. A tensor with fewer than
+ * `min_quantized` elements is "raw": its fp32 values travel unchanged. Every other tensor is cut
+ * into buckets of `bucket` elements that start at the tensor's first element; the last bucket of a
+ * tensor may be shorter. The quantized tensors form a "compact" vector in which each tensor is
+ * padded with zeros to whole buckets (zeros change no norm and quantize to level 0); Encode and
+ * Decode of the compact vector are exactly qsgd_encode / qsgd_decode_* on n_buckets * bucket
+ * coordinates, the uniform of a coordinate being keyed by its compact index. The padding exists
+ * in no buffer: the kernels read and write each bucket at its own place in g / x.
+ *
+ * Policy message = raw values in tensor order (fp32, zero-padded to 16 bytes) followed by the
+ * ordinary message of the compact vector. out_bits: [0] 32 * n_raw plus the ordinary [0],
+ * [1] byte offset of the offset table inside `out` (0 for QSGD_CODE_FIXED), [2] message bytes,
+ * [3] bytes of the raw region in front.
+ *
+ * qsgd_policy_plan_sizes / qsgd_policy_plan run on the host and touch no GPU. The first returns
+ * the array lengths, the second fills caller-owned HOST arrays:
+ *   bucket_src[n_buckets], bucket_len[n_buckets]   place in g and length of every bucket,
+ *   raw_src[n_raw_segments], raw_start[n_raw_segments + 1]   place in g of every raw tensor and
+ *                                                   its offset in the raw region (last = n_raw),
+ * and returns in *quads whether every bucket place and length is a multiple of 4 elements (then
+ * the kernels may use 16-byte accesses and bulk copies; otherwise they fall back to narrower ones).
+ * The caller copies the arrays to the device and hands them over in a qsgd_policy. Returns
+ * QSGD_OK, QSGD_ERR_NULL, QSGD_ERR_BUCKET or QSGD_ERR_SIZE (no elements at all).
+ */
+typedef struct {
+  const uint64_t* bucket_src;  /* device */
+  const uint32_t* bucket_len;  /* device */
+  uint64_t n_buckets;
+  const uint64_t* raw_src;     /* device */
+  const uint64_t* raw_start;   /* device */
+  uint64_t n_raw_segments;
+  uint64_t n_raw;
+  uint64_t n;                  /* elements of the flat gradient */
+  uint32_t quads;              /* as returned by qsgd_policy_plan */
+} qsgd_policy;
+
+int qsgd_policy_plan_sizes(const uint64_t* tensor_sizes, uint32_t T, uint32_t bucket, uint64_t min_quantized,
+                           uint64_t* n_buckets, uint64_t* n_raw_segments, uint64_t* n_raw);
+int qsgd_policy_plan(const uint64_t* tensor_sizes, uint32_t T, uint32_t bucket, uint64_t min_quantized,
+                     uint64_t* bucket_src, uint32_t* bucket_len, uint64_t* raw_src, uint64_t* raw_start,
+                     uint32_t* quads);
+
+/* Worst-case bytes of one policy message, and scratch bytes of qsgd_policy_encode. */
+size_t qsgd_policy_message_capacity(const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind);
+size_t qsgd_policy_workspace_bytes(const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind);
+
+/*
+ * Encode / Decode under the policy. Arguments as for qsgd_encode, qsgd_decode_accumulate and
+ * qsgd_decode_sgd_step, with the plan in place of n; `plan` is a host pointer to a struct of device
+ * pointers. msgs[k] points to the start of policy message k (its raw region), tables[k] to its
+ * offset table (msgs[k] + out_bits[1]). acc (n floats) is overwritten at every coordinate; x is
+ * updated at every coordinate; fused and unfused results are equal bit for bit. Errors as for the
+ * ordinary calls. Launches: the ordinary encode or decode kernels plus one small kernel for the
+ * raw tensors.
+ */
+int qsgd_policy_encode(const float* g, const qsgd_policy* plan, uint32_t bucket, uint32_t s, int norm_kind,
+                       int code_kind, uint64_t seed, uint32_t step, uint32_t worker, void* out,
+                       size_t out_capacity, uint64_t* out_bits, void* workspace, uint32_t* status_dev,
+                       qsgd_stream_t stream);
+int qsgd_policy_decode_accumulate(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
+                                  const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind,
+                                  float* acc, uint32_t* status_dev, qsgd_stream_t stream);
+int qsgd_policy_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
+                                const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind,
+                                float* x, float eta, uint32_t* status_dev, qsgd_stream_t stream);
+
+/*
  * Per-kernel timing (measurement aid; the paper has no counterpart). While enabled, every
  * kernel launch of the library is bracketed by two CUDA events on its stream.
  * qsgd_profile_collect waits for the recorded events, adds each kernel's elapsed time and

@@ -4,4 +4,6 @@ from .binding import (CODE_ELIAS, CODE_ELIAS_DENSE, CODE_FIXED, NORM_L2, NORM_MA
                       QsgdError, encode_alloc, new_status, qsgd_decode_accumulate,
                       qsgd_decode_sgd_step, qsgd_encode, qsgd_encode_elias_static, qsgd_fixed_layout, qsgd_launch_count,
                       qsgd_message_capacity, qsgd_profile_collect, qsgd_profile_enable,
-                      qsgd_sgd_step, qsgd_static_scratch_bytes, qsgd_workspace_bytes)
+                      qsgd_sgd_step, qsgd_static_scratch_bytes, qsgd_workspace_bytes,
+                      Policy, qsgd_policy_decode_accumulate, qsgd_policy_decode_sgd_step,
+                      qsgd_policy_encode, qsgd_policy_message_capacity, qsgd_policy_workspace_bytes)

@@ -19,13 +19,23 @@ EXPORTS = ["qsgd_message_capacity", "qsgd_workspace_bytes", "qsgd_fixed_layout",
            "qsgd_decode_accumulate", "qsgd_sgd_step", "qsgd_decode_sgd_step",
            "qsgd_status_string", "qsgd_launch_count", "qsgd_profile_enable",
            "qsgd_profile_kernel_count", "qsgd_profile_kernel_name", "qsgd_profile_collect",
-           "qsgd_static_scratch_bytes", "qsgd_encode_elias_static"]
+           "qsgd_static_scratch_bytes", "qsgd_encode_elias_static",
+           "qsgd_policy_plan_sizes", "qsgd_policy_plan", "qsgd_policy_message_capacity",
+           "qsgd_policy_workspace_bytes", "qsgd_policy_encode", "qsgd_policy_decode_accumulate",
+           "qsgd_policy_decode_sgd_step"]
 
 _lib = None
 
 
 class QsgdError(RuntimeError):
     pass
+
+
+class PolicyStruct(C.Structure):
+    """qsgd_policy of include/qsgd.h."""
+    _fields_ = [("bucket_src", C.c_void_p), ("bucket_len", C.c_void_p), ("n_buckets", C.c_uint64),
+                ("raw_src", C.c_void_p), ("raw_start", C.c_void_p), ("n_raw_segments", C.c_uint64),
+                ("n_raw", C.c_uint64), ("n", C.c_uint64), ("quads", C.c_uint32)]
 
 
 def lib():
@@ -62,6 +72,24 @@ def lib():
         L.qsgd_encode_elias_static.restype = C.c_int
         L.qsgd_launch_count.argtypes = []
         L.qsgd_launch_count.restype = u64
+        pu64, pu32, pp = C.POINTER(u64), C.POINTER(u32), C.POINTER(PolicyStruct)
+        L.qsgd_policy_plan_sizes.argtypes = [pu64, u32, u32, u64, pu64, pu64, pu64]
+        L.qsgd_policy_plan_sizes.restype = C.c_int
+        L.qsgd_policy_plan.argtypes = [pu64, u32, u32, u64, pu64, pu32, pu64, pu64, pu32]
+        L.qsgd_policy_plan.restype = C.c_int
+        L.qsgd_policy_message_capacity.argtypes = [pp, u32, u32, C.c_int]
+        L.qsgd_policy_message_capacity.restype = sz
+        L.qsgd_policy_workspace_bytes.argtypes = [pp, u32, u32, C.c_int]
+        L.qsgd_policy_workspace_bytes.restype = sz
+        L.qsgd_policy_encode.argtypes = [vp, pp, u32, u32, C.c_int, C.c_int, u64, u32, u32, vp, sz, vp,
+                                         vp, vp, vp]
+        L.qsgd_policy_encode.restype = C.c_int
+        L.qsgd_policy_decode_accumulate.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, pp, u32, u32,
+                                                    C.c_int, vp, vp, vp]
+        L.qsgd_policy_decode_accumulate.restype = C.c_int
+        L.qsgd_policy_decode_sgd_step.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, pp, u32, u32,
+                                                  C.c_int, vp, C.c_float, vp, vp]
+        L.qsgd_policy_decode_sgd_step.restype = C.c_int
         L.qsgd_profile_enable.argtypes = [C.c_int]
         L.qsgd_profile_enable.restype = None
         L.qsgd_profile_kernel_count.argtypes = []
@@ -188,6 +216,79 @@ def qsgd_decode_sgd_step(msgs, tables, n, bucket, s, code_kind, x, eta, status_d
     tp = None if tables is None else _ptr_array(tables)
     _check(lib().qsgd_decode_sgd_step(mp, tp, len(msgs), n, bucket, s, code_kind, x.data_ptr(),
                                       eta, status_dev.data_ptr(), _stream(stream)))
+
+
+# ------------------------------- per-tensor policy -------------------------------------------
+class Policy:
+    """A plan made by qsgd_policy_plan for tensors of the given sizes, with its arrays copied to
+    the device (the copies are the only thing this class adds to the C calls)."""
+
+    def __init__(self, tensor_sizes, bucket, min_quantized=10000, device="cuda"):
+        T = len(tensor_sizes)
+        sizes = (C.c_uint64 * max(T, 1))(*[int(m) for m in tensor_sizes])
+        nb, ns, nr = C.c_uint64(), C.c_uint64(), C.c_uint64()
+        _check(lib().qsgd_policy_plan_sizes(sizes, T, bucket, min_quantized, C.byref(nb), C.byref(ns), C.byref(nr)))
+        nb, ns, nr = nb.value, ns.value, nr.value
+        src = torch.zeros(max(nb, 1), dtype=torch.int64)
+        ln = torch.zeros(max(nb, 1), dtype=torch.int32)
+        rsrc = torch.zeros(max(ns, 1), dtype=torch.int64)
+        rstart = torch.zeros(ns + 1, dtype=torch.int64)
+        quads = C.c_uint32()
+        as_p = lambda t, ct: C.cast(t.data_ptr(), C.POINTER(ct))
+        _check(lib().qsgd_policy_plan(sizes, T, bucket, min_quantized, as_p(src, C.c_uint64), as_p(ln, C.c_uint32),
+                                      as_p(rsrc, C.c_uint64), as_p(rstart, C.c_uint64), C.byref(quads)))
+        self.bucket = bucket
+        self.host = {"bucket_src": src[:nb], "bucket_len": ln[:nb], "raw_src": rsrc[:ns], "raw_start": rstart}
+        self.dev = {k: v.to(device) for k, v in (("bucket_src", src), ("bucket_len", ln), ("raw_src", rsrc),
+                                                ("raw_start", rstart))}
+        self.n = int(sum(int(m) for m in tensor_sizes))
+        self.n_buckets, self.n_raw_segments, self.n_raw, self.quads = nb, ns, nr, quads.value
+        self.raw_prefix = (4 * nr + 15) // 16 * 16
+        self.struct = PolicyStruct(self.dev["bucket_src"].data_ptr(), self.dev["bucket_len"].data_ptr(), nb,
+                                   self.dev["raw_src"].data_ptr(), self.dev["raw_start"].data_ptr(), ns, nr,
+                                   self.n, quads.value)
+
+
+def qsgd_policy_message_capacity(plan, s, code_kind):
+    return int(lib().qsgd_policy_message_capacity(C.byref(plan.struct), plan.bucket, s, code_kind))
+
+
+def qsgd_policy_workspace_bytes(plan, s, code_kind):
+    return int(lib().qsgd_policy_workspace_bytes(C.byref(plan.struct), plan.bucket, s, code_kind))
+
+
+def qsgd_policy_encode(g, plan, s, norm_kind, code_kind, seed, step, worker, out, out_bits, workspace=None,
+                       status_dev=None, stream=None):
+    _require_cuda(g, "g")
+    _require_cuda(out, "out")
+    _require_cuda(out_bits, "out_bits")
+    _require_cuda(status_dev, "status_dev")
+    if g.numel() != plan.n:
+        raise QsgdError("g has %d elements, the plan covers %d" % (g.numel(), plan.n))
+    ws = None if workspace is None else C.c_void_p(workspace.data_ptr())
+    _check(lib().qsgd_policy_encode(g.data_ptr(), C.byref(plan.struct), plan.bucket, s, norm_kind, code_kind, seed,
+                                    step, worker, out.data_ptr(), out.numel() * out.element_size(),
+                                    out_bits.data_ptr(), ws, status_dev.data_ptr(), _stream(stream)))
+
+
+def qsgd_policy_decode_accumulate(msgs, tables, plan, s, code_kind, acc, status_dev, stream=None):
+    _require_cuda(acc, "acc")
+    if acc.numel() != plan.n:
+        raise QsgdError("acc has %d elements, the plan covers %d" % (acc.numel(), plan.n))
+    mp = _ptr_array(msgs)
+    tp = None if tables is None else _ptr_array(tables)
+    _check(lib().qsgd_policy_decode_accumulate(mp, tp, len(msgs), C.byref(plan.struct), plan.bucket, s, code_kind,
+                                               acc.data_ptr(), status_dev.data_ptr(), _stream(stream)))
+
+
+def qsgd_policy_decode_sgd_step(msgs, tables, plan, s, code_kind, x, eta, status_dev, stream=None):
+    _require_cuda(x, "x")
+    if x.numel() != plan.n:
+        raise QsgdError("x has %d elements, the plan covers %d" % (x.numel(), plan.n))
+    mp = _ptr_array(msgs)
+    tp = None if tables is None else _ptr_array(tables)
+    _check(lib().qsgd_policy_decode_sgd_step(mp, tp, len(msgs), C.byref(plan.struct), plan.bucket, s, code_kind,
+                                             x.data_ptr(), eta, status_dev.data_ptr(), _stream(stream)))
 
 
 # ------------------------------- conveniences (allocation only) -----------------------------

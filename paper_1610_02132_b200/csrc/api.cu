@@ -34,7 +34,7 @@ ScopedKernel::~ScopedKernel() {
 
 static const char* const kKernelNames[kKernCount] = {
     "quantize_fixed", "quantize_tail", "decode_fixed", "sgd_step", "elias_length",
-    "elias_scatter", "decode_elias", "decode_elias_sparse"};
+    "elias_scatter", "decode_elias", "decode_elias_sparse", "raw_gather", "raw_decode"};
 
 namespace {
 
@@ -133,7 +133,7 @@ int qsgd_encode(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int nor
     const FixedLayout L = make_fixed_layout(n, bucket, s);
     if (out_capacity < L.total) return QSGD_ERR_CAPACITY;
     return launch_quantize_fixed(g, n, bucket, s, norm_kind, seed, step, worker,
-                                 static_cast<uint8_t*>(out), status_dev, out_bits, nullptr, cs);
+                                 static_cast<uint8_t*>(out), status_dev, out_bits, nullptr, no_map(), cs);
   }
   if (!workspace) return QSGD_ERR_NULL;
   if (!aligned16(workspace)) return QSGD_ERR_ALIGN;
@@ -141,7 +141,7 @@ int qsgd_encode(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int nor
   if (out_capacity < align16(4 * B) + 8 * (B + 1)) return QSGD_ERR_CAPACITY;   // scales + table
   return launch_elias_encode(g, n, bucket, s, norm_kind, code_kind == QSGD_CODE_ELIAS_DENSE, seed,
                              step, worker, static_cast<uint8_t*>(out), out_capacity, out_bits,
-                             static_cast<uint8_t*>(workspace), status_dev, cs);
+                             static_cast<uint8_t*>(workspace), status_dev, no_map(), cs);
 }
 
 int qsgd_decode_accumulate(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
@@ -155,9 +155,9 @@ int qsgd_decode_accumulate(const void* const* msgs, const uint64_t* const* table
   st = resolve_peers(msgs, tables, K, n, bucket, s, code_kind, &ps);
   if (st) return st;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  if (code_kind == QSGD_CODE_FIXED) return launch_decode_fixed(ps, K, n, bucket, s, acc, false, 0.f, cs);
+  if (code_kind == QSGD_CODE_FIXED) return launch_decode_fixed(ps, K, n, bucket, s, acc, false, 0.f, no_map(), cs);
   return launch_decode_elias(ps, K, n, bucket, s, code_kind == QSGD_CODE_ELIAS_DENSE, acc, false, 0.f,
-                             status_dev, cs);
+                             status_dev, no_map(), cs);
 }
 
 int qsgd_sgd_step(float* x, const float* acc, float eta, uint32_t K, uint64_t n,
@@ -180,9 +180,159 @@ int qsgd_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables,
   st = resolve_peers(msgs, tables, K, n, bucket, s, code_kind, &ps);
   if (st) return st;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  if (code_kind == QSGD_CODE_FIXED) return launch_decode_fixed(ps, K, n, bucket, s, x, true, eta, cs);
+  if (code_kind == QSGD_CODE_FIXED) return launch_decode_fixed(ps, K, n, bucket, s, x, true, eta, no_map(), cs);
   return launch_decode_elias(ps, K, n, bucket, s, code_kind == QSGD_CODE_ELIAS_DENSE, x, true, eta,
-                             status_dev, cs);
+                             status_dev, no_map(), cs);
+}
+
+// ---- per-tensor policy --------------------------------------------------------------------------
+int qsgd_policy_plan_sizes(const uint64_t* tensor_sizes, uint32_t T, uint32_t bucket, uint64_t min_quantized,
+                           uint64_t* n_buckets, uint64_t* n_raw_segments, uint64_t* n_raw) {
+  if (!tensor_sizes || !n_buckets || !n_raw_segments || !n_raw) return QSGD_ERR_NULL;
+  if (bucket < 32 || bucket > QSGD_MAX_BUCKET || (bucket & 31u)) return QSGD_ERR_BUCKET;
+  uint64_t nb = 0, ns = 0, nr = 0, total = 0;
+  for (uint32_t t = 0; t < T; ++t) {
+    const uint64_t m = tensor_sizes[t];
+    total += m;
+    if (m >= min_quantized && m > 0) nb += (m + bucket - 1) / bucket;
+    else if (m > 0) { ++ns; nr += m; }
+  }
+  if (total == 0) return QSGD_ERR_SIZE;
+  *n_buckets = nb; *n_raw_segments = ns; *n_raw = nr;
+  return QSGD_OK;
+}
+
+int qsgd_policy_plan(const uint64_t* tensor_sizes, uint32_t T, uint32_t bucket, uint64_t min_quantized,
+                     uint64_t* bucket_src, uint32_t* bucket_len, uint64_t* raw_src, uint64_t* raw_start,
+                     uint32_t* quads) {
+  uint64_t nb, ns, nr;
+  const int st = qsgd_policy_plan_sizes(tensor_sizes, T, bucket, min_quantized, &nb, &ns, &nr);
+  if (st) return st;
+  if (!quads || (nb && (!bucket_src || !bucket_len)) || !raw_start || (ns && !raw_src)) return QSGD_ERR_NULL;
+  uint64_t off = 0, b = 0, seg = 0, r = 0;
+  bool q = true;
+  for (uint32_t t = 0; t < T; ++t) {
+    const uint64_t m = tensor_sizes[t];
+    if (m >= min_quantized && m > 0) {
+      for (uint64_t c = 0; c < m; c += bucket, ++b) {
+        bucket_src[b] = off + c;
+        bucket_len[b] = (uint32_t)(m - c < bucket ? m - c : bucket);
+        q = q && ((bucket_src[b] | bucket_len[b]) & 3ull) == 0;
+      }
+    } else if (m > 0) {
+      raw_src[seg] = off;
+      raw_start[seg] = r;
+      ++seg;
+      r += m;
+    }
+    off += m;
+  }
+  raw_start[seg] = r;
+  *quads = q ? 1u : 0u;
+  return QSGD_OK;
+}
+
+static int check_policy(const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind) {
+  if (!plan) return QSGD_ERR_NULL;
+  if (plan->n == 0 || (plan->n_buckets == 0 && plan->n_raw == 0)) return QSGD_ERR_SIZE;
+  if (plan->n_buckets && (!plan->bucket_src || !plan->bucket_len)) return QSGD_ERR_NULL;
+  if (plan->n_raw && (!plan->raw_src || !plan->raw_start || plan->n_raw_segments == 0)) return QSGD_ERR_NULL;
+  return check_shape(plan->n_buckets ? plan->n_buckets * bucket : 1, bucket, s, code_kind);
+}
+
+static RawSegments raw_of(const qsgd_policy* plan) {
+  return RawSegments{plan->raw_src, plan->raw_start, plan->n_raw_segments, plan->n_raw};
+}
+
+static BucketMap map_of(const qsgd_policy* plan) {
+  return BucketMap{plan->bucket_src, plan->bucket_len, plan->quads};
+}
+
+size_t qsgd_policy_message_capacity(const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind) {
+  if (check_policy(plan, bucket, s, code_kind) != QSGD_OK) return 0;
+  const size_t prefix = (size_t)align16(4 * plan->n_raw);
+  return prefix + (plan->n_buckets ? qsgd_message_capacity(plan->n_buckets * bucket, bucket, s, code_kind) : 0);
+}
+
+size_t qsgd_policy_workspace_bytes(const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind) {
+  if (check_policy(plan, bucket, s, code_kind) != QSGD_OK || plan->n_buckets == 0) return 0;
+  return qsgd_workspace_bytes(plan->n_buckets * bucket, bucket, s, code_kind);
+}
+
+int qsgd_policy_encode(const float* g, const qsgd_policy* plan, uint32_t bucket, uint32_t s, int norm_kind,
+                       int code_kind, uint64_t seed, uint32_t step, uint32_t worker, void* out,
+                       size_t out_capacity, uint64_t* out_bits, void* workspace, uint32_t* status_dev,
+                       qsgd_stream_t stream) {
+  if (!g || !out || !out_bits || !status_dev) return QSGD_ERR_NULL;
+  int st = check_policy(plan, bucket, s, code_kind);
+  if (st) return st;
+  if (norm_kind != QSGD_NORM_L2 && norm_kind != QSGD_NORM_MAX) return QSGD_ERR_KIND;
+  if (!aligned16(g) || !aligned16(out)) return QSGD_ERR_ALIGN;
+  const size_t prefix = (size_t)align16(4 * plan->n_raw);
+  if (out_capacity < prefix) return QSGD_ERR_CAPACITY;
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const uint64_t nc = plan->n_buckets * bucket;
+  if (nc) {
+    uint8_t* body = static_cast<uint8_t*>(out) + prefix;
+    const size_t cap = out_capacity - prefix;
+    if (code_kind == QSGD_CODE_FIXED) {
+      if (cap < make_fixed_layout(nc, bucket, s).total) return QSGD_ERR_CAPACITY;
+      st = launch_quantize_fixed(g, nc, bucket, s, norm_kind, seed, step, worker, body, status_dev, out_bits,
+                                 nullptr, map_of(plan), cs);
+    } else {
+      if (!workspace) return QSGD_ERR_NULL;
+      if (!aligned16(workspace)) return QSGD_ERR_ALIGN;
+      if (cap < align16(4 * plan->n_buckets) + 8 * (plan->n_buckets + 1)) return QSGD_ERR_CAPACITY;
+      st = launch_elias_encode(g, nc, bucket, s, norm_kind, code_kind == QSGD_CODE_ELIAS_DENSE, seed, step,
+                               worker, body, cap, out_bits, static_cast<uint8_t*>(workspace), status_dev,
+                               map_of(plan), cs);
+    }
+    if (st) return st;
+  }
+  return launch_raw_gather(g, raw_of(plan), static_cast<float*>(out), out_bits, nc != 0, cs);
+}
+
+static int policy_decode(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
+                         const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind, float* out,
+                         bool fused, float eta, uint32_t* status_dev, qsgd_stream_t stream) {
+  if (!out || !status_dev || !msgs) return QSGD_ERR_NULL;
+  int st = check_policy(plan, bucket, s, code_kind);
+  if (st) return st;
+  if (K < 1 || K > QSGD_MAX_PEERS) return QSGD_ERR_PEERS;
+  if (!aligned16(out)) return QSGD_ERR_ALIGN;
+  const size_t prefix = (size_t)align16(4 * plan->n_raw);
+  const void* body[QSGD_MAX_PEERS];
+  const float* raw[QSGD_MAX_PEERS];
+  for (uint32_t k = 0; k < K; ++k) {
+    if (!msgs[k]) return QSGD_ERR_NULL;
+    if (!aligned16(msgs[k])) return QSGD_ERR_ALIGN;
+    body[k] = static_cast<const uint8_t*>(msgs[k]) + prefix;
+    raw[k] = static_cast<const float*>(msgs[k]);
+  }
+  cudaStream_t cs = static_cast<cudaStream_t>(stream);
+  const uint64_t nc = plan->n_buckets * bucket;
+  if (nc) {
+    PeerSet ps;
+    st = resolve_peers(body, tables, K, nc, bucket, s, code_kind, &ps);
+    if (st) return st;
+    if (code_kind == QSGD_CODE_FIXED) st = launch_decode_fixed(ps, K, nc, bucket, s, out, fused, eta, map_of(plan), cs);
+    else st = launch_decode_elias(ps, K, nc, bucket, s, code_kind == QSGD_CODE_ELIAS_DENSE, out, fused, eta,
+                                  status_dev, map_of(plan), cs);
+    if (st) return st;
+  }
+  return launch_raw_decode(raw, K, raw_of(plan), out, fused, eta, cs);
+}
+
+int qsgd_policy_decode_accumulate(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
+                                  const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind,
+                                  float* acc, uint32_t* status_dev, qsgd_stream_t stream) {
+  return policy_decode(msgs, tables, K, plan, bucket, s, code_kind, acc, false, 0.f, status_dev, stream);
+}
+
+int qsgd_policy_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
+                                const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind,
+                                float* x, float eta, uint32_t* status_dev, qsgd_stream_t stream) {
+  return policy_decode(msgs, tables, K, plan, bucket, s, code_kind, x, true, eta, status_dev, stream);
 }
 
 const char* qsgd_status_string(int status) {

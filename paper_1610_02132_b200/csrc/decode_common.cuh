@@ -109,4 +109,39 @@ __device__ __forceinline__ void store_lane16(float* o, const float (&acc)[16], u
   }
 }
 
+// Where `want` consecutive coordinates of bucket b, starting at bucket-relative position c0, live in
+// the output array, and how many of them exist.
+struct OutSpan {
+  float* ptr;
+  uint32_t valid;
+};
+
+__device__ __forceinline__ OutSpan out_span(float* out, const BucketMap& map, uint64_t b, uint32_t c0, uint32_t d,
+                                            uint64_t n, uint32_t want) {
+  OutSpan sp;
+  if (map.src) {
+    const uint32_t L = __ldg(map.len + b);
+    sp.ptr = out + __ldg(map.src + b) + c0;
+    sp.valid = c0 < L ? min(want, L - c0) : 0u;
+  } else {
+    const uint64_t i0 = b * d + c0;
+    sp.ptr = out + i0;
+    sp.valid = i0 < n ? (uint32_t)min((uint64_t)want, n - i0) : 0u;
+  }
+  return sp;
+}
+
+// store_lane16 through a span: vector accesses when all 16 values exist and the place is 16-byte
+// aligned, element by element otherwise.
+template <bool FUSED>
+__device__ __forceinline__ void store_span16(const OutSpan& sp, const float (&acc)[16], float c) {
+  if (sp.valid == 16u && (reinterpret_cast<uintptr_t>(sp.ptr) & 15u) == 0) {
+    store_lane16<FUSED>(sp.ptr, acc, 0, 16, c);
+  } else {
+#pragma unroll
+    for (int e = 0; e < 16; ++e)
+      if ((uint32_t)e < sp.valid) sp.ptr[e] = FUSED ? __fsub_rn(sp.ptr[e], __fmul_rn(c, acc[e])) : acc[e];
+  }
+}
+
 }  // namespace qsgd

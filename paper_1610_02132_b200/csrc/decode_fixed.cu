@@ -30,6 +30,7 @@ struct DecodeParams {
   float* out;      // acc (overwritten) or x (updated in place)
   float c;         // eta / K (fused only)
   uint64_t chunks;
+  BucketMap map;
 };
 
 template <int LB, bool FUSED, bool SINGLE>
@@ -82,22 +83,10 @@ __global__ void __launch_bounds__(kThreads, 4) decode_fixed_kernel(const __grid_
     }
 
     if (!live) continue;
-    float* o = p.out + i0;
-    if (i0 + 16 <= p.n) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        float4 r = make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
-        if (FUSED) {
-          const float4 x = *reinterpret_cast<const float4*>(o + 4 * j);
-          r.x = __fsub_rn(x.x, __fmul_rn(p.c, r.x)); r.y = __fsub_rn(x.y, __fmul_rn(p.c, r.y));
-          r.z = __fsub_rn(x.z, __fmul_rn(p.c, r.z)); r.w = __fsub_rn(x.w, __fmul_rn(p.c, r.w));
-        }
-        *reinterpret_cast<float4*>(o + 4 * j) = r;
-      }
+    if (p.map.src) {                                              // per-tensor policy: buckets live elsewhere
+      store_span16<FUSED>(out_span(p.out, p.map, b, (uint32_t)(i0 - b * p.d), p.d, p.n, 16u), acc, p.c);
     } else {
-#pragma unroll
-      for (int e = 0; e < 16; ++e)
-        if (i0 + e < p.n) o[e] = FUSED ? __fsub_rn(o[e], __fmul_rn(p.c, acc[e])) : acc[e];
+      store_lane16<FUSED>(p.out + i0, acc, i0, p.n, p.c);
     }
   }
 }
@@ -149,9 +138,9 @@ int launch_lb(const DecodeParams& p, bool fused, bool single, cudaStream_t strea
 }  // namespace
 
 int launch_decode_fixed(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s,
-                        float* acc_or_x, bool fused, float eta, cudaStream_t stream) {
+                        float* acc_or_x, bool fused, float eta, const BucketMap& map, cudaStream_t stream) {
   DecodeParams p;
-  p.peers = peers; p.K = K; p.n = n; p.d = d; p.s = s; p.out = acc_or_x;
+  p.peers = peers; p.K = K; p.n = n; p.d = d; p.s = s; p.out = acc_or_x; p.map = map;
   p.c = eta / (float)K;
   p.chunks = (n + kChunk - 1) / kChunk;
   // one scale per chunk when the bucket size is 512 * 2^j

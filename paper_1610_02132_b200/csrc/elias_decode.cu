@@ -34,6 +34,7 @@ struct EliasDecodeParams {
   uint32_t* status;
   uint32_t warp_bytes; // shared memory per warp
   uint32_t defer_sparse;  // a sparse-regime kernel was launched beside this one
+  BucketMap map;       // where the buckets live in `out` (per-tensor policy), or no map
 };
 
 // Work split of the sparse-regime decoder (defined further down): a warp owns G <= 32 / Kpad
@@ -188,10 +189,18 @@ __global__ void __launch_bounds__(kThreads) decode_elias_slow_kernel(const __gri
     }
 
     // write the bucket: acc, or the SGD step on x
-    for (uint32_t c = lane * 4; c < db; c += 128) {
+    float* orow = p.out + base;
+    uint32_t dbv = db;                                  // coordinates of the bucket that exist in `out`
+    bool vec = true;
+    if (p.map.src) {
+      orow = p.out + __ldg(p.map.src + b);
+      dbv = min(db, __ldg(p.map.len + b));
+      vec = p.map.quads != 0u;
+    }
+    for (uint32_t c = lane * 4; c < dbv; c += 128) {
       const float4 a = *reinterpret_cast<const float4*>(acc + c);
-      float* o = p.out + base + c;
-      if (c + 4 <= db) {
+      float* o = orow + c;
+      if (vec && c + 4 <= dbv) {
         float4 r = a;
         if (FUSED) {
           const float4 x = *reinterpret_cast<const float4*>(o);
@@ -201,7 +210,7 @@ __global__ void __launch_bounds__(kThreads) decode_elias_slow_kernel(const __gri
         *reinterpret_cast<float4*>(o) = r;
       } else {
         const float t[4] = {a.x, a.y, a.z, a.w};
-        for (uint32_t j = 0; c + j < db; ++j) o[j] = FUSED ? __fsub_rn(o[j], __fmul_rn(p.c, t[j])) : t[j];
+        for (uint32_t j = 0; j < 4 && c + j < dbv; ++j) o[j] = FUSED ? __fsub_rn(o[j], __fmul_rn(p.c, t[j])) : t[j];
       }
     }
     __syncwarp();
@@ -255,6 +264,7 @@ struct FieldParams {
   uint32_t row_words;   // per peer row: d * lb / 32 level words, then d / 32 sign words (padded to 4)
   uint32_t bucket_words;  // K rows + K scales, padded to 4
   uint32_t defer_sparse;  // a sparse-regime kernel was launched beside this one
+  BucketMap map;          // where the buckets live in `out` (per-tensor policy), or no map
 };
 
 // Bit source over the payload: a 64-bit left-aligned window held as two 32-bit halves (all
@@ -451,6 +461,7 @@ struct SparseParams {
   uint32_t warp_words;   // shared-memory words per warp: G * R sums, 64 of scales and counts, 32 lists
   uint32_t quad_shift;   // log2(R / 4) when R is a power of two, else 32
   uint32_t check_regime; // 0: the host already knows that this kernel is the one to run
+  BucketMap map;         // where the buckets live in `out` (per-tensor policy), or no map
 };
 
 // The recursive Elias code (Definition A.1) of one integer below 2^16, decoded without branches
@@ -564,7 +575,14 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
     st.pend = kNoEntry;
     uint32_t db = 0;                                           // coordinates of this lane's bucket
     float A = 0.f;
-    if (pg < G && b0 + pg < p.B) db = (uint32_t)min((uint64_t)p.d, p.n - (b0 + pg) * p.d);
+    float* xrow = p.out + (b0 + pg) * (uint64_t)p.d;            // this lane's bucket in the output
+    if (pg < G && b0 + pg < p.B) {
+      db = (uint32_t)min((uint64_t)p.d, p.n - (b0 + pg) * p.d);
+      if (p.map.src) {                                           // per-tensor policy: the bucket lives elsewhere
+        db = min(db, __ldg(p.map.len + b0 + pg));
+        xrow = p.out + __ldg(p.map.src + b0 + pg);
+      }
+    }
     const bool parsing = db != 0u && pk < p.K;
     if (parsing) {
       const uint64_t b = b0 + pg;
@@ -583,7 +601,6 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
     }
     scales[lane] = A;
     const bool bad_scale = !(fabsf(A) <= 3.402823466e+38f);
-    float* xrow = p.out + (b0 + pg) * (uint64_t)p.d;            // this lane's bucket in x (valid when db != 0)
 
     for (uint32_t rbeg = 0; rbeg < p.d; rbeg += R) {
       const uint32_t rend = min(rbeg + R, p.d);
@@ -656,26 +673,34 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
         __syncwarp();
         continue;
       }
-      // Otherwise scan the G ranges (each contiguous in memory).
+      // Otherwise scan the G ranges (each contiguous in memory). The place and the length of
+      // bucket g are held by the lanes that parse it.
       const uint32_t range_quads = (rend - rbeg) >> 2;
+      const bool vec_ok = !p.map.src || p.map.quads != 0u;
+      const uint64_t my_row = (uint64_t)(xrow - p.out);
       for (uint32_t q0 = 0; q0 < G * tile_quads; q0 += 32 * kU) {
         float4 t[kU], x[kU];
         uint64_t at[kU];
-        uint32_t need = 0, full = 0;
+        uint32_t cnt[kU];                                   // values of the quad to write (0: none)
+        uint32_t full = 0;
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
           const uint32_t q = q0 + u * 32 + lane;
           const uint32_t g = p.quad_shift < 32u ? q >> p.quad_shift : q / tile_quads;
           const uint32_t j = q - g * tile_quads;
-          at[u] = (b0 + g) * p.d + rbeg + 4u * j;
+          const uint64_t row = __shfl_sync(0xffffffffu, my_row, (int)(g * Kpad));
+          const uint32_t dbg = __shfl_sync(0xffffffffu, db, (int)(g * Kpad));
+          const uint32_t pos = rbeg + 4u * j;
+          at[u] = row + pos;
+          cnt[u] = 0;
           t[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (q < G * tile_quads && j < range_quads && b0 + g < p.B && at[u] < p.n) {
+          if (q < G * tile_quads && j < range_quads && pos < dbg) {
             t[u] = tile4[q];
             const bool any = ((__float_as_uint(t[u].x) | __float_as_uint(t[u].y) | __float_as_uint(t[u].z) | __float_as_uint(t[u].w)) != 0u);
             if (any) tile4[q] = make_float4(0.f, 0.f, 0.f, 0.f);
             if (any || !skip_zero) {
-              need |= 1u << u;
-              if (at[u] + 4 <= p.n) full |= 1u << u;
+              cnt[u] = min(4u, dbg - pos);
+              if (cnt[u] == 4u && vec_ok) full |= 1u << u;
             }
           }
         }
@@ -686,7 +711,7 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
         }
 #pragma unroll
         for (int u = 0; u < kU; ++u) {
-          if (!((need >> u) & 1u)) continue;
+          if (cnt[u] == 0u) continue;
           float* o = p.out + at[u];
           if ((full >> u) & 1u) {
             float4 r = t[u];
@@ -695,10 +720,11 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
               r.z = __fsub_rn(x[u].z, __fmul_rn(p.c, r.z)); r.w = __fsub_rn(x[u].w, __fmul_rn(p.c, r.w));
             }
             *reinterpret_cast<float4*>(o) = r;
-          } else {                                            // the quad that straddles n
-            if (at[u] + 0 < p.n) o[0] = FUSED ? __fsub_rn(o[0], __fmul_rn(p.c, t[u].x)) : t[u].x;
-            if (at[u] + 1 < p.n) o[1] = FUSED ? __fsub_rn(o[1], __fmul_rn(p.c, t[u].y)) : t[u].y;
-            if (at[u] + 2 < p.n) o[2] = FUSED ? __fsub_rn(o[2], __fmul_rn(p.c, t[u].z)) : t[u].z;
+          } else {                                            // a ragged end, or a place that is not 16-byte aligned
+            o[0] = FUSED ? __fsub_rn(o[0], __fmul_rn(p.c, t[u].x)) : t[u].x;
+            if (cnt[u] > 1u) o[1] = FUSED ? __fsub_rn(o[1], __fmul_rn(p.c, t[u].y)) : t[u].y;
+            if (cnt[u] > 2u) o[2] = FUSED ? __fsub_rn(o[2], __fmul_rn(p.c, t[u].z)) : t[u].z;
+            if (cnt[u] > 3u) o[3] = FUSED ? __fsub_rn(o[3], __fmul_rn(p.c, t[u].w)) : t[u].w;
           }
         }
       }
@@ -714,7 +740,8 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
 // Launches the sparse-regime kernel when the configuration allows one (K <= 32, Code_s); the
 // caller then tells the other decoders to stand down when the predicate holds.
 int launch_sparse(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s, float* out, bool fused,
-                  float c, uint32_t* status, bool check_regime, cudaStream_t stream, bool* launched) {
+                  float c, uint32_t* status, bool check_regime, const BucketMap& map, cudaStream_t stream,
+                  bool* launched) {
   *launched = false;
   if (K > 32u) return 0;
   int dev = 0, sms = 0;
@@ -724,7 +751,7 @@ int launch_sparse(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint
   p.peers = peers; p.K = K; p.n = n; p.d = d; p.s = s;
   p.B = (n + d - 1) / d;
   p.sh = sparse_shape(K, d, p.B, (uint32_t)sms);
-  p.out = out; p.c = c; p.status = status; p.check_regime = check_regime ? 1u : 0u;
+  p.out = out; p.c = c; p.status = status; p.check_regime = check_regime ? 1u : 0u; p.map = map;
   p.warp_words = p.sh.G * p.sh.R + 64u + p.sh.G * p.sh.Kpad * p.sh.C;
   p.quad_shift = 32;
   const uint32_t tile_quads = p.sh.R >> 2;
@@ -838,7 +865,10 @@ __global__ void __launch_bounds__(128) decode_elias_fields_kernel(const __grid_c
         else if (SINGLE) add_peer_lut<LB, true>(acc, w, sb, __fmul_rn(__shfl_sync(0xffffffffu, A, 0), lut0), A);
         else add_peer_lut<LB, false>(acc, w, sb, lut0, A);
       }
-      if (live) store_lane16<FUSED>(p.out + i0, acc, i0, p.n, p.c);
+      if (live) {
+        if (p.map.src) store_span16<FUSED>(out_span(p.out, p.map, b, c, p.d, p.n, 16u), acc, p.c);
+        else store_lane16<FUSED>(p.out + i0, acc, i0, p.n, p.c);
+      }
     }
     __syncwarp();
   }
@@ -897,7 +927,7 @@ int launch_fields_lb(FieldParams& p, bool dense, bool fused, cudaStream_t stream
 
 int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s,
                         bool dense, float* acc_or_x, bool fused, float eta, uint32_t* status_dev,
-                        cudaStream_t stream) {
+                        const BucketMap& map, cudaStream_t stream) {
   // Which decoder? In a message the offset table follows the padded payload, so table - payload is
   // the payload size and the host can evaluate the regime predicate itself (to within the padding)
   // and launch one kernel. With tables kept elsewhere the sizes are only known on the device: both
@@ -919,11 +949,11 @@ int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d
     FieldParams f;
     f.peers = peers; f.K = K; f.n = n; f.d = d; f.s = s;
     f.B = B;
-    f.out = acc_or_x; f.c = eta / (float)K; f.status = status_dev;
+    f.out = acc_or_x; f.c = eta / (float)K; f.status = status_dev; f.map = map;
     bool handled = false;
     int st = 0;
     if (!dense && (host_sparse || !sizes_known))
-      st = launch_sparse(peers, K, n, d, s, acc_or_x, fused, f.c, status_dev, !sizes_known, stream, &sparse);
+      st = launch_sparse(peers, K, n, d, s, acc_or_x, fused, f.c, status_dev, !sizes_known, map, stream, &sparse);
     if (st) return st;
     if (sparse && sizes_known) return 0;                    // the host chose the sparse-regime kernel
     f.defer_sparse = sparse ? 1u : 0u;
@@ -939,7 +969,7 @@ int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d
   p.peers = peers; p.K = K; p.Kc = K; p.n = n; p.d = d; p.s = s;
   p.B = (n + d - 1) / d;
   p.out = acc_or_x; p.c = eta / (float)K; p.status = status_dev; p.warp_bytes = 0;
-  p.defer_sparse = sparse ? 1u : 0u;
+  p.defer_sparse = sparse ? 1u : 0u; p.map = map;
   if (s <= 127) return dense ? launch_slow<uint8_t, true>(p, fused, stream) : launch_slow<uint8_t, false>(p, fused, stream);
   return dense ? launch_slow<uint16_t, true>(p, fused, stream) : launch_slow<uint16_t, false>(p, fused, stream);
 }

@@ -553,10 +553,10 @@ size_t elias_workspace_bytes(uint64_t n, uint32_t d, uint32_t s) {
 int launch_elias_encode(const float* g, uint64_t n, uint32_t d, uint32_t s, int norm_kind,
                         bool dense, uint64_t seed, uint32_t step, uint32_t worker, uint8_t* out,
                         size_t out_capacity, uint64_t* out_bits, uint8_t* workspace,
-                        uint32_t* status_dev, cudaStream_t stream) {
+                        uint32_t* status_dev, const BucketMap& map, cudaStream_t stream) {
   const EliasWs w = carve(workspace, n, d, s);
   int st = launch_quantize_fixed(g, n, d, s, norm_kind, seed, step, worker, w.fixed, status_dev, nullptr,
-                                 &w.ctrl->arrived, stream);
+                                 &w.ctrl->arrived, map, stream);
   if (st) return st;
   const FixedLayout L = make_fixed_layout(n, d, s);
   BucketParams bp;
@@ -642,7 +642,7 @@ int qsgd_encode_elias_static(const float* g, uint64_t n, uint32_t bucket, uint32
   if (st) return st;
   return launch_elias_encode(g, n, bucket, s, norm_kind, code_kind == QSGD_CODE_ELIAS_DENSE, seed, step,
                              worker, static_cast<uint8_t*>(out), out_capacity, out_bits, scratch,
-                             status_dev, static_cast<cudaStream_t>(stream));
+                             status_dev, no_map(), static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

@@ -92,12 +92,25 @@ struct PeerSet {                 // K messages, resolved to region pointers on t
   const uint64_t* table[QSGD_MAX_PEERS];   // Elias: offset tables
 };
 
+// Per-tensor policy (Section 5, "Protocol"): the coordinates that get quantized form a "compact"
+// vector of whole buckets, and bucket b of it lives at elements [src[b], src[b] + len[b]) of the flat
+// gradient (len[b] <= d; the rest of the bucket is zero padding that exists nowhere in memory).
+// src == nullptr means the ordinary case: the compact vector is the flat array itself.
+struct BucketMap {
+  const uint64_t* src;     // device, one entry per bucket
+  const uint32_t* len;     // device, one entry per bucket
+  uint32_t quads;          // nonzero when every src and len is a multiple of 4 (16-byte accesses stay legal)
+};
+
+inline BucketMap no_map() { return BucketMap{nullptr, nullptr, 1u}; }
+
 int launch_quantize_fixed(const float* g, uint64_t n, uint32_t d, uint32_t s, int norm_kind,
                           uint64_t seed, uint32_t step, uint32_t worker, uint8_t* out,
-                          uint32_t* status_dev, uint64_t* info, uint32_t* clear_word, cudaStream_t stream);
+                          uint32_t* status_dev, uint64_t* info, uint32_t* clear_word, const BucketMap& map,
+                          cudaStream_t stream);
 
 int launch_decode_fixed(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s,
-                        float* acc_or_x, bool fused, float eta, cudaStream_t stream);
+                        float* acc_or_x, bool fused, float eta, const BucketMap& map, cudaStream_t stream);
 
 int launch_sgd_step(float* x, const float* acc, float eta, uint32_t K, uint64_t n,
                     cudaStream_t stream);
@@ -107,18 +120,36 @@ size_t elias_workspace_bytes(uint64_t n, uint32_t d, uint32_t s);
 int launch_elias_encode(const float* g, uint64_t n, uint32_t d, uint32_t s, int norm_kind,
                         bool dense, uint64_t seed, uint32_t step, uint32_t worker, uint8_t* out,
                         size_t out_capacity, uint64_t* out_bits, uint8_t* workspace,
-                        uint32_t* status_dev, cudaStream_t stream);
+                        uint32_t* status_dev, const BucketMap& map, cudaStream_t stream);
 
 int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s,
                         bool dense, float* acc_or_x, bool fused, float eta, uint32_t* status_dev,
-                        cudaStream_t stream);
+                        const BucketMap& map, cudaStream_t stream);
+
+// Raw tensors of the per-tensor policy: segment j holds elements [raw_src[j], raw_src[j] + raw_start[j+1]
+// - raw_start[j]) of the flat array and sits at raw_start[j] in a message's raw region.
+struct RawSegments {
+  const uint64_t* src;     // device, R entries
+  const uint64_t* start;   // device, R + 1 entries, start[R] = n_raw
+  uint64_t R;
+  uint64_t n_raw;
+};
+
+// Copies the raw values into the front of a message and moves the message sizes in info[0..3]
+// (written by the encoder of the compact part) behind that raw region.
+int launch_raw_gather(const float* g, const RawSegments& raw, float* out_raw, uint64_t* info, bool has_compact,
+                      cudaStream_t stream);
+
+// Sum of the K raw regions in ascending k from +0, put at the tensors' places in acc, or applied to x.
+int launch_raw_decode(const float* const* raw_regions, uint32_t K, const RawSegments& raw, float* acc_or_x,
+                      bool fused, float eta, cudaStream_t stream);
 
 // Every kernel launch is bracketed by one of these: it counts the launch and, while kernel
 // timing is switched on (qsgd_profile_enable), records a CUDA event before and after it on the
 // launching stream.
 enum KernelId {
   kKernQuantize = 0, kKernQuantizeTail, kKernDecodeFixed, kKernSgdStep, kKernEliasLength,
-  kKernEliasScatter, kKernDecodeElias, kKernDecodeEliasSparse, kKernCount
+  kKernEliasScatter, kKernDecodeElias, kKernDecodeEliasSparse, kKernRawGather, kKernRawDecode, kKernCount
 };
 
 struct ScopedKernel {

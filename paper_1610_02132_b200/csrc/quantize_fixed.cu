@@ -45,6 +45,7 @@ struct QuantizeParams {
   uint64_t* info;         // optional: the four message-info words of a fixed-width message
   uint64_t total_bytes;
   uint32_t* clear_word;   // optional: a word the kernel sets to zero (arrival counter of a later kernel)
+  BucketMap map;          // per-tensor policy: where each bucket lives in g, or no map
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -176,12 +177,38 @@ struct FastParams {
   uint32_t* clear_word;     // optional word set to zero by CTA 0
   PhiloxConsts pc;
   uint32_t main_ctas;       // CTAs that stream complete tiles
+  BucketMap map;            // per-tensor policy: where each bucket lives in g (quads set), or no map
   QuantizeParams tail;      // parameters of the extra CTA (used when gridDim.x > main_ctas)
 };
 
 template <int LB, int NORM>
 __device__ __forceinline__ void quantize_generic_tile(const QuantizeParams& p, uint32_t block, uint32_t nblocks,
                                                       float* tile, float* part, float* s_rcp);
+
+// Producer side of one stage: start the bulk copies of tile t. Ordinary case: one copy of the whole
+// tile. With a bucket map every bucket of the tile is copied from its own place; a bucket that is
+// shorter than d gets zeros behind its values (plain stores, ordered before the copies' arrival by
+// the release of the expect-tx arrive). The map guarantees 16-byte aligned places and lengths.
+__device__ __forceinline__ void issue_tile(const FastParams& p, float* tile, uint64_t* full_bar, uint32_t t) {
+  if (!p.map.src) {
+    mbar_expect_tx(full_bar, kTile * 4);
+    bulk_load(tile, p.g + (size_t)t * kTile, kTile * 4, full_bar);
+    return;
+  }
+  const uint32_t d = 1u << p.log2d, nb = kTile >> p.log2d;
+  const uint64_t b0 = (uint64_t)t << (12u - p.log2d);
+  uint32_t bytes = 0;
+  for (uint32_t j = 0; j < nb; ++j) {
+    const uint32_t L = min(__ldg(p.map.len + b0 + j), d);
+    for (uint32_t c = L; c < d; c += 4) *reinterpret_cast<float4*>(tile + j * d + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+    bytes += 4u * L;
+  }
+  mbar_expect_tx(full_bar, bytes);
+  for (uint32_t j = 0; j < nb; ++j) {
+    const uint32_t L = min(__ldg(p.map.len + b0 + j), d);
+    if (L) bulk_load(tile + j * d, p.g + __ldg(p.map.src + b0 + j), 4u * L, full_bar);
+  }
+}
 
 // CROSS: a bucket spans several warps (d >= 1024); otherwise a bucket is d / 16 <= 32 lanes.
 // CTAs 0 .. main_ctas - 1 stream the complete tiles; one optional extra CTA runs the ragged last
@@ -213,10 +240,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
     if (blockIdx.x == 0 && p.clear_word) *p.clear_word = 0u;
     for (int s = 0; s < kStages; ++s) {
       const uint32_t t = blockIdx.x + (uint32_t)s * grid;
-      if (t < p.full_tiles) {
-        mbar_expect_tx(&sm.full[s], kTile * 4);
-        bulk_load(sm.tile[s], p.g + (size_t)t * kTile, kTile * 4, &sm.full[s]);
-      }
+      if (t < p.full_tiles) issue_tile(p, sm.tile[s], &sm.full[s], t);
     }
   }
 
@@ -274,8 +298,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
       const uint32_t tn = t + (uint32_t)(kStages - 1) * grid;             // tile of iteration it - 1 + kStages
       if (tn < p.full_tiles) {
         if (mbar_wait_bounded(&sm.empty[ps], pphase)) {
-          mbar_expect_tx(&sm.full[ps], kTile * 4);
-          bulk_load(sm.tile[ps], p.g + (size_t)tn * kTile, kTile * 4, &sm.full[ps]);
+          issue_tile(p, sm.tile[ps], &sm.full[ps], tn);
         } else {
           atomicOr(p.status, QSGD_DEV_TIMEOUT);
         }
@@ -419,7 +442,23 @@ __device__ __forceinline__ void quantize_generic_tile(const QuantizeParams& p, u
 
   for (uint32_t i = tid * 4; i < p.tile_coords; i += kThreads * 4) {
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (i + 4 <= valid) {
+    if (p.map.src) {
+      // per-tensor policy: four coordinates of one bucket (d is a multiple of 32) from the
+      // bucket's own place; what lies behind the bucket's length is zero padding
+      if (i < valid) {
+        const uint32_t bi = i / p.d, c = i - bi * p.d;
+        const uint64_t b = t0 / p.d + bi;
+        const uint32_t L = __ldg(p.map.len + b);
+        const float* src = p.g + __ldg(p.map.src + b) + c;
+        if (c + 4 <= L && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+          v = __ldcs(reinterpret_cast<const float4*>(src));
+        } else {
+          float t[4] = {0.f, 0.f, 0.f, 0.f};
+          for (uint32_t j = 0; j < 4 && c + j < L; ++j) t[j] = src[j];
+          v = make_float4(t[0], t[1], t[2], t[3]);
+        }
+      }
+    } else if (i + 4 <= valid) {
       v = __ldcs(reinterpret_cast<const float4*>(p.g + t0 + i));
     } else if (i < valid) {
       float t[4] = {0.f, 0.f, 0.f, 0.f};
@@ -610,7 +649,10 @@ int launch_one(QuantizeParams& p, uint64_t seed, cudaStream_t stream) {
   const uint32_t d = p.d;
   const bool pow2 = (d & (d - 1)) == 0;
   uint32_t full_tiles = 0;
-  if (pow2 && p.n <= (1ull << 32)) full_tiles = (uint32_t)(p.n / kTile);
+  // with a bucket map the bulk copies need 16-byte aligned places and lengths, and one copy per
+  // bucket is only worth issuing from a single thread when buckets are not tiny
+  const bool map_ok = !p.map.src || (p.map.quads != 0u && d >= 256);
+  if (pow2 && p.n <= (1ull << 32) && map_ok) full_tiles = (uint32_t)(p.n / kTile);
   if (full_tiles > 0) {
     FastParams fp;
     fp.g = p.g; fp.full_tiles = full_tiles; fp.s = p.s;
@@ -619,6 +661,7 @@ int launch_one(QuantizeParams& p, uint64_t seed, cudaStream_t stream) {
     fp.A_out = p.A_out; fp.sign_out = p.sign_out; fp.level_out = p.level_out; fp.status = p.status;
     fp.info = p.info; fp.total_bytes = p.total_bytes; fp.clear_word = p.clear_word;
     fp.pc = make_philox_consts(seed, p.step, p.worker);
+    fp.map = p.map;
     // the ragged tail (fewer than 4096 coordinates) and the zero padding of the three regions go
     // to one extra CTA of the same launch; nothing to do when n is a multiple of the tile and
     // every region already ends on a 16-byte boundary
@@ -652,10 +695,11 @@ int launch_lb(QuantizeParams& p, int norm_kind, uint64_t seed, cudaStream_t stre
 
 int launch_quantize_fixed(const float* g, uint64_t n, uint32_t d, uint32_t s, int norm_kind,
                           uint64_t seed, uint32_t step, uint32_t worker, uint8_t* out,
-                          uint32_t* status_dev, uint64_t* info, uint32_t* clear_word, cudaStream_t stream) {
+                          uint32_t* status_dev, uint64_t* info, uint32_t* clear_word, const BucketMap& map,
+                          cudaStream_t stream) {
   const FixedLayout L = make_fixed_layout(n, d, s);
   QuantizeParams p;
-  p.g = g; p.n = n; p.d = d; p.s = s;
+  p.g = g; p.n = n; p.d = d; p.s = s; p.map = map;
   p.tile_coords = (kTile / d) * d;
   p.coord_base = 0;
   p.k0 = (uint32_t)seed; p.k1 = (uint32_t)(seed >> 32); p.step = step; p.worker = worker;
