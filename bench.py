@@ -37,6 +37,13 @@ WORKLOADS = {
                     desc="AlexNet-shaped flat gradient, layer sigma 1e-2/sqrt(fan_in)"),
     "resnet152": dict(n=60192808, d=512, s=15, norm="l2", codes=["fixed", "elias"], K=16, gen="mixture",
                       desc="ResNet-152-shaped flat gradient, 0.9 N(0,1e-4^2) + 0.1 N(0,1e-2^2)"),
+    # Per-tensor policy (tensors under 10K elements raw, buckets cut to the tensors) on the two model shapes
+    "alexnet_policy": dict(n=61100840, d=512, s=255, norm="max", codes=["fixed"], K=16, gen="alexnet",
+                           policy="alexnet",
+                           desc="AlexNet-shaped gradient under the per-tensor policy (8 bias tensors raw)"),
+    "resnet152_policy": dict(n=60192808, d=512, s=15, norm="l2", codes=["fixed", "elias"], K=16, gen="mixture",
+                             policy="resnet152",
+                             desc="ResNet-152-shaped gradient under the per-tensor policy (313 small tensors raw)"),
     "sweep_point": dict(n=2 ** 28, d=512, s=15, norm="l2", codes=["fixed"], K=16, gen="gauss1",
                         desc="bandwidth sweep point: N(0,1), n=2^28"),
 }
@@ -47,6 +54,12 @@ PHILOX_SEED = 7
 
 def elen(k):
     return 1 if k == 1 else k.bit_length() + elen(k.bit_length() - 1)
+
+
+def policy_sizes(name):
+    from paper_1610_02132_b200 import inputs as I
+    shapes = I.alexnet_shapes() if name == "alexnet" else I.resnet152_shapes()
+    return [int(np.prod(sh)) for sh in shapes]
 
 
 def fixed_bytes(n, d, s):
@@ -158,6 +171,15 @@ class HotPath:
         n, d, s, K = wl["n"], wl["d"], wl["s"], wl["K"]
         self.n, self.d, self.s, self.K = n, d, s, K
         self.B = (n + d - 1) // d
+        # per-tensor policy: nq coordinates are quantized (whole buckets), the rest travel raw in
+        # `prefix` bytes in front of each message
+        self.plan, self.nq, self.n_raw, self.prefix = None, n, 0, 0
+        if wl.get("policy"):
+            sizes = policy_sizes(wl["policy"])
+            assert sum(sizes) == n, "policy workloads run at the model's own size"
+            self.plan = Q.Policy(sizes, d, device=device)
+            self.B, self.n_raw, self.prefix = self.plan.n_buckets, self.plan.n_raw, self.plan.raw_prefix
+            self.nq = self.B * d
         self.norm = NORM[wl["norm"]]
         self.codes = [CODE[c] for c in wl["codes"]]
         # the K workers' gradients (rank shifts the seeds so replicas differ)
@@ -169,7 +191,7 @@ class HotPath:
             cap = self.message_capacity(code)
             self.msgs[code] = [torch.empty(cap, dtype=torch.uint8, device=device) for _ in range(K)]
             self.bits[code] = torch.zeros(K, 4, dtype=torch.int64, device=device)
-            wsb = max(Q.qsgd_workspace_bytes(n, d, s, code), 16)
+            wsb = max(Q.qsgd_workspace_bytes(self.nq, d, s, code), 16)
             self.ws[code] = torch.empty(wsb, dtype=torch.uint8, device=device)
         self.info = {}
 
@@ -178,16 +200,20 @@ class HotPath:
         longer than that is not worth sending); a first encode verifies it fits."""
         Q = self.Q
         if code == 0:
-            return Q.qsgd_message_capacity(self.n, self.d, self.s, code)
-        worst = Q.qsgd_message_capacity(self.n, self.d, self.s, code)
-        return min(worst, 2 * fixed_bytes(self.n, self.d, self.s) + 8 * (self.B + 1))
+            return self.prefix + Q.qsgd_message_capacity(self.nq, self.d, self.s, code)
+        worst = Q.qsgd_message_capacity(self.nq, self.d, self.s, code)
+        return self.prefix + min(worst, 2 * fixed_bytes(self.nq, self.d, self.s) + 8 * (self.B + 1))
 
     def encode_all(self, code, step, src=None):
         Q = self.Q
         g = self.g if src is None else src
         for w in range(self.K):
-            Q.qsgd_encode(g[w], self.d, self.s, self.norm, code, PHILOX_SEED, step, w,
-                          self.msgs[code][w], self.bits[code][w], self.ws[code], self.status)
+            if self.plan is not None:
+                Q.qsgd_policy_encode(g[w], self.plan, self.s, self.norm, code, PHILOX_SEED, step, w,
+                                     self.msgs[code][w], self.bits[code][w], self.ws[code], self.status)
+            else:
+                Q.qsgd_encode(g[w], self.d, self.s, self.norm, code, PHILOX_SEED, step, w,
+                              self.msgs[code][w], self.bits[code][w], self.ws[code], self.status)
 
     def resolve_tables(self, code):
         """Elias: the sender reads the message length back (it needs it to send the message);
@@ -204,30 +230,36 @@ class HotPath:
         for code in self.codes:
             self.encode_all(code, step_idx, src)
             tables = self.resolve_tables(code)
-            self.Q.qsgd_decode_sgd_step(self.msgs[code], tables, self.n, self.d, self.s, code, self.x,
-                                        ETA, self.status)
+            if self.plan is not None:
+                self.Q.qsgd_policy_decode_sgd_step(self.msgs[code], tables, self.plan, self.s, code, self.x,
+                                                   ETA, self.status)
+            else:
+                self.Q.qsgd_decode_sgd_step(self.msgs[code], tables, self.n, self.d, self.s, code, self.x,
+                                            ETA, self.status)
 
     def message_bytes(self, code):
         if code == 0:
-            return float(fixed_bytes(self.n, self.d, self.s))
+            return float(self.prefix + fixed_bytes(self.nq, self.d, self.s))
         info = self.info[code]
         return float(np.mean(info[:, 2].astype(np.float64)))
 
     def payload_bits_per_coord(self, code):
         if code == 0:
-            return 8.0 * fixed_bytes(self.n, self.d, self.s) / self.n
+            return 8.0 * (self.prefix + fixed_bytes(self.nq, self.d, self.s)) / self.n
         return float(np.mean(self.info[code][:, 0].astype(np.float64))) / self.n
 
 
 def kernel_algorithmic_bytes(hp, code_name):
     """Bytes each kernel must move per launch (the method's own inputs and outputs)."""
-    n, d, s, K, B = hp.n, hp.d, hp.s, hp.K, hp.B
-    MF = fixed_bytes(n, d, s)
-    out = {"quantize_fixed": 4 * n + MF, "decode_fixed": K * MF + 8 * n, "sgd_step": 12 * n}
+    d, s, K, B = hp.d, hp.s, hp.K, hp.B
+    n = hp.n - hp.n_raw                       # coordinates that are quantized (all of them without a policy)
+    MF = fixed_bytes(hp.nq, d, s)
+    out = {"quantize_fixed": 4 * n + MF, "decode_fixed": K * MF + 8 * n, "sgd_step": 12 * n,
+           "raw_gather": 8 * hp.n_raw, "raw_decode": (4 * K + 8) * hp.n_raw}
     if 1 in hp.info:
         info = hp.info[1]
-        msg = float(np.mean(info[:, 2].astype(np.float64)))
-        pay = float(np.mean(info[:, 1].astype(np.float64)))
+        msg = float(np.mean(info[:, 2].astype(np.float64))) - hp.prefix
+        pay = float(np.mean(info[:, 1].astype(np.float64))) - hp.prefix
         out.update({"decode_elias": K * msg + 8 * n, "decode_elias_sparse": K * msg + 8 * n,
                     "elias_scatter": MF + pay + 8 * (B + 1),
                     "elias_length": MF - 4 * ((n + 31) // 32) + 4 * B})
@@ -597,8 +629,13 @@ def run_oracle_sample(wl, steps=1, workers=2):
     full n (capped at 2^25 coordinates), every code kind of the workload: encode each, then
     decode + aggregate + SGD step."""
     from oracle import oracle as O
-    n = min(wl["n"], 2 ** 25)
-    n -= n % wl["d"] if n > wl["d"] else 0
+    plan = None
+    if wl.get("policy"):                              # the policy needs the whole tensor list
+        n = wl["n"]
+        plan = O.policy_plan(policy_sizes(wl["policy"]), wl["d"])
+    else:
+        n = min(wl["n"], 2 ** 25)
+        n -= n % wl["d"] if n > wl["d"] else 0
     d, s, norm = wl["d"], wl["s"], NORM[wl["norm"]]
     gs = [host_gradient(wl, w, n) for w in range(workers)]
     x = np.zeros(n, dtype=np.float32)
@@ -607,12 +644,19 @@ def run_oracle_sample(wl, steps=1, workers=2):
         for code_name in wl["codes"]:
             code = CODE[code_name]
             t0 = time.perf_counter()
-            msgs, tabs = [], []
+            msgs, tabs, infos = [], [], []
             for w, g in enumerate(gs):
-                m, info = O.encode(g, d, s, norm, code, PHILOX_SEED, it, w)
+                if plan is not None:
+                    m, info = O.policy_encode(g, plan, s, norm, code, PHILOX_SEED, it, w)
+                else:
+                    m, info = O.encode(g, d, s, norm, code, PHILOX_SEED, it, w)
+                    tabs.append(None if code == 0 else O.message_table(m, info, n, d))
                 msgs.append(m)
-                tabs.append(None if code == 0 else O.message_table(m, info, n, d))
-            st, acc = O.decode_accumulate(msgs, None if code == 0 else tabs, n, d, s, code)
+                infos.append(info)
+            if plan is not None:
+                st, acc = O.policy_decode_accumulate(msgs, infos, plan, s, code)
+            else:
+                st, acc = O.decode_accumulate(msgs, None if code == 0 else tabs, n, d, s, code)
             x = O.sgd_step(x, acc, ETA, workers)
             t_total += time.perf_counter() - t0
             bytes_total += 2 * workers * 4 * n

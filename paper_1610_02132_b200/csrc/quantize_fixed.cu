@@ -181,39 +181,61 @@ struct FastParams {
   QuantizeParams tail;      // parameters of the extra CTA (used when gridDim.x > main_ctas)
 };
 
-template <int LB, int NORM>
+template <int LB, int NORM, bool MAPPED>
 __device__ __forceinline__ void quantize_generic_tile(const QuantizeParams& p, uint32_t block, uint32_t nblocks,
                                                       float* tile, float* part, float* s_rcp);
 
-// Producer side of one stage: start the bulk copies of tile t. Ordinary case: one copy of the whole
-// tile. With a bucket map every bucket of the tile is copied from its own place; a bucket that is
-// shorter than d gets zeros behind its values (plain stores, ordered before the copies' arrival by
-// the release of the expect-tx arrive). The map guarantees 16-byte aligned places and lengths.
-__device__ __forceinline__ void issue_tile(const FastParams& p, float* tile, uint64_t* full_bar, uint32_t t) {
-  if (!p.map.src) {
-    mbar_expect_tx(full_bar, kTile * 4);
-    bulk_load(tile, p.g + (size_t)t * kTile, kTile * 4, full_bar);
+// Producer side of one stage, called by all lanes of warp 0: start the bulk copies of tile t.
+// Ordinary case: lane 0 starts one copy of the whole tile. With a bucket map, lane j looks up
+// bucket j of the tile (at most 16 buckets: d >= 256); when the buckets are complete and follow one
+// another in memory (the rule inside a tensor) it is again one copy, otherwise every lane copies its
+// own bucket and puts zeros behind a short one (plain stores, made visible to the consumers by the
+// warp barrier before lane 0's expect-tx arrive, which releases). The map guarantees 16-byte aligned
+// places and lengths.
+template <bool MAPPED>
+__device__ __forceinline__ void issue_tile(const FastParams& p, float* tile, uint64_t* full_bar, uint32_t t,
+                                           uint32_t lane) {
+  if (!MAPPED) {
+    if (lane == 0) {
+      mbar_expect_tx(full_bar, kTile * 4);
+      bulk_load(tile, p.g + (size_t)t * kTile, kTile * 4, full_bar);
+    }
     return;
   }
   const uint32_t d = 1u << p.log2d, nb = kTile >> p.log2d;
   const uint64_t b0 = (uint64_t)t << (12u - p.log2d);
-  uint32_t bytes = 0;
-  for (uint32_t j = 0; j < nb; ++j) {
-    const uint32_t L = min(__ldg(p.map.len + b0 + j), d);
-    for (uint32_t c = L; c < d; c += 4) *reinterpret_cast<float4*>(tile + j * d + c) = make_float4(0.f, 0.f, 0.f, 0.f);
-    bytes += 4u * L;
+  uint32_t L = 0;
+  uint64_t src = 0;
+  if (lane < nb) {
+    L = min(__ldg(p.map.len + b0 + lane), d);
+    src = __ldg(p.map.src + b0 + lane);
   }
-  mbar_expect_tx(full_bar, bytes);
-  for (uint32_t j = 0; j < nb; ++j) {
-    const uint32_t L = min(__ldg(p.map.len + b0 + j), d);
-    if (L) bulk_load(tile + j * d, p.g + __ldg(p.map.src + b0 + j), 4u * L, full_bar);
+  const uint64_t src0 = __shfl_sync(0xffffffffu, src, 0);
+  const bool in_line = lane >= nb || (L == d && src == src0 + (uint64_t)lane * d);
+  if (__all_sync(0xffffffffu, in_line)) {
+    if (lane == 0) {
+      mbar_expect_tx(full_bar, kTile * 4);
+      bulk_load(tile, p.g + src0, kTile * 4, full_bar);
+    }
+    return;
   }
+  if (lane < nb)
+    for (uint32_t c = L; c < d; c += 4) *reinterpret_cast<float4*>(tile + lane * d + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+  uint32_t bytes = lane < nb ? 4u * L : 0u;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) bytes += __shfl_xor_sync(0xffffffffu, bytes, o);
+  __syncwarp();
+  if (lane == 0) mbar_expect_tx(full_bar, bytes);
+  __syncwarp();
+  if (lane < nb && L) bulk_load(tile + lane * d, p.g + src, 4u * L, full_bar);
 }
 
 // CROSS: a bucket spans several warps (d >= 1024); otherwise a bucket is d / 16 <= 32 lanes.
 // CTAs 0 .. main_ctas - 1 stream the complete tiles; one optional extra CTA runs the ragged last
 // tile and the region padding through the generic tile code (its operands alias the tile ring).
-template <int LB, int NORM, bool CROSS>
+// MAPPED: buckets are fetched through a bucket map (per-tensor policy); a separate instantiation, so
+// that the ordinary kernel carries none of that code.
+template <int LB, int NORM, bool CROSS, bool MAPPED>
 __global__ void __launch_bounds__(kThreads, 4)
 quantize_pow2_kernel(const __grid_constant__ FastParams p) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -222,7 +244,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t grid = p.main_ctas;
   if (blockIdx.x >= grid) {                     // the extra CTA: ragged tail + padding
-    quantize_generic_tile<LB, NORM>(p.tail, 0u, 1u, sm.tile[0], sm.tile[1], sm.tile[1] + 1024);
+    quantize_generic_tile<LB, NORM, MAPPED>(p.tail, 0u, 1u, sm.tile[0], sm.tile[1], sm.tile[1] + 1024);
     return;
   }
   if (tid == 0) {
@@ -233,14 +255,14 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  if (tid == 0) {
-    if (blockIdx.x == 0 && p.info) {
+  if (MAPPED ? warp == 0 : tid == 0) {
+    if (tid == 0 && blockIdx.x == 0 && p.info) {
       p.info[0] = 8 * p.total_bytes; p.info[1] = 0; p.info[2] = p.total_bytes; p.info[3] = 0;
     }
-    if (blockIdx.x == 0 && p.clear_word) *p.clear_word = 0u;
+    if (tid == 0 && blockIdx.x == 0 && p.clear_word) *p.clear_word = 0u;
     for (int s = 0; s < kStages; ++s) {
       const uint32_t t = blockIdx.x + (uint32_t)s * grid;
-      if (t < p.full_tiles) issue_tile(p, sm.tile[s], &sm.full[s], t);
+      if (t < p.full_tiles) issue_tile<MAPPED>(p, sm.tile[s], &sm.full[s], t, lane);
     }
   }
 
@@ -288,20 +310,30 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
     if (lane == 0) mbar_arrive(&sm.empty[stage]);
     int flags = arrived ? 0 : 1;
     if (CROSS) flags = __syncthreads_or(flags | (shaky ? 2 : 0));
+    else if (MAPPED) flags = __any_sync(0xffffffffu, flags != 0) ? 1 : 0;      // the producer warp must leave together
     if (flags & 1) {
       atomicOr(p.status, QSGD_DEV_TIMEOUT);
       break;
     }
-    if (tid == 0 && it > 0) {
-      const uint32_t ps = stage == 0 ? kStages - 1 : stage - 1;           // stage of iteration it - 1
-      const uint32_t pphase = stage == 0 ? phase ^ 1 : phase;
-      const uint32_t tn = t + (uint32_t)(kStages - 1) * grid;             // tile of iteration it - 1 + kStages
-      if (tn < p.full_tiles) {
-        if (mbar_wait_bounded(&sm.empty[ps], pphase)) {
-          issue_tile(p, sm.tile[ps], &sm.full[ps], tn);
-        } else {
-          atomicOr(p.status, QSGD_DEV_TIMEOUT);
+    if (!MAPPED) {                                                        // ordinary case: thread 0 produces
+      if (tid == 0 && it > 0) {
+        const uint32_t ps = stage == 0 ? kStages - 1 : stage - 1;         // stage of iteration it - 1
+        const uint32_t pphase = stage == 0 ? phase ^ 1 : phase;
+        const uint32_t tn = t + (uint32_t)(kStages - 1) * grid;           // tile of iteration it - 1 + kStages
+        if (tn < p.full_tiles) {
+          if (mbar_wait_bounded(&sm.empty[ps], pphase)) issue_tile<false>(p, sm.tile[ps], &sm.full[ps], tn, 0u);
+          else atomicOr(p.status, QSGD_DEV_TIMEOUT);
         }
+      }
+    } else if (warp == 0 && it > 0) {                                     // bucket map: warp 0 produces
+      const uint32_t ps = stage == 0 ? kStages - 1 : stage - 1;
+      const uint32_t pphase = stage == 0 ? phase ^ 1 : phase;
+      const uint32_t tn = t + (uint32_t)(kStages - 1) * grid;
+      if (tn < p.full_tiles) {
+        const bool freed = __shfl_sync(0xffffffffu, lane == 0 ? (mbar_wait_bounded(&sm.empty[ps], pphase) ? 1 : 0) : 0, 0) != 0;
+        __syncwarp();                                                     // lane 0's acquire covers the warp
+        if (freed) issue_tile<true>(p, sm.tile[ps], &sm.full[ps], tn, lane);
+        else if (lane == 0) atomicOr(p.status, QSGD_DEV_TIMEOUT);
       }
     }
     float A;
@@ -420,7 +452,7 @@ constexpr int kMaxBucketsPerTile = kTile / 32;          // 128
 
 // One tile of the generic path. `block` / `nblocks` play the role of blockIdx / gridDim so that the
 // main kernel can run the ragged last tile in one extra CTA of its own grid.
-template <int LB, int NORM>
+template <int LB, int NORM, bool MAPPED>
 __device__ __forceinline__ void quantize_generic_tile(const QuantizeParams& p, uint32_t block, uint32_t nblocks,
                                                       float* tile, float* part, float* s_rcp) {
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -442,7 +474,7 @@ __device__ __forceinline__ void quantize_generic_tile(const QuantizeParams& p, u
 
   for (uint32_t i = tid * 4; i < p.tile_coords; i += kThreads * 4) {
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (p.map.src) {
+    if (MAPPED) {
       // per-tensor policy: four coordinates of one bucket (d is a multiple of 32) from the
       // bucket's own place; what lies behind the bucket's length is zero padding
       if (i < valid) {
@@ -596,12 +628,12 @@ __device__ __forceinline__ void quantize_generic_tile(const QuantizeParams& p, u
   }
 }
 
-template <int LB, int NORM>
+template <int LB, int NORM, bool MAPPED>
 __global__ void __launch_bounds__(kThreads) quantize_generic_kernel(const QuantizeParams p) {
   __shared__ __align__(16) float tile[kTile];
   __shared__ float part[kTile / 8];
   __shared__ float s_rcp[kMaxBucketsPerTile];
-  quantize_generic_tile<LB, NORM>(p, blockIdx.x, gridDim.x, tile, part, s_rcp);
+  quantize_generic_tile<LB, NORM, MAPPED>(p, blockIdx.x, gridDim.x, tile, part, s_rcp);
 }
 
 PhiloxConsts make_philox_consts(uint64_t seed, uint32_t step, uint32_t worker) {
@@ -621,10 +653,10 @@ PhiloxConsts make_philox_consts(uint64_t seed, uint32_t step, uint32_t worker) {
   return pc;
 }
 
-template <int LB, int NORM, bool CROSS>
+template <int LB, int NORM, bool CROSS, bool MAPPED>
 int launch_fast(FastParams& fp, bool with_tail, cudaStream_t stream) {
   static int ctas_per_sm = 0, sms = 0;
-  auto kern = quantize_pow2_kernel<LB, NORM, CROSS>;
+  auto kern = quantize_pow2_kernel<LB, NORM, CROSS, MAPPED>;
   const size_t smem = sizeof(TileSmem) + 128;
   if (ctas_per_sm == 0) {
     int dev = 0;
@@ -670,8 +702,10 @@ int launch_one(QuantizeParams& p, uint64_t seed, cudaStream_t stream) {
     fp.tail = p;
     fp.tail.info = nullptr;
     fp.tail.clear_word = nullptr;
-    return d >= 1024 ? launch_fast<LB, NORM, true>(fp, with_tail, stream)
-                     : launch_fast<LB, NORM, false>(fp, with_tail, stream);
+    if (fp.map.src) return d >= 1024 ? launch_fast<LB, NORM, true, true>(fp, with_tail, stream)
+                                     : launch_fast<LB, NORM, false, true>(fp, with_tail, stream);
+    return d >= 1024 ? launch_fast<LB, NORM, true, false>(fp, with_tail, stream)
+                     : launch_fast<LB, NORM, false, false>(fp, with_tail, stream);
   }
   // the fast path does not apply: everything through the generic kernel
   p.coord_base = 0;
@@ -680,7 +714,8 @@ int launch_one(QuantizeParams& p, uint64_t seed, cudaStream_t stream) {
   if (tiles == 0) tiles = 1;
   {
     ScopedKernel sk(kKernQuantizeTail, stream);
-    quantize_generic_kernel<LB, NORM><<<(uint32_t)tiles, kThreads, 0, stream>>>(p);
+    if (p.map.src) quantize_generic_kernel<LB, NORM, true><<<(uint32_t)tiles, kThreads, 0, stream>>>(p);
+    else quantize_generic_kernel<LB, NORM, false><<<(uint32_t)tiles, kThreads, 0, stream>>>(p);
   }
   return (int)cudaGetLastError();
 }
