@@ -919,7 +919,7 @@ int launch_fields(FieldParams& p, bool fused, cudaStream_t stream, bool* handled
 }
 
 // ------------------------------------------------------------------------------------------------
-// Field-rebuilding decoder for long buckets (d >= 2048): the same two phases, but a bucket is
+// Field-rebuilding decoder for long buckets (d >= 1024): the same two phases, but a bucket is
 // walked in ranges of 512 positions. A lane keeps its place in its string between ranges (bit
 // window, position, one decoded entry that lies past the range), so shared memory holds the fields
 // of one range only and as many warps fit on an SM as for d = 512; with whole-bucket fields a CTA
@@ -1098,7 +1098,7 @@ int launch_ranged(FieldParams& p, bool fused, cudaStream_t stream, bool* handled
 
 template <int LB>
 int launch_fields_lb(FieldParams& p, bool dense, bool fused, cudaStream_t stream, bool* handled) {
-  if (p.d >= 2048u && p.K <= 32u)       // long buckets: fields of one range at a time
+  if (p.d >= 1024u && p.K <= 32u)       // long buckets: fields of one range at a time
     return dense ? launch_ranged<LB, true>(p, fused, stream, handled) : launch_ranged<LB, false>(p, fused, stream, handled);
   return dense ? launch_fields<LB, true>(p, fused, stream, handled) : launch_fields<LB, false>(p, fused, stream, handled);
 }
