@@ -780,7 +780,7 @@ int launch_sparse(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint
 }
 
 template <int LB, bool DENSE, bool FUSED, bool SINGLE>
-__global__ void __launch_bounds__(128) decode_elias_fields_kernel(const __grid_constant__ FieldParams p) {
+__global__ void __launch_bounds__(320) decode_elias_fields_kernel(const __grid_constant__ FieldParams p) {
   extern __shared__ __align__(16) uint32_t fsm[];
   __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
   __shared__ uint16_t elias_lut[1u << kLutBits];
@@ -892,9 +892,17 @@ int launch_fields(FieldParams& p, bool fused, cudaStream_t stream, bool* handled
   p.G = G;
   const size_t per_warp = (size_t)G * p.bucket_words * 4;
   const size_t budget = (size_t)max_smem - (LB == 8 ? 32768 : 128) - 8192 - 1024;
-  int warps = 4;
-  while (warps > 1 && (size_t)warps * per_warp > (warps == 4 ? (96u << 10) : budget)) warps >>= 1;
-  if ((size_t)warps * per_warp > budget) return 0;               // caller falls back to the slow kernel
+  // Warps per CTA: the count that leaves the most warps resident on an SM. The code table and the
+  // level table are per CTA, the fields per warp; the parse is latency-bound, so warps are what counts.
+  const size_t per_cta = (LB == 8 ? 32768 : 128) + 8192 + 1024;
+  const size_t per_sm = 227u << 10;
+  int warps = 0, best = 0;
+  for (int w = 1; w <= 10; ++w) {
+    if ((size_t)w * per_warp > budget) break;
+    const int resident = (int)(per_sm / ((size_t)w * per_warp + per_cta)) * w;
+    if (resident > best) { best = resident; warps = w; }
+  }
+  if (warps == 0) return 0;                                      // caller falls back to the slow kernel
   const bool single = p.d >= 512 && (p.d & (p.d - 1)) == 0 && LB != 8;
   void (*kern)(FieldParams);
   if (fused) kern = single ? decode_elias_fields_kernel<LB, DENSE, true, true> : decode_elias_fields_kernel<LB, DENSE, true, false>;
