@@ -503,14 +503,13 @@ template <typename F>
 __device__ __forceinline__ uint32_t advance(LaneParse& st, uint32_t rend, uint32_t limit, uint32_t db, uint32_t s,
                                             F&& sink) {
   uint32_t n = 0;
-  for (;;) {
-    if (st.pend != kNoEntry) {
-      if ((st.pend & 0xFFFFu) >= rend || n >= limit) break;
-      sink(n, st.pend);
-      ++n;
-      st.pend = kNoEntry;
-    }
-    if (st.used >= st.total || st.err != 0u) break;
+  if (st.pend != kNoEntry) {                          // the entry that an earlier call had to hold back
+    if ((st.pend & 0xFFFFu) >= rend || limit == 0u) return 0u;
+    sink(0u, st.pend);
+    n = 1;
+    st.pend = kNoEntry;
+  }
+  while (st.used < st.total && st.err == 0u) {
     uint32_t gap, level, len;
     st.src.refill();                                  // >= 33 valid bits: a code takes at most 23
     bool ok = elias_from_window(st.src.hi, gap, len);
@@ -532,9 +531,15 @@ __device__ __forceinline__ uint32_t advance(LaneParse& st, uint32_t rend, uint32
       st.err |= st.at >= db ? QSGD_DEV_POSITION : 0u;
       st.err |= level > s ? QSGD_DEV_LEVEL : 0u;
       st.err |= st.used > st.total ? QSGD_DEV_OVERRUN : 0u;
-    } else {
-      st.pend = st.at | (level << 16) | (neg << 31);
+      break;
     }
+    const uint32_t en = st.at | (level << 16) | (neg << 31);
+    if (st.at >= rend || n >= limit) {                // past the range, or no room: keep it for the next call
+      st.pend = en;
+      break;
+    }
+    sink(n, en);
+    ++n;
   }
   return n;
 }
@@ -758,7 +763,18 @@ int launch_sparse(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint
   if ((tile_quads & (tile_quads - 1)) == 0)
     for (p.quad_shift = 0; (1u << p.quad_shift) < tile_quads; ++p.quad_shift) {}
   const size_t per_warp = (size_t)p.warp_words * 4;              // at most 16.3 KB
-  const int warps = 8 * per_warp <= (100u << 10) ? 8 : 4;
+  // Warps per CTA: on a problem of about one wave, the count that spreads the warps most evenly
+  // over the SMs (the busiest SM sets the time); 8, or 4 when 8 do not fit, otherwise.
+  const uint64_t all_groups = (p.B + p.sh.G - 1) / p.sh.G;
+  int warps = 8 * per_warp <= (100u << 10) ? 8 : 4;
+  if (all_groups <= (uint64_t)sms * 32u) {
+    uint64_t best = ~0ull;
+    for (int w = warps; w >= 4; --w) {
+      const uint64_t ctas = (all_groups + w - 1) / w;
+      const uint64_t busiest = (ctas + sms - 1) / sms * w;      // warps on the fullest SM
+      if (busiest < best) { best = busiest; warps = w; }
+    }
+  }
   auto kern = fused ? decode_elias_sparse_kernel<true> : decode_elias_sparse_kernel<false>;
   const size_t smem = (size_t)warps * per_warp;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
