@@ -11,18 +11,33 @@ from paper_1610_02132_b200 import inputs as I
 
 pytestmark = pytest.mark.gpu
 
-N, D, S = 4096 + 300, 512, 3
+# (n, d, s, input): one shape per Elias decoder -- whole-bucket fields (d < 1024), fields by ranges
+# (d >= 1024), and the entry-list decoder of the sparse regime (short strings)
+SHAPES = [(4096 + 300, 512, 3, "gauss"), (2 * 4096 + 300, 4096, 3, "gauss"), (3 * 4096 + 300, 4096, 1, "sparse")]
 
 
-def good_message(code_kind=O.CODE_ELIAS, seed=5):
-    g = I.gaussian(N, 1.0, seed=seed)
-    m, info = O.encode(g, D, S, O.NORM_L2, code_kind, 7, 0, 0)
+@pytest.fixture(params=SHAPES, ids=["fields", "ranged", "sparse"])
+def shape(request):
+    return request.param
+
+
+def gradient(shape, seed):
+    n, _, _, kind = shape
+    return I.gaussian(n, 1.0, seed=seed) if kind == "gauss" else I.sparse_laplace(n, 1e-3, 0.3, seed=seed)
+
+
+def good_message(shape, code_kind=O.CODE_ELIAS, seed=5):
+    _, d, s, _ = shape
+    m, info = O.encode(gradient(shape, seed), d, s, O.NORM_L2, code_kind, 7, 0, 0)
     return m, info
 
 
-def run_decode(msg_np, info, code_kind=O.CODE_ELIAS, table_np=None, s=S, n=N):
+def run_decode(shape, msg_np, info, code_kind=O.CODE_ELIAS, table_np=None, s=None, n=None):
     """Decode one (possibly corrupted) message on the GPU; returns (status, acc, guard ok)."""
-    B = O.n_buckets(n, D)
+    d = shape[1]
+    s = shape[2] if s is None else s
+    n = shape[0] if n is None else n
+    B = O.n_buckets(n, d)
     buf = torch.from_numpy(np.concatenate([msg_np, np.zeros(64, np.uint8)])).cuda()
     if table_np is None:
         table = buf[info[1]: info[1] + 8 * (B + 1)].view(torch.int64)
@@ -30,69 +45,85 @@ def run_decode(msg_np, info, code_kind=O.CODE_ELIAS, table_np=None, s=S, n=N):
         table = torch.from_numpy(table_np.view(np.int64)).cuda()
     acc = torch.full((n + 256,), 7.0, dtype=torch.float32, device="cuda")
     status = Q.new_status()
-    Q.qsgd_decode_accumulate([buf], [table], n, D, s, code_kind, acc[:n], status)
+    Q.qsgd_decode_accumulate([buf], [table], n, d, s, code_kind, acc[:n], status)
+    x = torch.full((n + 256,), 3.0, dtype=torch.float32, device="cuda")
+    status2 = Q.new_status()
+    Q.qsgd_decode_sgd_step([buf], [table], n, d, s, code_kind, x[:n], 0.5, status2)
     torch.cuda.synchronize()
-    return int(status.item()), acc[:n].cpu().numpy(), bool((acc[n:] == 7.0).all())
+    guard = bool((acc[n:] == 7.0).all()) and bool((x[n:] == 3.0).all())
+    assert (int(status.item()) != 0) == (int(status2.item()) != 0)
+    return int(status.item()) | int(status2.item()), acc[:n].cpu().numpy(), guard
 
 
-def test_well_formed_stream_has_clean_status():
-    m, info = good_message()
-    st, acc, guard = run_decode(m, info)
-    ref = O.decode(m, O.message_table(m, info, N, D), N, D, S, O.CODE_ELIAS)[1]
+def test_well_formed_stream_has_clean_status(shape):
+    n, d, s, _ = shape
+    m, info = good_message(shape)
+    st, acc, guard = run_decode(shape, m, info)
+    ref = O.decode(m, O.message_table(m, info, n, d), n, d, s, O.CODE_ELIAS)[1]
     assert st == 0 and guard and np.array_equal(acc.view(np.uint32), ref.view(np.uint32))
 
 
-def test_truncated_bucket_is_flagged():
-    m, info = good_message()
-    t = O.message_table(m, info, N, D).copy()
-    t[3] -= 5                                    # bucket 2 loses its last 5 bits (bucket 3 starts early)
-    st, _, guard = run_decode(m, info, table_np=t)
+def test_truncated_bucket_is_flagged(shape):
+    n, d, s, _ = shape
+    m, info = good_message(shape)
+    t = O.message_table(m, info, n, d).copy()
+    t[2] -= 5                                    # bucket 1 loses its last 5 bits (bucket 2 starts early)
+    st, _, guard = run_decode(shape, m, info, table_np=t)
     assert st != 0 and guard
-    assert O.elias_unpack(m[: info[1]], t, N, D, S)[0] != 0        # the oracle rejects it too
+    assert O.elias_unpack(m[: info[1]], t, n, d, s)[0] != 0        # the oracle rejects it too
 
 
-def test_offsets_not_ascending_and_short_bucket():
-    m, info = good_message()
-    t = O.message_table(m, info, N, D).copy()
-    t[2], t[3] = t[3], t[2]
-    st, _, guard = run_decode(m, info, table_np=t)
+def test_offsets_not_ascending_and_short_bucket(shape):
+    n, d, s, _ = shape
+    m, info = good_message(shape)
+    t = O.message_table(m, info, n, d).copy()
+    t[1], t[2] = t[2], t[1]
+    st, _, guard = run_decode(shape, m, info, table_np=t)
     assert st & Q.binding.DEV_TABLE and guard
-    t = O.message_table(m, info, N, D).copy()
+    t = O.message_table(m, info, n, d).copy()
     t[1] = t[0] + 8                              # shorter than the 32-bit scale
-    st, _, guard = run_decode(m, info, table_np=t)
+    st, _, guard = run_decode(shape, m, info, table_np=t)
     assert st != 0 and guard
 
 
-def test_level_above_s_is_flagged():
-    g = I.gaussian(N, 1.0, seed=6)
-    m, info = O.encode(g, D, 15, O.NORM_MAX, O.CODE_ELIAS, 7, 0, 0)      # levels up to 15
-    st, _, guard = run_decode(m, info, s=3)                                # decoder told s = 3
+def test_level_above_s_is_flagged(shape):
+    n, d, s, _ = shape
+    s_sent = 15 if s == 3 else 3
+    g = gradient(shape, 6)
+    norm = O.NORM_MAX
+    if shape[3] == "sparse":                      # keep the strings short: one dominant coordinate gets level 3
+        g[100] = 1.0
+        norm = O.NORM_L2
+    m, info = O.encode(g, d, s_sent, norm, O.CODE_ELIAS, 7, 0, 0)         # levels above s occur
+    assert O.elias_unpack(m[: info[1]], O.message_table(m, info, n, d), n, d, s)[0] != 0
+    st, _, guard = run_decode(shape, m, info)                              # decoder told the smaller s
     assert st & Q.binding.DEV_LEVEL and guard
 
 
-def test_gap_past_the_bucket_is_flagged():
+def test_gap_past_the_bucket_is_flagged(shape):
     # a stream encoded for n coordinates decoded as if the vector ended earlier: the last
     # bucket's positions overshoot the (shorter) tail bucket
-    n_short = 4096 + 40
-    g = I.gaussian(N, 1.0, seed=7)
-    g[4096 + 250] = 50.0                          # certainly a nonzero beyond position 40
-    m, info = O.encode(g, D, S, O.NORM_L2, O.CODE_ELIAS, 7, 0, 0)
-    st, _, guard = run_decode(m, info, n=n_short)
+    n, d, s, _ = shape
+    base = n // d * d
+    g = gradient(shape, 7)
+    g[base + 250] = 50.0                          # certainly a nonzero beyond position 40
+    m, info = O.encode(g, d, s, O.NORM_L2, O.CODE_ELIAS, 7, 0, 0)
+    st, _, guard = run_decode(shape, m, info, n=base + 40)
     assert st & (Q.binding.DEV_POSITION | Q.binding.DEV_OVERRUN) and guard
 
 
-def test_random_garbage_payload_terminates():
-    m, info = good_message()
+def test_random_garbage_payload_terminates(shape):
+    m, info = good_message(shape)
     r = np.random.default_rng(1)
     bad = m.copy()
     bad[: info[1]] = r.integers(0, 256, info[1], dtype=np.uint8)          # table intact, payload noise
-    st, _, guard = run_decode(bad, info)
+    st, _, guard = run_decode(shape, bad, info)
     assert st != 0 and guard
     for kind in (O.CODE_ELIAS_DENSE,):
-        m2, info2 = good_message(kind)
+        m2, info2 = good_message(shape, kind)
         bad = m2.copy()
         bad[: info2[1]] = r.integers(0, 256, info2[1], dtype=np.uint8)
-        st, _, guard = run_decode(bad, info2, code_kind=kind)
+        st, _, guard = run_decode(shape, bad, info2, code_kind=kind)
         assert st != 0 and guard
 
 
