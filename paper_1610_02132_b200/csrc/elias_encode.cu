@@ -189,10 +189,89 @@ struct LaneSummary {
   int32_t last;       // last nonzero position, -1 if none
 };
 
+// Sum over the nonzero fields of one level word of 1 + |Elias(level)| (sign bit and level code),
+// without a loop: |Elias(level)| grows by 1, 2, 3, 1, 4, 1, 1, 1 when the level reaches 1, 2, 4, 8,
+// 16, 32, 64, 128 (Appendix A.2 lengths 1, 3, 6, 7, 11, 12, 13, 14), so the per-field sum is a weighted
+// count of "level >= 2^j" masks, added up across the fields of the word.
+template <int LB>
+__device__ __forceinline__ uint32_t level_code_bits(uint32_t w) {
+  if (LB == 1) return 2u * (uint32_t)__popc(w);
+  if (LB == 2) {
+    const uint32_t b1 = (w >> 1) & 0x55555555u;
+    return 2u * (uint32_t)(__popc(b1 | (w & 0x55555555u)) + __popc(b1));
+  }
+  if (LB == 4) {
+    const uint32_t t3 = w >> 3;
+    const uint32_t ge8 = t3 & 0x11111111u;
+    const uint32_t ge4 = (t3 | (w >> 2)) & 0x11111111u;
+    const uint32_t ge2 = (ge4 | (w >> 1)) & 0x11111111u;
+    const uint32_t ge1 = (ge2 | w) & 0x11111111u;
+    const uint32_t x = ge8 + 3u * ge4 + 2u * (ge1 + ge2);              // at most 8 per nibble
+    const uint32_t y = (x & 0x0F0F0F0Fu) + ((x >> 4) & 0x0F0F0F0Fu);
+    return (y * 0x01010101u) >> 24;
+  }
+  const uint32_t ge128 = (w >> 7) & 0x01010101u;
+  const uint32_t ge64 = (ge128 | (w >> 6)) & 0x01010101u;
+  const uint32_t ge32 = (ge64 | (w >> 5)) & 0x01010101u;
+  const uint32_t ge16 = (ge32 | (w >> 4)) & 0x01010101u;
+  const uint32_t ge8 = (ge16 | (w >> 3)) & 0x01010101u;
+  const uint32_t ge4 = (ge8 | (w >> 2)) & 0x01010101u;
+  const uint32_t ge2 = (ge4 | (w >> 1)) & 0x01010101u;
+  const uint32_t ge1 = (ge2 | w) & 0x01010101u;
+  const uint32_t x = 2u * (ge1 + ge2) + 3u * ge4 + ge8 + 4u * ge16 + ge32 + ge64 + ge128;   // at most 15 per byte
+  return (x * 0x01010101u) >> 24;
+}
+
+// Sum of |Elias(gap)| over the set bits of a 64-coordinate block except the lowest, gap = distance to
+// the previous set bit, without a loop: P = "some set bit lies 1 .. 2^b - 1 positions below" is built
+// by doubling, and the set bits whose gap has bit length b are those in P_b but not in P_(b-1).
+__device__ __forceinline__ uint32_t gap_code_bits(unsigned long long m) {
+  unsigned long long prev = 0ull, P = m << 1;
+  uint32_t bits = (uint32_t)__popcll(m & P);                            // gap 1: code "0"
+  prev = P; P = P | (m << 2) | (P << 2);
+  bits += 3u * (uint32_t)__popcll(m & P & ~prev);                       // gaps 2 .. 3
+  prev = P; P = P | (m << 4) | (P << 4);
+  bits += 6u * (uint32_t)__popcll(m & P & ~prev);                       // gaps 4 .. 7
+  prev = P; P = P | (m << 8) | (P << 8);
+  bits += 7u * (uint32_t)__popcll(m & P & ~prev);                       // gaps 8 .. 15
+  prev = P; P = P | (m << 16) | (P << 16);
+  bits += 11u * (uint32_t)__popcll(m & P & ~prev);                      // gaps 16 .. 31
+  prev = P; P = P | (m << 32) | (P << 32);
+  bits += 12u * (uint32_t)__popcll(m & P & ~prev);                      // gaps 32 .. 63
+  return bits;
+}
+
+// whole_blocks: the lanes' ranges are multiples of 64 coordinates, so every level word this lane
+// reads holds only its own coordinates (or, in the last bucket, coordinates past the end of the vector).
 template <int LB>
 __device__ __forceinline__ LaneSummary summarize_sparse(const uint32_t* tab, const uint32_t* __restrict__ lwb,
-                                                        uint32_t c_lo, uint32_t c_hi) {
+                                                        uint32_t c_lo, uint32_t c_hi, bool whole_blocks) {
   LaneSummary s{0u, -1, -1};
+  if (whole_blocks) {
+    // Blocks of 64 coordinates, no loop over the nonzeros: code lengths come from counting. Fields
+    // past the end of the vector are zero in the fixed-width layout, so a ragged c_hi needs no mask
+    // beyond not reading words that start past it.
+    constexpr uint32_t kFields = 32u / LB;
+    for (uint32_t c0 = c_lo; c0 < c_hi; c0 += 64u) {
+      const uint32_t* wp = lwb + ((c0 * LB) >> 5);
+      unsigned long long m = 0ull;
+      uint32_t bits = 0;
+#pragma unroll
+      for (uint32_t j = 0; j < 2u * LB; ++j) {
+        const uint32_t w = (c0 + j * kFields < c_hi) ? __ldg(wp + j) : 0u;
+        m |= (unsigned long long)nonzero_mask<LB>(w) << (j * kFields);
+        bits += level_code_bits<LB>(w);
+      }
+      if (m) {
+        const int32_t lowest = (int32_t)c0 + __ffsll((long long)m) - 1;
+        if (s.first < 0) s.first = lowest;
+        else bits += tab_len(tab, (uint32_t)(lowest - s.last));          // gap across two blocks of this lane
+        s.last = (int32_t)c0 + 63 - __clzll((long long)m);
+        s.bits += bits + gap_code_bits(m);
+      }
+    }
+    return s;
+  }
   for_each_nonzero<LB>(lwb, c_lo, c_hi, [&](uint32_t pos, uint32_t level) {
     const bool is_first = s.first < 0;
     const uint32_t gap_bits = tab_len(tab, is_first ? 1u : pos - (uint32_t)s.last);
@@ -246,14 +325,14 @@ struct BucketParams {
 template <int LB, bool DENSE>
 __device__ __forceinline__ uint32_t lane_bits(const uint32_t* tab, const uint32_t* __restrict__ lwb, uint32_t lpb,
                                               uint32_t c_lo, uint32_t c_hi, uint32_t tl, bool live,
-                                              int32_t* prev_out) {
+                                              bool whole_blocks, int32_t* prev_out) {
   uint32_t bits = 0;
   int32_t prev = -1;
   if (DENSE) {
     if (live) bits = summarize_dense<LB>(tab, lwb, c_lo, c_hi);
   } else {
     LaneSummary s{0u, -1, -1};
-    if (live) s = summarize_sparse<LB>(tab, lwb, c_lo, c_hi);
+    if (live) s = summarize_sparse<LB>(tab, lwb, c_lo, c_hi, whole_blocks);
     prev = prev_nonzero_before_lane(s.last, tl, lpb);
     bits = s.bits + (s.first >= 0 ? tab_len(tab, (uint32_t)(s.first - prev)) : 0u);
   }
@@ -358,7 +437,7 @@ __global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketPara
   const uint32_t c_lo = min(tl * p.seg, db), c_hi = min(c_lo + p.seg, db);
   const uint32_t* lwb = p.level + ((base * LB) >> 5);            // the bucket's first level word
   int32_t prev;
-  const uint32_t bits = lane_bits<LB, DENSE>(tab, lwb, p.lpb, c_lo, c_hi, tl, live, &prev);
+  const uint32_t bits = lane_bits<LB, DENSE>(tab, lwb, p.lpb, c_lo, c_hi, tl, live, (p.seg & 63u) == 0u, &prev);
   if (live) lane_rec[b * p.lpb + tl] = bits | ((uint32_t)(prev + 1) << 16);   // reused by the scatter
   const uint32_t L = team_sum(bits, p.lpb);
   if (live && tl == 0) len[b] = L;
