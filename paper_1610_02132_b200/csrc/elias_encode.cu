@@ -560,12 +560,17 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
       }
     } else {
       for_each_nonzero<LB>(lwb, c_lo, c_hi, [&](uint32_t pos, uint32_t level) {
-        uint32_t ln;
-        uint32_t code = tab_code(tab, pos - (uint32_t)prev, &ln);
-        bw.put(code, ln);
+        uint32_t gl, ll;
+        const uint32_t gcode = tab_code(tab, pos - (uint32_t)prev, &gl);
         const uint32_t sg = (__ldg(swb + (pos >> 5)) >> (pos & 31)) & 1u;
-        code = tab_code(tab, level, &ln);
-        bw.put((sg << ln) | code, ln + 1);
+        uint32_t lcode = tab_code(tab, level, &ll);
+        lcode |= sg << ll;
+        if (gl + ll + 1u <= 32u) {                     // gap, sign and level in one piece (the rule)
+          bw.put((gcode << (ll + 1u)) | lcode, gl + ll + 1u);
+        } else {
+          bw.put(gcode, gl);
+          bw.put(lcode, ll + 1u);
+        }
         prev = (int32_t)pos;
       });
     }
