@@ -142,3 +142,21 @@ def layered_gaussian_device(shapes, seed=0, base_sigma=1e-2, device="cuda"):
     for lo, hi, sig in layer_sigmas(shapes, base_sigma):
         out[lo:hi].mul_(float(sig))
     return out
+
+
+# ---- finite-sum problem for the variance-reduced variant (Section 3.3) -------------------------------
+def least_squares_problem(m, n, seed=0, noise=0.01):
+    """m unit-norm random rows A[m, n] and targets b = A x_true + noise (fp32). With the ridge term
+    the functions f_j(x) = (a_j . x - b_j)^2 / 2 + lam |x|^2 / 2 are (1 + lam)-smooth and their mean
+    is at least lam-strongly convex, so the condition number is set by lam."""
+    r = _rng(seed)
+    A = r.standard_normal((m, n)).astype(np.float64)
+    A /= np.linalg.norm(A, axis=1, keepdims=True)
+    x_true = r.standard_normal(n)
+    b = A @ x_true + noise * r.standard_normal(m)
+    return A.astype(np.float32), b.astype(np.float32)
+
+
+def sample_indices(P, T, K, m, seed=0):
+    """The uniformly random function indices j[p, t, i] in [0, m) that the K processors draw."""
+    return _rng(seed).integers(0, m, size=(P, T, K), dtype=np.int64)
