@@ -666,6 +666,46 @@ def run_oracle_sample(wl, steps=1, workers=2):
                 workers, wl["K"], n, wl["n"], ",".join(wl["codes"]), steps)}
 
 
+def run_qsvrg(args):
+    """QSVRG (Section 3.3) on a synthetic ridge least-squares problem, n = 4096 (one bucket, s = 64),
+    K = 8 processors, dense code: time per inner iteration (K encodes + one fused decode + the torch
+    gradient arithmetic). Vectors of 16 KB make this launch-bound; reported for completeness."""
+    import torch
+    import paper_1610_02132_b200 as Q
+    from paper_1610_02132_b200 import inputs as I
+    from paper_1610_02132_b200 import qsvrg as GV
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    n, m, K, lam = 4096, 16384, 8, 0.1
+    A, b = I.least_squares_problem(m, n, seed=1)
+    gs, gj = GV.least_squares_gradients(torch.from_numpy(A).cuda(), torch.from_numpy(b).cuda(), lam, K)
+    T = max(args.steps, 1) * 20
+    idx = I.sample_indices(2, T, K, m, seed=3)
+    eta = 0.1 / (1 + lam)
+    GV.qsvrg(gs, gj, n, K, 1, max(args.warmup, 3) * 5, eta, idx, np.zeros(n, np.float32))      # warm-up
+    torch.cuda.synchronize()
+    l0 = Q.qsgd_launch_count()
+    t0 = time.perf_counter()
+    out = GV.qsvrg(gs, gj, n, K, 1, T, eta, idx, np.zeros(n, np.float32))
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    A64, b64 = A.astype(np.float64), b.astype(np.float64)
+    f = lambda x: 0.5 * np.mean((A64 @ x - b64) ** 2) + 0.5 * lam * np.dot(x, x)  # noqa: E731
+    line = {
+        "metric": "QSGD encode + decode+aggregate throughput, fp32 gradient GB/s",
+        "value": 2 * K * 4 * n * (T + 1) / dt / 1e9, "unit": "GB/s", "n_gpus": 1, "steps": T, "warmup": args.warmup,
+        "ms_per_step": 1e3 * dt / (T + 1), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "qsvrg: ridge least squares, unit rows, one epoch", "n": n, "bucket": n, "s": 64,
+                   "norm": "l2", "codes": ["elias_dense"], "K": K, "m": m, "T": T},
+        "gpu_launches": int(Q.qsgd_launch_count() - l0),
+        "bits_per_processor": int(out["bits"][0]), "bound_bits": float((32 + 2.8 * n) * (T + 1)),
+        "f_start": float(f(np.zeros(n))), "f_after_epoch": float(f(out["y"][-1].astype(np.float64))),
+    }
+    print(json.dumps(line))
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -700,7 +740,7 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS) + ["sweep"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS) + ["sweep", "qsvrg"])
     ap.add_argument("--n", type=int, default=None)
     ap.add_argument("--d", type=int, default=None)
     ap.add_argument("--s", type=int, default=None)
@@ -728,6 +768,8 @@ def main():
         args.warmup = max(args.warmup, 3)
     if args.workload == "sweep":
         run_sweep(args)
+    elif args.workload == "qsvrg":
+        run_qsvrg(args)
     elif args.exchange:
         run_exchange(args)
     else:

@@ -8,7 +8,8 @@ TEST INFRASTRUCTURE ONLY, like oracle.py. Written step by step in the paper's or
              x_(t+1) = x_t - eta * (1 / K) * sum_i u_i;
   end:       y^(p+1) = (1 / T) * sum_t x_t.
 
-Q~(v) = Q(v, s) with s = floor(sqrt(n)) levels and the 2-norm of the whole vector (one bucket = n).
+Q~(v) = Q(v, s) with s = floor(sqrt(n)) levels and the 2-norm of the whole vector (one bucket = n);
+the max-norm of Section 4 can be chosen instead.
 Every broadcast goes through Encode and Decode of the oracle, so message bits are the paper's
 |Code'_s| (or |Code_s|, or the fixed-width size). The gradients come from caller-supplied functions so
 that a test can hand the same arithmetic to this file and to the GPU path.
@@ -23,7 +24,7 @@ def default_levels(n):
 
 
 def qsvrg(grad_share, grad_sample, n, K, P, T, eta, indices, x0, code_kind=O.CODE_ELIAS_DENSE, s=None,
-          seed=7, quantize_full=True):
+          seed=7, quantize_full=True, norm_kind=O.NORM_L2):
     """grad_share(i, y) -> grad h_i(y); grad_sample(j, x) -> grad f_j(x); indices[p, t, i] = j.
     quantize_full: the appendix quantizes the per-epoch broadcast of grad h_i, the main text sends it
     in full precision (then H_p is the fp32 sum in processor order and costs 32 n bits each).
@@ -38,7 +39,7 @@ def qsvrg(grad_share, grad_sample, n, K, P, T, eta, indices, x0, code_kind=O.COD
         """Every processor encodes its vector; returns the messages as all processors decode them."""
         msgs, tabs = [], []
         for i, v in enumerate(vectors):
-            m, info = O.encode(np.asarray(v, dtype=np.float32), n, s, O.NORM_L2, code_kind, seed, step, i)
+            m, info = O.encode(np.asarray(v, dtype=np.float32), n, s, norm_kind, code_kind, seed, step, i)
             bits[i] += info[0]
             msgs.append(m)
             tabs.append(None if code_kind == O.CODE_FIXED else O.message_table(m, info, n, n))
