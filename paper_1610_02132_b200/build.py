@@ -8,7 +8,7 @@ CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libqsgd.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-shared", "-Xcompiler", "-fPIC", "--cudart", "shared"]
+              "-shared", "-Xcompiler", "-fPIC", "--cudart", "shared", "--threads", "0"]
 
 
 def sources():

@@ -1,0 +1,435 @@
+// Decode-and-aggregate, Elias path, optionally fused with the SGD step (Section 3.1: "read off
+// 32 bits to construct the norm, then iteratively ... read off the positions and values of the
+// nonzeros"; Appendix A.2 decoder; Algorithm 1 for the sum and the step).
+//
+// A string S can only be parsed front to back, but buckets and peers are independent once the
+// per-bucket offset table gives each string's first bit. A warp owns a group of G buckets.
+// Phase 1 (parse): lane (g, k) reads peer k's string of bucket g through a 64-bit register
+// window (next word prefetched) and rebuilds that peer's *fixed-width fields* -- level fields
+// and sign bitmap -- for the bucket in shared memory. Phase 2 (apply): exactly the fixed-width
+// decoder's inner loop, reading the fields from shared memory: every lane takes 16 coordinates
+// and adds the peers in ascending k, which fixes the summation order however phase 1 was
+// scheduled. Shapes whose fields do not fit in shared memory go to the
+// decoder of elias_decode_slow.cu.
+#include "elias_decode.cuh"
+
+namespace qsgd {
+
+namespace {
+
+template <int LB, bool DENSE>
+__device__ __forceinline__ uint32_t parse_to_fields(const uint32_t* __restrict__ words,
+                                                    const uint64_t* __restrict__ table, uint64_t b,
+                                                    uint64_t B, uint32_t db, uint32_t d, uint32_t s,
+                                                    const uint16_t* lut, uint32_t* __restrict__ row,
+                                                    float* A_out) {
+  const uint64_t lo = __ldg(table + b), hi = __ldg(table + b + 1), all = __ldg(table + B);
+  *A_out = 0.f;
+  if (hi < lo || hi - lo < 32 || hi > all) return QSGD_DEV_TABLE;
+  const uint64_t cap_bits = (uint64_t)((const uint8_t*)table - (const uint8_t*)words) * 8ull;
+  if ((const uint8_t*)table > (const uint8_t*)words && all > cap_bits) return QSGD_DEV_TABLE;
+  if (hi - lo > 32ull + (uint64_t)db * 40ull) return QSGD_DEV_OVERRUN;   // longer than any legal string
+  const uint32_t total = (uint32_t)(hi - lo) - 32u;
+  BitSrc src;
+  src.open(words, lo);
+  *A_out = __uint_as_float(src.take(32));
+  uint32_t* srow = row + ((d * LB) >> 5);            // sign bitmap of this peer row
+  uint32_t used = 0, err = 0;
+  // The row is zero and only this lane writes it, so fields are OR-ed in place.
+  if (DENSE) {
+    for (uint32_t c = 0; c < db; ++c) {
+      src.refill();
+      const uint32_t neg = src.hi >> 31;
+      uint32_t v;
+      if (!read_int(src, lut, 1u, v, used)) { err = QSGD_DEV_OVERRUN; break; }
+      if (used > total) { err = QSGD_DEV_OVERRUN; break; }
+      if (v - 1u > s) { err = QSGD_DEV_LEVEL; break; }
+      if (v > 1u) {
+        row[(c * LB) >> 5] |= (v - 1u) << ((c * LB) & 31);
+        if (neg) srow[c >> 5] |= 1u << (c & 31);
+      }
+    }
+    if (!err && used != total) err = QSGD_DEV_OVERRUN;
+  } else {
+    uint32_t at = 0xFFFFFFFFu;                        // position of the previous nonzero (-1)
+    while (used < total && err == 0u) {
+      // One refill leaves >= 33 bits: enough for a table-decoded triple (<= 12 + 1 + 12 bits).
+      src.refill();
+      uint32_t gap, level, neg;
+      const uint32_t e1 = lut[src.hi >> (32 - kLutBits)];
+      if (e1) {
+        gap = e1 & 0xFFu;
+        src.drop(e1 >> 8);
+        used += e1 >> 8;
+      } else {
+        if (!src.elias(gap, used)) { err = QSGD_DEV_OVERRUN; break; }
+        src.refill();
+      }
+      neg = src.hi >> 31;
+      const uint32_t e2 = lut[(src.hi << 1) >> (32 - kLutBits)];
+      if (e2) {
+        level = e2 & 0xFFu;
+        src.drop((e2 >> 8) + 1u);
+        used += (e2 >> 8) + 1u;
+      } else {
+        src.drop(1);
+        used += 1;
+        if (!src.elias(level, used)) { err = QSGD_DEV_OVERRUN; break; }
+      }
+      at += gap;
+      err |= at >= db ? QSGD_DEV_POSITION : 0u;
+      err |= (level < 1u || level > s) ? QSGD_DEV_LEVEL : 0u;
+      err |= used > total ? QSGD_DEV_OVERRUN : 0u;
+      if (err == 0u) {
+        row[(at * LB) >> 5] |= level << ((at * LB) & 31);
+        srow[at >> 5] |= neg << (at & 31);
+      }
+    }
+  }
+  return err;
+}
+
+template <int LB, bool DENSE, bool FUSED, bool SINGLE>
+__global__ void __launch_bounds__(320) decode_elias_fields_kernel(const __grid_constant__ FieldParams p) {
+  extern __shared__ __align__(16) uint32_t fsm[];
+  __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
+  __shared__ uint16_t elias_lut[1u << kLutBits];
+  if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const float sf = (float)p.s;
+  float lut0 = 0.f;
+  fill_elias_lut(elias_lut);
+  if (LB == 8) {
+    for (uint32_t i = tid; i < 256 * 32; i += blockDim.x) xi_tab[i] = __fdiv_rn((float)(i >> 5), sf);
+  }
+  __syncthreads();
+  if (LB != 8) {
+    const uint32_t level = lane & ((1u << LB) - 1u), neg = (lane >> LB) & 1u;
+    const float q = __fdiv_rn((float)level, sf);
+    lut0 = neg ? -q : q;
+  }
+  const uint8_t* tab_lane = reinterpret_cast<const uint8_t*>(xi_tab) + 4 * lane;
+
+  const uint32_t warp_words = p.G * p.bucket_words;
+  uint32_t* mine = fsm + (size_t)warp * warp_words;
+  const uint32_t level_words = (p.d * LB) >> 5;
+  const uint32_t pg = lane / p.Kpad, pk = lane % p.Kpad;      // parse role: bucket in group, peer
+  const uint32_t slots_per_bucket = p.d >> 4;                 // 16-coordinate lane slots
+  const uint32_t total_slots = p.G * slots_per_bucket;
+  const uint64_t groups = (p.B + p.G - 1) / p.G;
+
+  for (uint64_t grp = (uint64_t)blockIdx.x * nwarps + warp; grp < groups; grp += (uint64_t)gridDim.x * nwarps) {
+    const uint64_t b0 = grp * p.G;
+    for (uint32_t q = lane; q < (warp_words >> 2); q += 32) reinterpret_cast<uint4*>(mine)[q] = make_uint4(0u, 0u, 0u, 0u);
+    __syncwarp();
+    // ---- phase 1: one lane per (bucket, peer) ------------------------------------------------
+    for (uint32_t k = pk; k < p.K; k += 32) {
+      const uint64_t b = b0 + pg;
+      if (pg < p.G && b < p.B) {
+        uint32_t* bucket = mine + pg * p.bucket_words;
+        const uint64_t base = b * p.d;
+        const uint32_t db = (uint32_t)min((uint64_t)p.d, p.n - base);
+        float A;
+        const uint32_t st = parse_to_fields<LB, DENSE>(p.peers.payload[k], p.peers.table[k], b, p.B, db, p.d,
+                                                       p.s, elias_lut, bucket + k * p.row_words, &A);
+        reinterpret_cast<float*>(bucket + p.K * p.row_words)[k] = A;
+        if (st) atomicOr(p.status, st);
+      }
+      if (p.Kpad < 32) break;
+    }
+    __syncwarp();
+    // ---- phase 2: the fixed-width decoder's inner loop over the rebuilt fields ----------------
+    for (uint32_t s0 = 0; s0 < total_slots; s0 += 32) {
+      const uint32_t slot = s0 + lane;
+      const uint32_t g = slot / slots_per_bucket, c = (slot - g * slots_per_bucket) << 4;
+      const uint64_t b = b0 + g;
+      const uint64_t i0 = b * p.d + c;
+      const bool live = slot < total_slots && b < p.B && i0 < p.n;
+      const uint32_t* bucket = mine + (live ? g : 0) * p.bucket_words;
+      const float* scales = reinterpret_cast<const float*>(bucket + p.K * p.row_words);
+      float acc[16];
+#pragma unroll
+      for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+#pragma unroll 2
+      for (uint32_t k = 0; k < p.K; ++k) {
+        const uint32_t* row = bucket + k * p.row_words;
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        uint32_t sb = 0;
+        float A = 0.f;
+        if (live) {
+          A = scales[k];
+          sb = (row[level_words + (c >> 5)] >> (c & 31)) & 0xFFFFu;
+          if (LB == 8) {
+            const uint4 t = *reinterpret_cast<const uint4*>(row + (c >> 2));
+            w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
+          } else if (LB == 4) {
+            const uint2 t = *reinterpret_cast<const uint2*>(row + (c >> 3));
+            w[0] = t.x; w[1] = t.y;
+          } else if (LB == 2) {
+            w[0] = row[c >> 4];
+          } else {
+            w[0] = (row[c >> 5] >> (c & 31)) & 0xFFFFu;
+          }
+        }
+        if (LB == 8) add_peer_tab(acc, w, sb, tab_lane, A);
+        else if (SINGLE) add_peer_lut<LB, true>(acc, w, sb, __fmul_rn(__shfl_sync(0xffffffffu, A, 0), lut0), A);
+        else add_peer_lut<LB, false>(acc, w, sb, lut0, A);
+      }
+      if (live) {
+        if (p.map.src) store_span16<FUSED>(out_span(p.out, p.map, b, c, p.d, p.n, 16u), acc, p.c);
+        else store_lane16<FUSED>(p.out + i0, acc, i0, p.n, p.c);
+      }
+    }
+    __syncwarp();
+  }
+}
+
+template <int LB, bool DENSE>
+int launch_fields(FieldParams& p, bool fused, cudaStream_t stream, bool* handled) {
+  *handled = false;
+  int dev = 0, max_smem = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const uint32_t level_words = (p.d * LB) >> 5, sign_words = p.d >> 5;
+  p.row_words = (level_words + sign_words + 3u) & ~3u;
+  p.bucket_words = (p.K * p.row_words + p.K + 3u) & ~3u;
+  uint32_t kpad = 1;
+  while (kpad < p.K && kpad < 32) kpad <<= 1;
+  p.Kpad = kpad;
+  uint32_t G = p.K <= 32 ? 32 / kpad : 1;
+  while (G > 1 && (size_t)G * p.bucket_words * 4 > (16u << 10)) G >>= 1;
+  p.G = G;
+  const size_t per_warp = (size_t)G * p.bucket_words * 4;
+  const size_t budget = (size_t)max_smem - (LB == 8 ? 32768 : 128) - 8192 - 1024;
+  // Warps per CTA: the count that leaves the most warps resident on an SM. The code table and the
+  // level table are per CTA, the fields per warp; the parse is latency-bound, so warps are what counts.
+  const size_t per_cta = (LB == 8 ? 32768 : 128) + 8192 + 1024;
+  const size_t per_sm = 227u << 10;
+  int warps = 0, best = 0;
+  for (int w = 1; w <= 10; ++w) {
+    if ((size_t)w * per_warp > budget) break;
+    const int resident = (int)(per_sm / ((size_t)w * per_warp + per_cta)) * w;
+    if (resident > best) { best = resident; warps = w; }
+  }
+  if (warps == 0) return 0;                                      // caller falls back to the slow kernel
+  const bool single = p.d >= 512 && (p.d & (p.d - 1)) == 0 && LB != 8;
+  void (*kern)(FieldParams);
+  if (fused) kern = single ? decode_elias_fields_kernel<LB, DENSE, true, true> : decode_elias_fields_kernel<LB, DENSE, true, false>;
+  else kern = single ? decode_elias_fields_kernel<LB, DENSE, false, true> : decode_elias_fields_kernel<LB, DENSE, false, false>;
+  const size_t smem = (size_t)warps * per_warp;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return (int)e;
+  int occ = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, warps * 32, smem);
+  if (e != cudaSuccess) return (int)e;
+  if (occ < 1) occ = 1;
+  const uint64_t groups = (p.B + G - 1) / G;
+  const uint64_t want = (groups + warps - 1) / warps;
+  const uint64_t cap = (uint64_t)sms * occ;
+  const uint32_t grid = (uint32_t)(want < cap ? want : cap);
+  {
+    ScopedKernel sk(kKernDecodeElias, stream);
+    kern<<<grid, warps * 32, smem, stream>>>(p);
+  }
+  *handled = true;
+  return (int)cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// Field-rebuilding decoder for long buckets (d >= 1024): the same two phases, but a bucket is
+// walked in ranges of 512 positions. A lane keeps its place in its string between ranges (bit
+// window, position, one decoded entry that lies past the range), so shared memory holds the fields
+// of one range only and as many warps fit on an SM as for d = 512; with whole-bucket fields a CTA
+// of d = 4096 is down to one or two warps.
+// ------------------------------------------------------------------------------------------------
+template <int LB, bool DENSE, bool FUSED>
+__global__ void __launch_bounds__(128) decode_elias_ranged_kernel(const __grid_constant__ FieldParams p) {
+  constexpr uint32_t kR = 512;                                  // positions per range = one warp pass of phase 2
+  constexpr uint32_t kLevelWords = kR * LB / 32, kRowWords = kLevelWords + kR / 32;
+  extern __shared__ __align__(16) uint32_t fsm[];
+  __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
+  if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const float sf = (float)p.s;
+  float lut0 = 0.f;
+  if (LB == 8) {
+    for (uint32_t i = tid; i < 256 * 32; i += blockDim.x) xi_tab[i] = __fdiv_rn((float)(i >> 5), sf);
+  }
+  __syncthreads();
+  if (LB != 8) {
+    const uint32_t level = lane & ((1u << LB) - 1u), neg = (lane >> LB) & 1u;
+    const float q = __fdiv_rn((float)level, sf);
+    lut0 = neg ? -q : q;
+  }
+  const uint8_t* tab_lane = reinterpret_cast<const uint8_t*>(xi_tab) + 4 * lane;
+
+  // per warp: G * K rows of kRowWords (level fields, then sign bits, of one range) | 32 scales
+  const uint32_t rows_words = p.G * p.K * kRowWords;
+  uint32_t* mine = fsm + (size_t)warp * (rows_words + 32u);
+  float* scales = reinterpret_cast<float*>(mine + rows_words);
+  const uint32_t pg = lane / p.Kpad, pk = lane % p.Kpad;      // parse role: bucket in group, peer
+  uint32_t* row = mine + (pg * p.K + pk) * kRowWords;         // this lane's row (when it parses)
+  const uint64_t groups = (p.B + p.G - 1) / p.G;
+
+  for (uint64_t grp = (uint64_t)blockIdx.x * nwarps + warp; grp < groups; grp += (uint64_t)gridDim.x * nwarps) {
+    const uint64_t b0 = grp * p.G;
+    // ---- open this lane's string ---------------------------------------------------------------
+    LaneParse st;
+    st.used = st.total = st.err = 0u;
+    st.at = 0xFFFFFFFFu;
+    st.pend = kNoEntry;
+    uint32_t db = 0;
+    float A = 0.f;
+    if (pg < p.G && b0 + pg < p.B) db = (uint32_t)min((uint64_t)p.d, p.n - (b0 + pg) * p.d);
+    const bool parsing = db != 0u && pk < p.K;
+    if (parsing) {
+      const uint64_t b = b0 + pg;
+      const uint32_t* words = p.peers.payload[pk];
+      const uint64_t* table = p.peers.table[pk];
+      const uint64_t lo = __ldg(table + b), hi = __ldg(table + b + 1), all = __ldg(table + p.B);
+      const uint64_t cap_bits = (uint64_t)((const uint8_t*)table - (const uint8_t*)words) * 8ull;
+      if (hi < lo || hi - lo < 32 || hi > all) st.err = QSGD_DEV_TABLE;
+      else if ((const uint8_t*)table > (const uint8_t*)words && all > cap_bits) st.err = QSGD_DEV_TABLE;
+      else if (hi - lo > 32ull + (uint64_t)db * 40ull) st.err = QSGD_DEV_OVERRUN;   // longer than any legal string
+      else {
+        st.total = (uint32_t)(hi - lo) - 32u;
+        st.src.open(words, lo);
+        A = __uint_as_float(st.src.take(32));
+      }
+    }
+    scales[lane] = A;
+    const bool readable = parsing && st.err == 0u;
+
+    for (uint32_t rbeg = 0; rbeg < p.d; rbeg += kR) {
+      const uint32_t rend = min(rbeg + kR, p.d);
+      for (uint32_t q = lane; q < (rows_words >> 2); q += 32) reinterpret_cast<uint4*>(mine)[q] = make_uint4(0u, 0u, 0u, 0u);
+      __syncwarp();
+      // ---- phase 1: this lane's entries of the range, OR-ed into its zeroed row ----------------
+      if (readable) {
+        uint32_t* srow = row + kLevelWords;
+        if (DENSE) {
+          for (uint32_t c = rbeg; c < min(rend, db) && st.err == 0u; ++c) {
+            st.src.refill();
+            const uint32_t neg = st.src.hi >> 31;
+            uint32_t v, len;
+            const bool ok = elias_from_window(st.src.hi << 1, v, len);
+            st.src.drop(len + 1u);
+            st.used += len + 1u;
+            if (!ok || st.used > st.total) st.err = QSGD_DEV_OVERRUN;
+            else if (v - 1u > p.s) st.err = QSGD_DEV_LEVEL;
+            else if (v > 1u) {
+              const uint32_t pos = c - rbeg;
+              row[(pos * LB) >> 5] |= (v - 1u) << ((pos * LB) & 31);
+              srow[pos >> 5] |= neg << (pos & 31);
+            }
+          }
+        } else {
+          advance(st, rend, 0xFFFFFFFFu, db, p.s, [&](uint32_t, uint32_t en) {
+            const uint32_t pos = (en & 0xFFFFu) - rbeg;
+            row[(pos * LB) >> 5] |= ((en >> 16) & 0xFFu) << ((pos * LB) & 31);
+            srow[pos >> 5] |= (en >> 31) << (pos & 31);
+          });
+        }
+      }
+      __syncwarp();
+      // ---- phase 2: one warp pass per bucket over the range's fields, ascending k ---------------
+      for (uint32_t g = 0; g < p.G; ++g) {
+        const uint64_t b = b0 + g;
+        const uint32_t cl = lane << 4, c = rbeg + cl;           // position in the range / in the bucket
+        const uint64_t i0 = b * p.d + c;
+        const bool live = b < p.B && c < rend && i0 < p.n;
+        if (!__any_sync(0xffffffffu, live)) continue;
+        float acc[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) acc[e] = 0.f;
+#pragma unroll 2
+        for (uint32_t k = 0; k < p.K; ++k) {
+          const uint32_t* rk = mine + (g * p.K + k) * kRowWords;
+          uint32_t w[4] = {0u, 0u, 0u, 0u};
+          uint32_t sb = 0;
+          const float Ak = scales[g * p.Kpad + k];
+          if (live) {
+            sb = (rk[kLevelWords + (cl >> 5)] >> (cl & 31)) & 0xFFFFu;
+            if (LB == 8) {
+              const uint4 t = *reinterpret_cast<const uint4*>(rk + (cl >> 2));
+              w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
+            } else if (LB == 4) {
+              const uint2 t = *reinterpret_cast<const uint2*>(rk + (cl >> 3));
+              w[0] = t.x; w[1] = t.y;
+            } else if (LB == 2) {
+              w[0] = rk[cl >> 4];
+            } else {
+              w[0] = (rk[cl >> 5] >> (cl & 31)) & 0xFFFFu;
+            }
+          }
+          if (LB == 8) add_peer_tab(acc, w, sb, tab_lane, live ? Ak : 0.f);
+          else add_peer_lut<LB, true>(acc, w, sb, __fmul_rn(Ak, lut0), Ak);
+        }
+        if (live) {
+          if (p.map.src) store_span16<FUSED>(out_span(p.out, p.map, b, c, p.d, p.n, 16u), acc, p.c);
+          else store_lane16<FUSED>(p.out + i0, acc, i0, p.n, p.c);
+        }
+      }
+      __syncwarp();
+    }
+    // a string must end exactly where the table says
+    if (readable && st.err == 0u && (st.used != st.total || st.pend != kNoEntry)) st.err = QSGD_DEV_OVERRUN;
+    if (st.err) atomicOr(p.status, st.err);
+    __syncwarp();
+  }
+}
+
+template <int LB, bool DENSE>
+int launch_ranged(FieldParams& p, bool fused, cudaStream_t stream, bool* handled) {
+  *handled = false;
+  if (p.K > 32u) return 0;
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  constexpr uint32_t kRowWords = 512u * LB / 32u + 16u;
+  uint32_t kpad = 1;
+  while (kpad < p.K) kpad <<= 1;
+  p.Kpad = kpad;
+  p.G = 32u / kpad;
+  const size_t per_warp = ((size_t)p.G * p.K * kRowWords + 32u) * 4;   // at most 18.6 KB
+  const int warps = 4;
+  auto kern = fused ? decode_elias_ranged_kernel<LB, DENSE, true> : decode_elias_ranged_kernel<LB, DENSE, false>;
+  const size_t smem = (size_t)warps * per_warp;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return (int)e;
+  int occ = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, warps * 32, smem);
+  if (e != cudaSuccess) return (int)e;
+  if (occ < 1) occ = 1;
+  const uint64_t groups = (p.B + p.G - 1) / p.G;
+  const uint64_t want = (groups + warps - 1) / warps;
+  const uint64_t cap = (uint64_t)sms * occ;
+  const uint32_t grid = (uint32_t)(want < cap ? want : cap);
+  {
+    ScopedKernel sk(kKernDecodeElias, stream);
+    kern<<<grid, warps * 32, smem, stream>>>(p);
+  }
+  *handled = true;
+  return (int)cudaGetLastError();
+}
+
+template <int LB>
+int launch_fields_lb(FieldParams& p, bool dense, bool fused, cudaStream_t stream, bool* handled) {
+  if (p.d >= 1024u && p.K <= 32u)       // long buckets: fields of one range at a time
+    return dense ? launch_ranged<LB, true>(p, fused, stream, handled) : launch_ranged<LB, false>(p, fused, stream, handled);
+  return dense ? launch_fields<LB, true>(p, fused, stream, handled) : launch_fields<LB, false>(p, fused, stream, handled);
+}
+
+}  // namespace
+
+int launch_elias_fields(FieldParams& p, bool dense, bool fused, cudaStream_t stream, bool* handled) {
+  switch (level_bits_for(p.s)) {
+    case 1: return launch_fields_lb<1>(p, dense, fused, stream, handled);
+    case 2: return launch_fields_lb<2>(p, dense, fused, stream, handled);
+    case 4: return launch_fields_lb<4>(p, dense, fused, stream, handled);
+    default: return launch_fields_lb<8>(p, dense, fused, stream, handled);
+  }
+}
+
+}  // namespace qsgd
