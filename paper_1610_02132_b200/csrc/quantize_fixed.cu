@@ -142,15 +142,46 @@ constexpr uint32_t kTwo23Bits = 0x4B000000u;
 
 // One coordinate. Returns the raw bits of 2^23 + level (level clamped to s); pushes the sign
 // bit into `sw`.
+// RAW_SIGN: push the sign bit of v as it is; the caller clears the signs of zero levels afterwards
+// with a mask derived from the packed level words (cheaper than two more operations per coordinate
+// when a word holds many fields).
+template <bool RAW_SIGN>
 __device__ __forceinline__ uint32_t quantize_one(float v, float r, float sf, float cap, uint32_t rnd,
                                                  uint32_t& sw) {
   const float t = __fmul_rn(__fmul_rn(sf, fabsf(v)), r);
   const float c = fma_rn(__uint2float_rn(rnd >> 8), 5.9604644775390625e-08f, t);
   const float fl = fminf(__fadd_rd(c, kTwo23), cap);       // 2^23 + min(floor(c), s)
-  const float lf = __fsub_rn(fl, kTwo23);                   // the level as a float, exact
-  const float sv = fma_rn(lf, v, 0.0f);                     // sign set iff level > 0 and v < 0
-  sw = __funnelshift_l(__float_as_uint(sv), sw, 1);
+  if (RAW_SIGN) {
+    sw = __funnelshift_l(__float_as_uint(v), sw, 1);
+  } else {
+    const float lf = __fsub_rn(fl, kTwo23);                 // the level as a float, exact
+    const float sv = fma_rn(lf, v, 0.0f);                   // sign set iff level > 0 and v < 0
+    sw = __funnelshift_l(__float_as_uint(sv), sw, 1);
+  }
   return __float_as_uint(fl);
+}
+
+// Bit e of the result is set iff level field e of the 16 coordinates packed in lw is nonzero.
+template <int LB>
+__device__ __forceinline__ uint32_t nonzero_fields16(const uint32_t (&lw)[4]) {
+  if (LB == 1) return lw[0] & 0xFFFFu;
+  if (LB == 2) {
+    uint32_t y = (lw[0] | (lw[0] >> 1)) & 0x55555555u;
+    y = (y | (y >> 1)) & 0x33333333u;
+    y = (y | (y >> 2)) & 0x0F0F0F0Fu;
+    y = (y | (y >> 4)) & 0x00FF00FFu;
+    return (y | (y >> 8)) & 0xFFFFu;
+  }
+  uint32_t m = 0;                                           // LB == 4: two words of eight fields
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    uint32_t y = lw[h] | (lw[h] >> 1);
+    y = (y | (y >> 2)) & 0x11111111u;
+    y = (y | (y >> 3)) & 0x03030303u;
+    y = (y | (y >> 6)) & 0x000F000Fu;
+    m |= ((y | (y >> 12)) & 0xFFu) << (8 * h);
+  }
+  return m;
 }
 
 constexpr int kStages = 3;
@@ -392,7 +423,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
       const uint32_t rr[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
 #pragma unroll
       for (int e = 3; e >= 0; --e) {
-        const uint32_t bits = quantize_one(v[4 * c4 + e], r, sf, cap, rr[e], sw);
+        const uint32_t bits = quantize_one<LB != 8>(v[4 * c4 + e], r, sf, cap, rr[e], sw);
         if (LB == 8) lw[c4] = lw[c4] * 256u + bits;
         else if (LB == 4) lw[c4 >> 1] = lw[c4 >> 1] * 16u + bits;
         else if (LB == 2) lw[0] = lw[0] * 4u + bits;
@@ -411,6 +442,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
     } else {
       lw[0] = (lw[0] - kTwo23Bits * 0xFFFFu) & 0xFFFFu;
     }
+    if (LB != 8) sw &= nonzero_fields16<LB>(lw);          // canonical sign: 0 where the level is 0
 
     // ---- stores (full tiles only: no bounds to check) -----------------------------------------
     {
