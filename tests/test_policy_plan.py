@@ -55,3 +55,24 @@ def test_plan_rejects_bad_arguments():
         Q.Policy([0, 0], 512, device="cpu")
     with pytest.raises(Q.QsgdError):
         Q.Policy([100], 100, device="cpu")
+
+
+def test_policy_entry_points_validate_before_launching():
+    """Argument errors come back as negative status codes with no GPU work (none is available here)."""
+    import ctypes as C
+    from paper_1610_02132_b200 import binding as B
+    L = B.lib()
+    pl = Q.Policy([64, 20000], 512, device="cpu")
+    st = B.PolicyStruct(0, 0, pl.n_buckets, 0, 0, pl.n_raw_segments, pl.n_raw, pl.n, 1)    # null plan arrays
+    assert L.qsgd_policy_encode(None, C.byref(st), 512, 15, 0, 0, 7, 0, 0, None, 0, None, None, None, None) == -1
+    assert L.qsgd_policy_message_capacity(C.byref(st), 512, 15, 0) == 0
+    good = B.PolicyStruct(16, 16, pl.n_buckets, 16, 16, pl.n_raw_segments, pl.n_raw, pl.n, 1)    # non-null, never read
+    assert L.qsgd_policy_message_capacity(C.byref(good), 512, 15, 0) == \
+        pl.raw_prefix + Q.qsgd_message_capacity(pl.n_buckets * 512, 512, 15, 0)
+    assert L.qsgd_policy_message_capacity(C.byref(good), 100, 15, 0) == 0                        # bad bucket
+    assert L.qsgd_policy_workspace_bytes(C.byref(good), 512, 15, 0) == 0                         # fixed-width: none
+    assert L.qsgd_policy_workspace_bytes(C.byref(good), 512, 15, 1) == Q.qsgd_workspace_bytes(pl.n_buckets * 512, 512, 15, 1)
+    msgs = (C.c_void_p * 1)(16)
+    assert L.qsgd_policy_decode_sgd_step(msgs, None, 0, C.byref(good), 512, 15, 0, 16, 0.1, 16, None) == -7   # K = 0
+    assert L.qsgd_policy_decode_sgd_step(msgs, None, 1, C.byref(good), 512, 15, 0, 8, 0.1, 16, None) == -5    # x misaligned
+    assert L.qsgd_policy_decode_sgd_step(msgs, None, 1, C.byref(good), 512, 15, 1, 16, 0.1, 16, None) == -1   # Elias needs tables
