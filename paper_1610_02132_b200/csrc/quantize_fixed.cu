@@ -125,14 +125,16 @@ __device__ __forceinline__ uint4 philox_q(uint32_t q, const PhiloxConsts& pc) {
   c1 = (uint32_t)p1;
   c2 = (uint32_t)(p0 >> 32) ^ pc.z2;
   uint32_t c3 = (uint32_t)p0;
+  // rounds 3 .. 9: the high and low halves by separate multiplies (measured slightly faster than the
+  // 64-bit products here; the first rounds stay as they are, where it measured slower)
 #pragma unroll
   for (int r = 0; r < 7; ++r) {
-    p0 = (uint64_t)kM0 * c0;
-    p1 = (uint64_t)kM1 * c2;
-    c0 = (uint32_t)(p1 >> 32) ^ c1 ^ pc.k[r][0];
-    c1 = (uint32_t)p1;
-    c2 = (uint32_t)(p0 >> 32) ^ c3 ^ pc.k[r][1];
-    c3 = (uint32_t)p0;
+    const uint32_t h0 = __umulhi(kM0, c0), l0 = kM0 * c0;
+    const uint32_t h1 = __umulhi(kM1, c2), l1 = kM1 * c2;
+    c0 = h1 ^ c1 ^ pc.k[r][0];
+    c1 = l1;
+    c2 = h0 ^ c3 ^ pc.k[r][1];
+    c3 = l0;
   }
   return make_uint4(c0, c1, c2, c3);
 }
