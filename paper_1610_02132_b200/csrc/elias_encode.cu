@@ -495,8 +495,19 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
   extern __shared__ uint32_t stage[];
   __shared__ uint32_t warp_sum[kWarps];
   __shared__ uint32_t tab[17];
+  // whole code words (code | length << 16) of the integers met most: every level, and gaps below 64
+  __shared__ uint32_t level_code[1u << LB];
+  __shared__ uint32_t gap_code[64];
   if (!ctrl->ok) return;
   fill_code_table(tab);
+  if (!DENSE) {
+    for (uint32_t k = threadIdx.x; k < (1u << LB) + 64u; k += kThreads) {
+      const uint32_t v = k < (1u << LB) ? k : k - (1u << LB);
+      uint32_t ln = 0;
+      const uint32_t code = v ? elias_code(v, &ln) : 0u;
+      (k < (1u << LB) ? level_code[v] : gap_code[v]) = code | (ln << 16);
+    }
+  }
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t tl = lane & (p.lpb - 1), team = lane / p.lpb, bpw = 32 / p.lpb;
   const uint64_t b = (uint64_t)blockIdx.x * p.nbc + warp * bpw + team;
@@ -557,6 +568,46 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
         uint32_t ln;
         const uint32_t code = tab_code(tab, level_at<LB>(lwb, c) + 1u, &ln);
         bw.put((sg << ln) | code, ln + 1);
+      }
+    } else if ((p.seg & 63u) == 0u) {
+      // Ranges of whole 64-coordinate blocks (every power-of-two d >= 64): the block's nonzero mask
+      // and sign bits sit in registers, code words come whole from the two tables.
+      constexpr uint32_t kFields = 32u / LB, kMask = (1u << LB) - 1u;
+      for (uint32_t c0 = c_lo; c0 < c_hi; c0 += 64u) {
+        const uint32_t* wp = lwb + ((c0 * LB) >> 5);
+        unsigned long long m = 0ull;
+#pragma unroll
+        for (uint32_t j = 0; j < 2u * LB; ++j) {
+          const uint32_t w = (c0 + j * kFields < c_hi) ? __ldg(wp + j) : 0u;
+          m |= (unsigned long long)nonzero_mask<LB>(w) << (j * kFields);
+        }
+        const uint32_t s0 = __ldg(swb + (c0 >> 5)), s1 = (c0 + 32u < c_hi) ? __ldg(swb + (c0 >> 5) + 1) : 0u;
+        const unsigned long long signs = (unsigned long long)s0 | ((unsigned long long)s1 << 32);
+        while (m) {
+          const uint32_t off = (uint32_t)__ffsll((long long)m) - 1u;
+          m &= m - 1ull;
+          const uint32_t pos = c0 + off, bit = off * LB;
+          const uint32_t level = (__ldg(wp + (bit >> 5)) >> (bit & 31u)) & kMask;
+          const uint32_t gap = pos - (uint32_t)prev;
+          uint32_t gcode, gl;
+          if (gap < 64u) {
+            const uint32_t e = gap_code[gap];
+            gcode = e & 0xFFFFu;
+            gl = e >> 16;
+          } else {
+            gcode = tab_code(tab, gap, &gl);
+          }
+          const uint32_t e = level_code[level];
+          const uint32_t ll = e >> 16;
+          const uint32_t lcode = (e & 0xFFFFu) | ((uint32_t)((signs >> off) & 1ull) << ll);
+          if (gl + ll + 1u <= 32u) {                     // gap, sign and level in one piece (the rule)
+            bw.put((gcode << (ll + 1u)) | lcode, gl + ll + 1u);
+          } else {
+            bw.put(gcode, gl);
+            bw.put(lcode, ll + 1u);
+          }
+          prev = (int32_t)pos;
+        }
       }
     } else {
       for_each_nonzero<LB>(lwb, c_lo, c_hi, [&](uint32_t pos, uint32_t level) {
