@@ -52,7 +52,7 @@ __device__ __forceinline__ uint32_t parse_to_fields(const uint32_t* __restrict__
     if (!err && used != total) err = QSGD_DEV_OVERRUN;
   } else {
     uint32_t at = 0xFFFFFFFFu;                        // position of the previous nonzero (-1)
-    while (used < total && err == 0u) {
+    while (used < total) {
       // One refill leaves >= 33 bits: enough for a table-decoded triple (<= 12 + 1 + 12 bits).
       src.refill();
       uint32_t gap, level, neg;
@@ -77,13 +77,14 @@ __device__ __forceinline__ uint32_t parse_to_fields(const uint32_t* __restrict__
         if (!src.elias(level, used)) { err = QSGD_DEV_OVERRUN; break; }
       }
       at += gap;
-      err |= at >= db ? QSGD_DEV_POSITION : 0u;
-      err |= (level < 1u || level > s) ? QSGD_DEV_LEVEL : 0u;
-      err |= used > total ? QSGD_DEV_OVERRUN : 0u;
-      if (err == 0u) {
-        row[(at * LB) >> 5] |= level << ((at * LB) & 31);
-        srow[at >> 5] |= neg << (at & 31);
+      if (at >= db || level - 1u >= s || used > total) {     // one rarely taken branch for all three checks
+        err = at >= db ? QSGD_DEV_POSITION : 0u;
+        err |= level - 1u >= s ? QSGD_DEV_LEVEL : 0u;
+        err |= used > total ? QSGD_DEV_OVERRUN : 0u;
+        break;
       }
+      row[(at * LB) >> 5] |= level << ((at * LB) & 31);
+      srow[at >> 5] |= neg << (at & 31);
     }
   }
   return err;
