@@ -124,7 +124,12 @@ int qsgd_encode(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int nor
  * acc_i = ((+0 + g^0_i) + g^1_i) + ... in ascending k, where g^k_i = +-(A * (level / s)).
  *   msgs    host array of K device pointers to messages (16-byte aligned)
  *   tables  host array of K device pointers to the offset tables (Elias kinds; msgs[k] +
- *           out_bits[1]); NULL for fixed-width
+ *           out_bits[1]); NULL for fixed-width. A payload must be readable for 16 bytes past
+ *           its padded length (true when its table follows it, as Encode writes it). With the
+ *           table directly behind the payload the library reads the payload sizes off the
+ *           pointers and chooses between its decoders on the host; with tables kept elsewhere
+ *           it decides on the device (two launches, one of which returns at once). Results
+ *           are the same either way.
  *   acc     n fp32 values, overwritten
  */
 int qsgd_decode_accumulate(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
