@@ -31,9 +31,14 @@ def least_squares_gradients(A, b, lam, K):
         return (Ai.t() @ (Ai @ y - bi)) / m + (lam / K) * y
 
     def grad_sample(j, x):
+        """One function index, or a tensor of K indices: then a [K, n] tensor, one row per index."""
+        if torch.is_tensor(j) and j.dim() == 1:
+            a = A[j]                                              # [K, n]
+            return a * (a @ x - b[j]).unsqueeze(1) + lam * x
         a = A[j]
         return a * (torch.dot(a, x) - b[j]) + lam * x
 
+    grad_sample.batched = True
     return grad_share, grad_sample
 
 
@@ -55,6 +60,8 @@ def qsvrg(grad_share, grad_sample, n, K, P, T, eta, indices, x0, code_kind=Q.COD
     ws = torch.empty(max(Q.qsgd_workspace_bytes(n, n, s, code_kind), 16), dtype=torch.uint8, device=dev)
     status = Q.new_status(dev)
     H = torch.zeros(n, dtype=torch.float32, device=dev)
+    own_tables = torch.zeros(K, 2, dtype=torch.int64, device=dev)
+    idx_dev = torch.as_tensor(np.asarray(indices), dtype=torch.int64).to(dev)
 
     def broadcast(vectors, step):
         for i, v in enumerate(vectors):
@@ -63,10 +70,10 @@ def qsvrg(grad_share, grad_sample, n, K, P, T, eta, indices, x0, code_kind=Q.COD
         total_bits.add_(info[:, 0])
         if code_kind == Q.CODE_FIXED:
             return None
-        # the table offset is static here: one bucket, so the padded payload cannot be read off the
-        # host side without a copy; read the K offsets back (what a sender needs anyway to send)
-        offs = info[:, 1].cpu().tolist()
-        return [msgs[i][offs[i]: offs[i] + 16].view(torch.int64) for i in range(K)]
+        # One bucket per message: its offset table is (0, payload bits). Building it on the device
+        # from the size words avoids reading the table's place in the message back to the host.
+        own_tables[:, 1] = info[:, 0]
+        return [own_tables[i] for i in range(K)]
 
     for p in range(P):
         step0 = p * (T + 1)
@@ -82,12 +89,16 @@ def qsvrg(grad_share, grad_sample, n, K, P, T, eta, indices, x0, code_kind=Q.COD
         x_sum = torch.zeros(n, dtype=torch.float64, device=dev)
         for t in range(T):
             x_sum.add_(x.double())
-            us = []
-            for i in range(K):
-                j = int(indices[p, t, i])
-                gx = torch.as_tensor(grad_sample(j, x), dtype=torch.float32).to(dev)
-                gy = torch.as_tensor(grad_sample(j, y), dtype=torch.float32).to(dev)
-                us.append((gx - gy) + H)
+            if getattr(grad_sample, "batched", False):            # all K update vectors in a few tensor operations
+                js = idx_dev[p, t]
+                us = (grad_sample(js, x) - grad_sample(js, y)) + H
+            else:
+                us = []
+                for i in range(K):
+                    j = int(indices[p, t, i])
+                    gx = torch.as_tensor(grad_sample(j, x), dtype=torch.float32).to(dev)
+                    gy = torch.as_tensor(grad_sample(j, y), dtype=torch.float32).to(dev)
+                    us.append((gx - gy) + H)
             tables = broadcast(us, step0 + 1 + t)
             Q.qsgd_decode_sgd_step(msgs, tables, n, n, s, code_kind, x, eta, status)
         # a true fp64 division (a tensor divisor: a Python scalar would be turned into a multiplication)
