@@ -60,13 +60,14 @@ extern "C" {
 #define QSGD_CODE_ELIAS 1
 #define QSGD_CODE_ELIAS_DENSE 2
 
+#define QSGD_MAX_COORDS (1ull << 32) /* largest n accepted (16 GiB of fp32 gradient per call) */
 #define QSGD_MAX_BUCKET 4096
 #define QSGD_MAX_LEVELS 255
 #define QSGD_MAX_PEERS 64
 
 #define QSGD_OK 0
 #define QSGD_ERR_NULL (-1)      /* a required pointer is null                         */
-#define QSGD_ERR_SIZE (-2)      /* n == 0                                             */
+#define QSGD_ERR_SIZE (-2)      /* n == 0 or n > QSGD_MAX_COORDS                      */
 #define QSGD_ERR_BUCKET (-3)    /* bucket not a multiple of 32 in [32, 4096]          */
 #define QSGD_ERR_LEVELS (-4)    /* s outside [1, 255]                                 */
 #define QSGD_ERR_ALIGN (-5)     /* a pointer is not 16-byte aligned                   */
@@ -100,9 +101,16 @@ int qsgd_fixed_layout(uint64_t n, uint32_t bucket, uint32_t s, uint64_t* layout)
 
 /*
  * Encode (Algorithm 1, "M^i <- Encode(g^i)"; Section 3.1, Eq. 2 and the string S).
- * Per bucket: scale A (fp32; 2-norm accumulated in fp32 per 8 values and fp64 across them,
- * or the exact maximum); a scale below the smallest normal fp32 makes a zero bucket (A = +0,
- * all levels 0). Per coordinate i (global index): u = Philox4x32-10(counter = (i / 4 lo,
+ * Per bucket: scale A in fp32, the exact maximum or the 2-norm. The 2-norm is the correctly
+ * rounded square root of a sum of squares that the streaming kernels (power-of-two bucket, at
+ * least 4096 coordinates) accumulate in fp32 -- a chain of 16 fused multiply-adds per thread,
+ * then a shuffle tree over the bucket's lanes, then, for buckets of 1024 and more, up to 8
+ * sequential adds across warps -- and redo in fp64 when that sum leaves [8e-28, 1e30]; the
+ * generic kernel (other shapes, ragged tail) sums 8 squares in fp32 and those partial sums in
+ * fp64. Either way A lies within 1e-6 relative of the exact norm (at most 29 roundings of 2^-24
+ * on the sum, halved by the root), but the two kernels may give last-place differences for the
+ * same bucket, so a message is reproducible for a given (n, bucket), not across shapes. A scale
+ * below the smallest normal fp32 makes a zero bucket (A = +0, all levels 0). Per coordinate i (global index): u = Philox4x32-10(counter = (i / 4 lo,
  * i / 4 hi, step, worker), key = seed lo, hi) word i % 4, top 24 bits times 2^-24;
  * level = min(floor((s * |g_i|) * (1 / A) + u), s).
  *   g            n fp32 values, 16-byte aligned, read once
@@ -150,6 +158,19 @@ const char* qsgd_status_string(int status);
 
 /* Number of kernels this library has launched in this process (all calls, all streams). */
 uint64_t qsgd_launch_count(void);
+
+/*
+ * TEST HOOK, not part of the codec (the paper has no counterpart). The streaming encoder waits for
+ * its bulk copies with bounded polling; when a wait runs out the warp (or CTA) raises
+ * QSGD_DEV_TIMEOUT in status_dev, stops encoding, still waits -- with the full built-in bound --
+ * for the copies it has in flight, and returns. qsgd_test_set_wait_polls sets the bound of the
+ * main-loop waits for later launches of this process (0 = every such wait gives up at once), so a
+ * test can drive that path without any fault; qsgd_test_default_wait_polls returns the built-in
+ * bound to restore. Output written by a launch that timed out is unspecified inside the message
+ * buffer and never outside it.
+ */
+void qsgd_test_set_wait_polls(uint32_t polls);
+uint32_t qsgd_test_default_wait_polls(void);
 
 /*
  * Elias Encode that allocates nothing and needs no caller-supplied workspace. (The paper has no

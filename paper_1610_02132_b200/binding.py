@@ -22,7 +22,7 @@ EXPORTS = ["qsgd_message_capacity", "qsgd_workspace_bytes", "qsgd_fixed_layout",
            "qsgd_static_scratch_bytes", "qsgd_encode_elias_static",
            "qsgd_policy_plan_sizes", "qsgd_policy_plan", "qsgd_policy_message_capacity",
            "qsgd_policy_workspace_bytes", "qsgd_policy_encode", "qsgd_policy_decode_accumulate",
-           "qsgd_policy_decode_sgd_step"]
+           "qsgd_policy_decode_sgd_step", "qsgd_test_set_wait_polls", "qsgd_test_default_wait_polls"]
 
 _lib = None
 
@@ -90,6 +90,10 @@ def lib():
         L.qsgd_policy_decode_sgd_step.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, pp, u32, u32,
                                                   C.c_int, vp, C.c_float, vp, vp]
         L.qsgd_policy_decode_sgd_step.restype = C.c_int
+        L.qsgd_test_set_wait_polls.argtypes = [u32]
+        L.qsgd_test_set_wait_polls.restype = None
+        L.qsgd_test_default_wait_polls.argtypes = []
+        L.qsgd_test_default_wait_polls.restype = u32
         L.qsgd_profile_enable.argtypes = [C.c_int]
         L.qsgd_profile_enable.restype = None
         L.qsgd_profile_kernel_count.argtypes = []
@@ -134,6 +138,15 @@ def qsgd_fixed_layout(n, bucket, s):
 
 def qsgd_launch_count():
     return int(lib().qsgd_launch_count())
+
+
+def qsgd_test_set_wait_polls(polls):
+    """Test hook: bound of the streaming encoder's main-loop waits (0 = give up at once)."""
+    lib().qsgd_test_set_wait_polls(int(polls))
+
+
+def qsgd_test_default_wait_polls():
+    return int(lib().qsgd_test_default_wait_polls())
 
 
 def qsgd_profile_enable(on):

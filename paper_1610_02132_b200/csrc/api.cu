@@ -41,7 +41,7 @@ namespace {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int check_shape(uint64_t n, uint32_t bucket, uint32_t s, int code_kind) {
-  if (n == 0) return QSGD_ERR_SIZE;
+  if (n == 0 || n > QSGD_MAX_COORDS) return QSGD_ERR_SIZE;
   if (bucket < 32 || bucket > QSGD_MAX_BUCKET || (bucket & 31u)) return QSGD_ERR_BUCKET;
   if (s < 1 || s > QSGD_MAX_LEVELS) return QSGD_ERR_LEVELS;
   if (code_kind != QSGD_CODE_FIXED && code_kind != QSGD_CODE_ELIAS && code_kind != QSGD_CODE_ELIAS_DENSE)
@@ -339,7 +339,7 @@ const char* qsgd_status_string(int status) {
   switch (status) {
     case QSGD_OK: return "ok";
     case QSGD_ERR_NULL: return "a required pointer is null";
-    case QSGD_ERR_SIZE: return "n must be positive";
+    case QSGD_ERR_SIZE: return "n must lie in [1, 2^32]";
     case QSGD_ERR_BUCKET: return "bucket must be a multiple of 32 in [32, 4096]";
     case QSGD_ERR_LEVELS: return "s must lie in [1, 255]";
     case QSGD_ERR_ALIGN: return "pointer not 16-byte aligned";
@@ -351,6 +351,10 @@ const char* qsgd_status_string(int status) {
     default: return status > 0 ? cudaGetErrorString((cudaError_t)status) : "unknown status";
   }
 }
+
+void qsgd_test_set_wait_polls(uint32_t polls) { set_quantize_poll_limit(polls); }
+
+uint32_t qsgd_test_default_wait_polls(void) { return default_quantize_poll_limit(); }
 
 uint64_t qsgd_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -110,15 +110,11 @@ __global__ void __launch_bounds__(kThreads) sgd_step_kernel(float* __restrict__ 
 
 template <int LB, bool FUSED, bool SINGLE>
 int launch_one(const DecodeParams& p, cudaStream_t stream) {
-  static int sms = 0, occ = 0;
+  static KernelSite site;
   auto kern = decode_fixed_kernel<LB, FUSED, SINGLE>;
-  if (sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, 0);
-    if (occ < 1) occ = 1;
-  }
+  int sms = 0, occ = 0;
+  const int st = site.lookup(kern, kThreads, 0, &sms, &occ);
+  if (st) return st;
   const uint64_t want = (p.chunks + kWarps - 1) / kWarps;
   const uint64_t cap = (uint64_t)sms * occ;
   const uint32_t grid = (uint32_t)(want < cap ? want : cap);

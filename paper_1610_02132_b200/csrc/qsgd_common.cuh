@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/qsgd.h"
 
 namespace qsgd {
@@ -151,6 +153,47 @@ enum KernelId {
   kKernQuantize = 0, kKernQuantizeTail, kKernDecodeFixed, kKernSgdStep, kKernEliasLength,
   kKernEliasScatter, kKernDecodeElias, kKernDecodeEliasSparse, kKernRawGather, kKernRawDecode, kKernCount
 };
+
+// Launch facts of one kernel that belong to a device, not to the process: the opt-in to more than
+// 48 KB of dynamic shared memory, the SM count and the resident CTAs per SM. Looked up once per
+// device, with that device current, under a lock; one instance per kernel (a function-local static).
+constexpr int kMaxDevices = 64;
+
+struct KernelSite {
+  std::mutex mu;
+  bool ready[kMaxDevices] = {};
+  int sms[kMaxDevices] = {};
+  int occ[kMaxDevices] = {};
+
+  template <class Kernel>
+  int lookup(Kernel kern, int threads, size_t smem, int* sms_out, int* occ_out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return (int)e;
+    if (dev < 0 || dev >= kMaxDevices) return (int)cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!ready[dev]) {
+      e = cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev);
+      if (e != cudaSuccess) return (int)e;
+      if (smem > 48 * 1024) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return (int)e;
+      }
+      int o = 0;
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o, kern, threads, smem);
+      if (e != cudaSuccess) return (int)e;
+      occ[dev] = o > 0 ? o : 1;
+      ready[dev] = true;
+    }
+    *sms_out = sms[dev];
+    *occ_out = occ[dev];
+    return 0;
+  }
+};
+
+// Test hook: bound (in polls) of the waits inside the streaming encoder's main loop.
+void set_quantize_poll_limit(uint32_t polls);
+uint32_t default_quantize_poll_limit();
 
 struct ScopedKernel {
   ScopedKernel(KernelId id, cudaStream_t stream);

@@ -1,16 +1,27 @@
 // Encode, fixed-width path: bucket scale + Philox stochastic rounding + bit packing in one pass
 // over the gradient (Section 3.1, Eq. 2; Section 4 bucketing / max-norm; Section 5 bit widths).
 //
-// Main kernel (bucket size a power of two): persistent CTAs walk tiles of 4096 coordinates.
-// Tiles arrive in shared memory through a ring of 1-D TMA bulk copies (cp.async.bulk +
-// mbarrier), so no thread spends instructions on loads. A thread owns 16 consecutive
-// coordinates: it pulls them into registers once, the bucket scale is reduced with shuffles
-// (plus one shared-memory exchange when a bucket spans several warps), and the same registers
-// are then quantized, so the gradient is read from HBM exactly once. The arithmetic is written
-// to keep the instruction count per coordinate low, because at HBM speed this kernel has only
-// about 25 issue slots per coordinate:
-//   * the uniform u = m * 2^-24 (m = top 24 Philox bits) enters as fma(m, 2^-24, t), which
-//     rounds exactly like t + u because m * 2^-24 is exact;
+// Two streaming kernels for power-of-two bucket sizes, both persistent and fed by 1-D TMA bulk
+// copies (cp.async.bulk + mbarrier), so no thread spends instructions on global loads:
+//   * quantize_warp_kernel (d <= 512, no bucket map): every warp runs its own pipeline over
+//     chunks of 512 coordinates (whole buckets) with a private ring of shared-memory stages that
+//     its lane 0 refills as soon as the warp has taken a stage into registers. No CTA-wide
+//     barrier and no separate "empty" barrier exist, and every decision is warp-uniform.
+//   * quantize_pow2_kernel (d >= 1024, or buckets fetched through a bucket map): the CTA walks
+//     tiles of 4096 coordinates through a shared ring; scales of buckets that span several
+//     warps meet in shared memory.
+// A thread owns 16 consecutive coordinates: it pulls them into registers once, the bucket scale
+// is reduced with shuffles, and the same registers are then quantized, so the gradient is read
+// from HBM exactly once. The kernels are bound by the integer (ALU) and multiply (FMA-heavy)
+// pipes, which Philox alone loads with 2 + 2 instructions per round; everything else is written
+// to stay off those two pipes where it can:
+//   * the uniform u = m * 2^-24 (m = top 24 Philox bits) needs no integer-to-float conversion:
+//     the bit pattern m read as an fp32 is the subnormal (or smallest-normal) number m * 2^-149,
+//     and fma(that, 2^125, t) has the exact product m * 2^-24 and rounds once, exactly like
+//     t + u (subnormal operands are not flushed: the library is compiled without -ftz);
+//   * with the 2-norm, a level can exceed s only at a coordinate that holds nearly all of its
+//     bucket's norm; a warp checks that once per chunk and skips the per-coordinate clamp
+//     otherwise;
 //   * floor(c) is the round-down add c + 2^23, whose mantissa then holds the integer;
 //   * level fields are packed by Horner multiply-adds on those raw float bits, the constant
 //     exponent bits being removed once per word;
@@ -18,6 +29,8 @@
 //     sign word with a funnel shift.
 // A generic kernel (any bucket size that is a multiple of 32) keeps the simple structure.
 #include <float.h>
+
+#include <atomic>
 
 #include "qsgd_common.cuh"
 
@@ -79,9 +92,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after ~2^22 polls and reports it instead of spinning forever.
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
-  for (uint32_t it = 0; it < (1u << 22); ++it)
+// Bounded wait: gives up after `polls` tries and reports it instead of spinning forever.
+constexpr uint32_t kDrainPolls = 1u << 22;   // bound of the waits that drain copies in flight
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t polls) {
+  for (uint32_t it = 0; it < polls; ++it)
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
@@ -139,20 +153,36 @@ __device__ __forceinline__ uint4 philox_q(uint32_t q, const PhiloxConsts& pc) {
   return make_uint4(c0, c1, c2, c3);
 }
 
+// The uniforms of the 16 coordinates of one thread (Philox blocks q0 .. q0 + 3) as fp32 bit
+// patterns m = word >> 8 (see quantize_one).
+__device__ __forceinline__ void philox_uniforms16(uint32_t q0, const PhiloxConsts& pc, float (&um)[16]) {
+#pragma unroll
+  for (int b = 0; b < 4; ++b) {
+    const uint4 w = philox_q(q0 + b, pc);
+    um[4 * b] = __uint_as_float(w.x >> 8);
+    um[4 * b + 1] = __uint_as_float(w.y >> 8);
+    um[4 * b + 2] = __uint_as_float(w.z >> 8);
+    um[4 * b + 3] = __uint_as_float(w.w >> 8);
+  }
+}
+
 constexpr float kTwo23 = 8388608.0f;
 constexpr uint32_t kTwo23Bits = 0x4B000000u;
 
-// One coordinate. Returns the raw bits of 2^23 + level (level clamped to s); pushes the sign
-// bit into `sw`.
+constexpr float kTwo125 = 4.253529586511730793292182592897102643e+37f;
+
+// One coordinate. Returns the raw bits of 2^23 + level (level clamped to s when CLAMP); pushes the
+// sign bit into `sw`. `um` is the bit pattern m = top 24 Philox bits read as an fp32, i.e. m * 2^-149.
 // RAW_SIGN: push the sign bit of v as it is; the caller clears the signs of zero levels afterwards
 // with a mask derived from the packed level words (cheaper than two more operations per coordinate
 // when a word holds many fields).
-template <bool RAW_SIGN>
-__device__ __forceinline__ uint32_t quantize_one(float v, float r, float sf, float cap, uint32_t rnd,
+template <bool RAW_SIGN, bool CLAMP>
+__device__ __forceinline__ uint32_t quantize_one(float v, float r, float sf, float cap, float um,
                                                  uint32_t& sw) {
   const float t = __fmul_rn(__fmul_rn(sf, fabsf(v)), r);
-  const float c = fma_rn(__uint2float_rn(rnd >> 8), 5.9604644775390625e-08f, t);
-  const float fl = fminf(__fadd_rd(c, kTwo23), cap);       // 2^23 + min(floor(c), s)
+  const float c = fma_rn(um, kTwo125, t);                    // t + m * 2^-24, one rounding
+  float fl = __fadd_rd(c, kTwo23);                           // 2^23 + floor(c)
+  if (CLAMP) fl = fminf(fl, cap);                            // 2^23 + min(floor(c), s)
   if (RAW_SIGN) {
     sw = __funnelshift_l(__float_as_uint(v), sw, 1);
   } else {
@@ -161,6 +191,40 @@ __device__ __forceinline__ uint32_t quantize_one(float v, float r, float sf, flo
     sw = __funnelshift_l(__float_as_uint(sv), sw, 1);
   }
   return __float_as_uint(fl);
+}
+
+// Rounds and packs the 16 coordinates of a thread, highest first: level fields by Horner
+// multiply-adds on the raw float bits (the constant exponent bits are removed once per word),
+// sign bits by funnel shifts; signs of zero levels are cleared at the end.
+template <int LB, bool CLAMP>
+__device__ __forceinline__ void quantize16(const float (&v)[16], const float (&um)[16], float r, float sf,
+                                           float cap, uint32_t (&lw)[4], uint32_t& sw) {
+  sw = 0;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) lw[j] = 0u;                 // LB = 8: 4 words; 4: 2; 2: 1; 1: half
+#pragma unroll
+  for (int c4 = 3; c4 >= 0; --c4) {
+#pragma unroll
+    for (int e = 3; e >= 0; --e) {
+      const uint32_t bits = quantize_one<LB != 8, CLAMP>(v[4 * c4 + e], r, sf, cap, um[4 * c4 + e], sw);
+      if (LB == 8) lw[c4] = lw[c4] * 256u + bits;
+      else if (LB == 4) lw[c4 >> 1] = lw[c4 >> 1] * 16u + bits;
+      else if (LB == 2) lw[0] = lw[0] * 4u + bits;
+      else lw[0] = lw[0] * 2u + bits;
+    }
+  }
+  // remove the exponent bits that rode along: sum over the fields of 0x4B000000 << (LB * e)
+  if (LB == 8) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) lw[j] -= kTwo23Bits * 0x01010101u;
+  } else if (LB == 4) {
+    lw[0] -= kTwo23Bits * 0x11111111u;
+    lw[1] -= kTwo23Bits * 0x11111111u;
+  } else if (LB == 2) {
+    lw[0] -= kTwo23Bits * 0x55555555u;
+  } else {
+    lw[0] = (lw[0] - kTwo23Bits * 0xFFFFu) & 0xFFFFu;
+  }
 }
 
 // Bit e of the result is set iff level field e of the 16 coordinates packed in lw is nonzero.
@@ -184,6 +248,29 @@ __device__ __forceinline__ uint32_t nonzero_fields16(const uint32_t (&lw)[4]) {
     m |= ((y | (y >> 12)) & 0xFFu) << (8 * h);
   }
   return m;
+}
+
+// Stores the sign and level words of the 16 coordinates of every lane of a warp; `c` is the index
+// of the warp's chunk of 512 coordinates (complete chunks only: no bounds to check).
+template <int LB>
+__device__ __forceinline__ void store_chunk(uint32_t* sign_out, uint32_t* level_out, uint32_t c, uint32_t lane,
+                                            uint32_t sw, const uint32_t (&lw)[4]) {
+  {
+    uint32_t w = (sw & 0xFFFFu) << (16 * (lane & 1));
+    w |= __shfl_xor_sync(0xffffffffu, w, 1);
+    if ((lane & 1) == 0) sign_out[c * 16u + (lane >> 1)] = w;
+  }
+  if (LB == 8) {
+    *reinterpret_cast<uint4*>(level_out + ((size_t)c * 128u + lane * 4u)) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+  } else if (LB == 4) {
+    *reinterpret_cast<uint2*>(level_out + ((size_t)c * 64u + lane * 2u)) = make_uint2(lw[0], lw[1]);
+  } else if (LB == 2) {
+    level_out[(size_t)c * 32u + lane] = lw[0];
+  } else {
+    uint32_t w = lw[0] << (16 * (lane & 1));
+    w |= __shfl_xor_sync(0xffffffffu, w, 1);
+    if ((lane & 1) == 0) level_out[c * 16u + (lane >> 1)] = w;
+  }
 }
 
 constexpr int kStages = 3;
@@ -210,6 +297,7 @@ struct FastParams {
   uint32_t* clear_word;     // optional word set to zero by CTA 0
   PhiloxConsts pc;
   uint32_t main_ctas;       // CTAs that stream complete tiles
+  uint32_t poll_limit;      // bound of the main-loop waits (the final drain keeps its own bound)
   BucketMap map;            // per-tensor policy: where each bucket lives in g (quads set), or no map
   QuantizeParams tail;      // parameters of the extra CTA (used when gridDim.x > main_ctas)
 };
@@ -310,7 +398,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
   uint32_t stage = 0, phase = 0, it = 0;
   for (uint32_t t = blockIdx.x; t < p.full_tiles; t += grid, ++it) {
     const float* tile = sm.tile[stage];
-    const bool arrived = mbar_wait_bounded(&sm.full[stage], phase);
+    const bool arrived = mbar_wait_bounded(&sm.full[stage], phase, p.poll_limit);
 
     // ---- registers <- 16 consecutive coordinates; partial of the scale ----------------------
     float v[16];
@@ -341,11 +429,13 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
     // thread refills the stage that was released one iteration ago (its arrivals are long in) ----
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.empty[stage]);
+    // a wait that ran out ends the loop; the decision is taken per CTA (CROSS: the scales meet
+    // in shared memory) or per warp (its lanes meet in shuffles), never per lane
     int flags = arrived ? 0 : 1;
     if (CROSS) flags = __syncthreads_or(flags | (shaky ? 2 : 0));
-    else if (MAPPED) flags = __any_sync(0xffffffffu, flags != 0) ? 1 : 0;      // the producer warp must leave together
+    else flags = __any_sync(0xffffffffu, flags != 0) ? 1 : 0;
     if (flags & 1) {
-      atomicOr(p.status, QSGD_DEV_TIMEOUT);
+      if (lane == 0) atomicOr(p.status, QSGD_DEV_TIMEOUT);
       break;
     }
     if (!MAPPED) {                                                        // ordinary case: thread 0 produces
@@ -354,7 +444,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
         const uint32_t pphase = stage == 0 ? phase ^ 1 : phase;
         const uint32_t tn = t + (uint32_t)(kStages - 1) * grid;           // tile of iteration it - 1 + kStages
         if (tn < p.full_tiles) {
-          if (mbar_wait_bounded(&sm.empty[ps], pphase)) issue_tile<false>(p, sm.tile[ps], &sm.full[ps], tn, 0u);
+          if (mbar_wait_bounded(&sm.empty[ps], pphase, p.poll_limit)) issue_tile<false>(p, sm.tile[ps], &sm.full[ps], tn, 0u);
           else atomicOr(p.status, QSGD_DEV_TIMEOUT);
         }
       }
@@ -363,7 +453,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
       const uint32_t pphase = stage == 0 ? phase ^ 1 : phase;
       const uint32_t tn = t + (uint32_t)(kStages - 1) * grid;
       if (tn < p.full_tiles) {
-        const bool freed = __shfl_sync(0xffffffffu, lane == 0 ? (mbar_wait_bounded(&sm.empty[ps], pphase) ? 1 : 0) : 0, 0) != 0;
+        const bool freed = __shfl_sync(0xffffffffu, lane == 0 ? (mbar_wait_bounded(&sm.empty[ps], pphase, p.poll_limit) ? 1 : 0) : 0, 0) != 0;
         __syncwarp();                                                     // lane 0's acquire covers the warp
         if (freed) issue_tile<true>(p, sm.tile[ps], &sm.full[ps], tn, lane);
         else if (lane == 0) atomicOr(p.status, QSGD_DEV_TIMEOUT);
@@ -415,55 +505,14 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
     const float r = A > 0.f ? __frcp_rn(A) : 0.f;
     if (leader) p.A_out[(t << buckets_per_tile_log2) + my_bucket] = A;
 
-    // ---- stochastic rounding and packing, highest coordinate first --------------------------
-    const uint32_t q0 = t * (kTile / 4) + tid * 4;     // Philox block of v[0..3]
-    uint32_t sw = 0;
-    uint32_t lw[4] = {0u, 0u, 0u, 0u};                 // LB = 8: 4 words; 4: 2; 2: 1; 1: half
-#pragma unroll
-    for (int c4 = 3; c4 >= 0; --c4) {
-      const uint4 rnd = philox_q(q0 + c4, p.pc);
-      const uint32_t rr[4] = {rnd.x, rnd.y, rnd.z, rnd.w};
-#pragma unroll
-      for (int e = 3; e >= 0; --e) {
-        const uint32_t bits = quantize_one<LB != 8>(v[4 * c4 + e], r, sf, cap, rr[e], sw);
-        if (LB == 8) lw[c4] = lw[c4] * 256u + bits;
-        else if (LB == 4) lw[c4 >> 1] = lw[c4 >> 1] * 16u + bits;
-        else if (LB == 2) lw[0] = lw[0] * 4u + bits;
-        else lw[0] = lw[0] * 2u + bits;
-      }
-    }
-    // remove the exponent bits that rode along: sum over the fields of 0x4B000000 << (LB * e)
-    if (LB == 8) {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) lw[j] -= kTwo23Bits * 0x01010101u;
-    } else if (LB == 4) {
-      lw[0] -= kTwo23Bits * 0x11111111u;
-      lw[1] -= kTwo23Bits * 0x11111111u;
-    } else if (LB == 2) {
-      lw[0] -= kTwo23Bits * 0x55555555u;
-    } else {
-      lw[0] = (lw[0] - kTwo23Bits * 0xFFFFu) & 0xFFFFu;
-    }
+    // ---- stochastic rounding and packing ----------------------------------------------------
+    float um[16];
+    philox_uniforms16(t * (kTile / 4) + tid * 4, p.pc, um);
+    uint32_t sw, lw[4];
+    quantize16<LB, true>(v, um, r, sf, cap, lw, sw);
     if (LB != 8) sw &= nonzero_fields16<LB>(lw);          // canonical sign: 0 where the level is 0
 
-    // ---- stores (full tiles only: no bounds to check) -----------------------------------------
-    {
-      uint32_t w = (sw & 0xFFFFu) << (16 * (lane & 1));
-      w |= __shfl_xor_sync(0xffffffffu, w, 1);
-      if ((lane & 1) == 0) p.sign_out[t * (kTile / 32) + (tid >> 1)] = w;
-    }
-    if (LB == 8) {
-      *reinterpret_cast<uint4*>(p.level_out + (size_t)(t * (kTile / 4) + tid * 4)) =
-          make_uint4(lw[0], lw[1], lw[2], lw[3]);
-    } else if (LB == 4) {
-      *reinterpret_cast<uint2*>(p.level_out + (size_t)(t * (kTile / 8) + tid * 2)) = make_uint2(lw[0], lw[1]);
-    } else if (LB == 2) {
-      p.level_out[t * (kTile / 16) + tid] = lw[0];
-    } else {
-      uint32_t w = lw[0] << (16 * (lane & 1));
-      w |= __shfl_xor_sync(0xffffffffu, w, 1);
-      if ((lane & 1) == 0) p.level_out[t * (kTile / 32) + (tid >> 1)] = w;
-    }
+    store_chunk<LB>(p.sign_out, p.level_out, t * (kTile / 512) + warp, lane, sw, lw);
     if (++stage == kStages) { stage = 0; phase ^= 1; }
   }
 
@@ -473,7 +522,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
     for (uint32_t j = 0; j < (uint32_t)kStages; ++j) {
       const uint32_t itj = it + j;
       const uint64_t t = (uint64_t)blockIdx.x + (uint64_t)itj * grid;
-      if (t < p.full_tiles) mbar_wait_bounded(&sm.full[itj % kStages], (itj / kStages) & 1);
+      if (t < p.full_tiles) mbar_wait_bounded(&sm.full[itj % kStages], (itj / kStages) & 1, kDrainPolls);
     }
   }
 }
@@ -662,6 +711,163 @@ __device__ __forceinline__ void quantize_generic_tile(const QuantizeParams& p, u
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Per-warp streaming kernel: d <= 512 (a bucket never leaves a warp), no bucket map.
+// Warp w of CTA b takes chunks b * 8 + w, + 8 * main_ctas, ... of 512 coordinates. Its ring of
+// kWarpStages stages is private: lane 0 arms a stage (expect-tx + bulk copy), all lanes wait on
+// the stage's barrier, pull their 16 values into registers, and after the shuffle reduction of
+// the scale (which cannot finish before every lane's values have arrived) lane 0 re-arms the
+// stage for the chunk kWarpStages rounds ahead. One optional extra CTA runs the ragged last
+// tile and the region padding through the generic tile code.
+// ---------------------------------------------------------------------------------------------
+constexpr int kWarpStages = 3;
+constexpr int kChunk = 512;
+
+struct __align__(16) WarpRings {
+  float chunk[kThreads / 32][kWarpStages][kChunk];
+  uint64_t full[kThreads / 32][kWarpStages];
+};
+
+template <int LB, int NORM>
+__global__ void __launch_bounds__(kThreads, 4)
+quantize_warp_kernel(const __grid_constant__ FastParams p) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  WarpRings& sm = *reinterpret_cast<WarpRings*>(smem_raw);
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t grid = p.main_ctas;
+  if (blockIdx.x >= grid) {                     // the extra CTA: ragged tail + padding
+    float* scratch = &sm.chunk[0][0][0];
+    quantize_generic_tile<LB, NORM, false>(p.tail, 0u, 1u, scratch, scratch + kTile, scratch + kTile + 1024);
+    return;
+  }
+  const uint32_t chunks = p.full_tiles * (kTile / kChunk), stride = grid * (kThreads / 32);
+  uint32_t c = blockIdx.x * (kThreads / 32) + warp;
+  if (lane == 0) {
+    for (int s = 0; s < kWarpStages; ++s) mbar_init(&sm.full[warp][s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (tid == 0 && blockIdx.x == 0 && p.info) {
+      p.info[0] = 8 * p.total_bytes; p.info[1] = 0; p.info[2] = p.total_bytes; p.info[3] = 0;
+    }
+    if (tid == 0 && blockIdx.x == 0 && p.clear_word) *p.clear_word = 0u;
+    for (int s = 0; s < kWarpStages; ++s) {
+      const uint32_t cs = c + (uint32_t)s * stride;
+      if (cs < chunks) {
+        mbar_expect_tx(&sm.full[warp][s], kChunk * 4);
+        bulk_load(sm.chunk[warp][s], p.g + (size_t)cs * kChunk, kChunk * 4, &sm.full[warp][s]);
+      }
+    }
+  }
+  __syncwarp();
+
+  const float sf = (float)p.s;
+  const float cap = kTwo23 + sf;
+  const uint32_t team_w = 1u << (p.log2d - 4);                   // lanes per bucket (2 .. 32)
+  const bool leader = (lane & (team_w - 1u)) == 0;
+  const uint32_t my_bucket = (lane * 16u) >> p.log2d;            // bucket of this lane in a chunk
+  const uint32_t buckets_per_chunk_log2 = 9u - p.log2d;
+
+  uint32_t stage = 0, phase = 0;
+  for (; c < chunks; c += stride) {
+    const float* src = sm.chunk[warp][stage];
+    const bool arrived = mbar_wait_bounded(&sm.full[warp][stage], phase, p.poll_limit);
+    if (!__all_sync(0xffffffffu, arrived)) {                       // the warp leaves together
+      if (lane == 0) atomicOr(p.status, QSGD_DEV_TIMEOUT);
+      break;
+    }
+
+    // ---- registers <- 16 consecutive coordinates; the uniforms; partial of the scale ---------
+    float v[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float4 a = *reinterpret_cast<const float4*>(src + lane * 16 + j * 4);
+      v[4 * j] = a.x; v[4 * j + 1] = a.y; v[4 * j + 2] = a.z; v[4 * j + 3] = a.w;
+    }
+    float um[16];
+    philox_uniforms16(c * (kChunk / 4) + lane * 4, p.pc, um);
+    float part = 0.f;
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      if (NORM == QSGD_NORM_L2) part = fmaf(v[e], v[e], part);
+      else part = fmaxf(part, fabsf(v[e]));
+    }
+    const float mine = part;                                       // this thread's share of the scale
+    if (team_w == 32u) {
+#pragma unroll
+      for (uint32_t o = 16; o > 0; o >>= 1) {
+        const float q = __shfl_xor_sync(0xffffffffu, part, o);
+        part = (NORM == QSGD_NORM_L2) ? part + q : fmaxf(part, q);
+      }
+    } else {
+#pragma unroll
+      for (uint32_t o = 16; o > 0; o >>= 1) {
+        const float q = __shfl_xor_sync(0xffffffffu, part, o);
+        const float merged = (NORM == QSGD_NORM_L2) ? part + q : fmaxf(part, q);
+        part = (o < team_w) ? merged : part;
+      }
+    }
+
+    // ---- the stage is in registers: refill it with the chunk kWarpStages rounds ahead --------
+    __syncwarp();
+    if (lane == 0) {
+      const uint32_t cn = c + (uint32_t)kWarpStages * stride;
+      if (cn < chunks) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // our reads before the copy's writes
+        mbar_expect_tx(&sm.full[warp][stage], kChunk * 4);
+        bulk_load(sm.chunk[warp][stage], p.g + (size_t)cn * kChunk, kChunk * 4, &sm.full[warp][stage]);
+      }
+    }
+
+    // ---- scale ---------------------------------------------------------------------------------
+    // 2-norm: an fp32 sum of squares outside [8e-28, 1e30] may have lost bits to underflow or
+    // overflowed; such buckets are redone in fp64 (rare, the warp branches together)
+    float A;
+    bool shaky = false;
+    if (NORM == QSGD_NORM_L2) {
+      shaky = !(part >= 8.0e-28f && part <= 1.0e30f) && part != 0.f;
+      A = __fsqrt_rn(part);
+      if (__any_sync(0xffffffffu, shaky)) {
+        double wide = 0.0;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) wide = fma((double)v[e], (double)v[e], wide);
+#pragma unroll
+        for (uint32_t o = 16; o > 0; o >>= 1) {
+          const double q = __shfl_xor_sync(0xffffffffu, wide, o);
+          wide = (o < team_w) ? wide + q : wide;
+        }
+        if (shaky) A = __double2float_rn(sqrt(wide));
+      }
+    } else {
+      A = part;
+    }
+    if (!(A >= FLT_MIN)) A = 0.f;                      // zero bucket: Q(0) = 0
+    const float r = A > 0.f ? __frcp_rn(A) : 0.f;
+    if (leader) p.A_out[(c << buckets_per_chunk_log2) + my_bucket] = A;
+
+    // ---- stochastic rounding and packing -------------------------------------------------------
+    // floor(t + u) can pass s only where t = (s |v|) / A reaches s, i.e. |v| is A up to rounding.
+    // With the 2-norm that needs one coordinate to hold (nearly) all of the bucket's sum of
+    // squares; a thread whose 16 squares stay under 0.9 of the sum holds no such coordinate, and
+    // a warp of such threads rounds without the clamp. (Not so for the max-norm, where the
+    // largest coordinate always has |v| = A.)
+    uint32_t sw, lw[4];
+    bool clamp = true;
+    if (NORM == QSGD_NORM_L2) clamp = __any_sync(0xffffffffu, shaky || !(mine <= 0.9f * part));
+    if (clamp) quantize16<LB, true>(v, um, r, sf, cap, lw, sw);
+    else quantize16<LB, false>(v, um, r, sf, cap, lw, sw);
+    if (LB != 8) sw &= nonzero_fields16<LB>(lw);          // canonical sign: 0 where the level is 0
+    store_chunk<LB>(p.sign_out, p.level_out, c, lane, sw, lw);
+    if (++stage == kWarpStages) { stage = 0; phase ^= 1; }
+  }
+
+  // Leave no bulk copy in flight: a warp that stopped early waits (bounded) for the stages it armed.
+  if (lane == 0 && c < chunks) {
+    for (uint32_t j = 0; j < (uint32_t)kWarpStages; ++j) {
+      if (c + j * stride < chunks) mbar_wait_bounded(&sm.full[warp][stage], phase, kDrainPolls);
+      if (++stage == kWarpStages) { stage = 0; phase ^= 1; }
+    }
+  }
+}
+
 template <int LB, int NORM, bool MAPPED>
 __global__ void __launch_bounds__(kThreads) quantize_generic_kernel(const QuantizeParams p) {
   __shared__ __align__(16) float tile[kTile];
@@ -687,26 +893,25 @@ PhiloxConsts make_philox_consts(uint64_t seed, uint32_t step, uint32_t worker) {
   return pc;
 }
 
+std::atomic<uint32_t> g_poll_limit{kDrainPolls};
+
 template <int LB, int NORM, bool CROSS, bool MAPPED>
 int launch_fast(FastParams& fp, bool with_tail, cudaStream_t stream) {
-  static int ctas_per_sm = 0, sms = 0;
-  auto kern = quantize_pow2_kernel<LB, NORM, CROSS, MAPPED>;
-  const size_t smem = sizeof(TileSmem) + 128;
-  if (ctas_per_sm == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return (int)e;
-    int occ = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, kThreads, smem);
-    if (e != cudaSuccess) return (int)e;
-    ctas_per_sm = occ > 0 ? occ : 1;
-  }
+  constexpr bool kPerWarp = !CROSS && !MAPPED;
+  static KernelSite site;
+  const size_t smem = (kPerWarp ? sizeof(WarpRings) : sizeof(TileSmem)) + 128;
+  int sms = 0, ctas_per_sm = 0;
+  int st;
+  if (kPerWarp) st = site.lookup(quantize_warp_kernel<LB, NORM>, kThreads, smem, &sms, &ctas_per_sm);
+  else st = site.lookup(quantize_pow2_kernel<LB, NORM, CROSS, MAPPED>, kThreads, smem, &sms, &ctas_per_sm);
+  if (st) return st;
   const uint32_t cap = (uint32_t)(sms * ctas_per_sm);
   fp.main_ctas = fp.full_tiles < cap ? fp.full_tiles : cap;
+  fp.poll_limit = g_poll_limit.load(std::memory_order_relaxed);
   ScopedKernel sk(kKernQuantize, stream);
-  kern<<<fp.main_ctas + (with_tail ? 1u : 0u), kThreads, smem, stream>>>(fp);
+  const uint32_t grid = fp.main_ctas + (with_tail ? 1u : 0u);
+  if (kPerWarp) quantize_warp_kernel<LB, NORM><<<grid, kThreads, smem, stream>>>(fp);
+  else quantize_pow2_kernel<LB, NORM, CROSS, MAPPED><<<grid, kThreads, smem, stream>>>(fp);
   return (int)cudaGetLastError();
 }
 
@@ -788,5 +993,8 @@ int launch_quantize_fixed(const float* g, uint64_t n, uint32_t d, uint32_t s, in
     default: return launch_lb<8>(p, norm_kind, seed, stream);
   }
 }
+
+void set_quantize_poll_limit(uint32_t polls) { g_poll_limit.store(polls, std::memory_order_relaxed); }
+uint32_t default_quantize_poll_limit() { return kDrainPolls; }
 
 }  // namespace qsgd

@@ -48,5 +48,9 @@ def test_host_side_queries_and_validation():
     assert L.qsgd_encode(16, 10, 512, 15, 5, 0, 0, 0, 0, 16, 0, 16, None, 16, None) == -8
     assert L.qsgd_encode(24, 10, 512, 15, 0, 0, 0, 0, 0, 16, 0, 16, None, 16, None) == -5
     assert L.qsgd_encode(16, 10, 512, 15, 0, 0, 0, 0, 0, 16, 8, 16, None, 16, None) == -6
+    # n beyond 2^32 coordinates is refused by every shape check (16 GiB of gradient per call)
+    assert L.qsgd_encode(16, 2 ** 32 + 1, 512, 15, 0, 0, 0, 0, 0, 16, 0, 16, None, 16, None) == -2
+    assert Q.qsgd_message_capacity(2 ** 32 + 1, 512, 15, 0) == 0
+    assert Q.qsgd_message_capacity(2 ** 32, 512, 15, 0) > 0
     assert L.qsgd_status_string(-3).decode().startswith("bucket")
     assert Q.qsgd_launch_count() == 0

@@ -71,6 +71,31 @@ def test_degenerate_buckets(code_kind):
             assert np.all(acc[1536:] == 3.0)
 
 
+@pytest.mark.parametrize("d", [128, 512, 4096])
+@pytest.mark.parametrize("shape", ["equal", "ascending", "descending", "one_large"])
+def test_two_norm_tolerance_on_adversarial_inputs(d, shape):
+    """fp32 accumulation of the sum of squares must stay within 1e-6 of the exact norm also when the
+    rounding errors cannot cancel: all magnitudes equal (every partial sum rounds the same way),
+    magnitudes sorted (small terms meet a large running sum, or the reverse), one dominant value."""
+    n = 6 * 4096 + 2 * d + 40
+    rng = np.random.default_rng(d)
+    if shape == "equal":
+        g = np.full(n, 0.3337, dtype=np.float32) * rng.choice([-1.0, 1.0], n).astype(np.float32)
+    elif shape == "one_large":
+        g = np.full(n, 1e-3, dtype=np.float32)
+        g[::d] = 0.777
+    else:
+        g = (1.0 + 1e-3 * np.arange(n, dtype=np.float64) % d).astype(np.float32)
+        g = np.sort(g.reshape(-1)[: n]) if shape == "ascending" else np.sort(g)[::-1].copy()
+        g = (g * (1.0 + (np.arange(n) % d) / d)).astype(np.float32)
+        if shape == "descending":
+            g = g[::-1].copy()
+    for s in (1, 15):
+        m, info = encode_parity(np.ascontiguousarray(g, dtype=np.float32), d, s, O.NORM_L2, O.CODE_FIXED,
+                                seed=3, step=1, worker=0)
+        decode_parity([m], [info], n, d, s, O.CODE_FIXED)
+
+
 def test_many_peers_and_philox_keying():
     n, d, s = 20000, 512, 15
     g = make(n, "gauss", 5)
