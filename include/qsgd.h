@@ -132,26 +132,58 @@ int qsgd_encode(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int nor
  * acc_i = ((+0 + g^0_i) + g^1_i) + ... in ascending k, where g^k_i = +-(A * (level / s)).
  *   msgs    host array of K device pointers to messages (16-byte aligned)
  *   tables  host array of K device pointers to the offset tables (Elias kinds; msgs[k] +
- *           out_bits[1]); NULL for fixed-width. A payload must be readable for 16 bytes past
- *           its padded length (true when its table follows it, as Encode writes it). With the
- *           table directly behind the payload the library reads the payload sizes off the
- *           pointers and chooses between its decoders on the host; with tables kept elsewhere
- *           it decides on the device (two launches, one of which returns at once). Results
- *           are the same either way.
+ *           out_bits[1]); NULL for fixed-width. With the table directly behind the payload the
+ *           library reads the payload sizes off the pointers and chooses between its decoders on
+ *           the host; with tables kept elsewhere it decides on the device (two launches, one of
+ *           which returns at once). Results are the same either way.
+ *   payload_bytes  host array of K payload lengths in bytes (the padded payload, = out_bits[1]
+ *           of each message), or NULL. The decoders read no payload bit at or beyond
+ *           8 * payload_bytes[k]: a table whose last entry claims more is refused with
+ *           QSGD_DEV_TABLE before any payload read. With NULL the bound is the table's own address
+ *           when the table lies behind the payload (as Encode writes it); for a table kept
+ *           elsewhere there is then no bound and the caller vouches for the table. In every case a
+ *           payload must be readable for 16 bytes past its padded length (true when its table
+ *           follows it): the bit window prefetches two words ahead.
  *   acc     n fp32 values, overwritten
  */
-int qsgd_decode_accumulate(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
-                           uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* acc,
-                           uint32_t* status_dev, qsgd_stream_t stream);
+int qsgd_decode_accumulate(const void* const* msgs, const uint64_t* const* tables,
+                           const uint64_t* payload_bytes, uint32_t K, uint64_t n, uint32_t bucket,
+                           uint32_t s, int code_kind, float* acc, uint32_t* status_dev,
+                           qsgd_stream_t stream);
 
 /* SGD step (Algorithm 1, last line): c = eta / K once; x_i <- x_i - c * acc_i. */
 int qsgd_sgd_step(float* x, const float* acc, float eta, uint32_t K, uint64_t n,
                   qsgd_stream_t stream);
 
 /* Decode, sum and step in one pass over x; bit-identical to the two calls above. */
-int qsgd_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
-                         uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* x,
-                         float eta, uint32_t* status_dev, qsgd_stream_t stream);
+int qsgd_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables,
+                         const uint64_t* payload_bytes, uint32_t K, uint64_t n, uint32_t bucket,
+                         uint32_t s, int code_kind, float* x, float eta, uint32_t* status_dev,
+                         qsgd_stream_t stream);
+
+/*
+ * The same two calls for messages exactly as Encode left them (Algorithm 1, "receive M^l, decode"):
+ * a packaging that needs no host read-back between Encode and Decode. Where the offset table of an
+ * Elias message starts is known only on the device (out_bits[1], written by Encode on the stream);
+ * instead of table pointers the caller passes
+ *   infos      host array of K DEVICE pointers to the four out_bits words of each message (8-byte
+ *              aligned; for a received message: wherever its info words were put), and
+ *   msg_bytes  host array of K byte counts: how much of message buffer k may be read (its capacity
+ *              as allocated is fine).
+ * The kernels take table k at msgs[k] + infos[k][1]; that place must be 16-byte aligned with all
+ * 8 * (B + 1) table bytes inside msg_bytes[k], and infos[k][1] bounds the payload, else
+ * QSGD_DEV_TABLE is raised and nothing of that message is read. The choice among the Elias
+ * decoders is made on the device (two launches, one returns at once). For QSGD_CODE_FIXED infos
+ * and msg_bytes are ignored (may be NULL). Results are bit-identical to the calls above.
+ */
+int qsgd_decode_accumulate_packed(const void* const* msgs, const uint64_t* const* infos,
+                                  const uint64_t* msg_bytes, uint32_t K, uint64_t n, uint32_t bucket,
+                                  uint32_t s, int code_kind, float* acc, uint32_t* status_dev,
+                                  qsgd_stream_t stream);
+int qsgd_decode_sgd_step_packed(const void* const* msgs, const uint64_t* const* infos,
+                                const uint64_t* msg_bytes, uint32_t K, uint64_t n, uint32_t bucket,
+                                uint32_t s, int code_kind, float* x, float eta, uint32_t* status_dev,
+                                qsgd_stream_t stream);
 
 /* Text for a negative return code ("ok" for 0). Host pointer to a static string. */
 const char* qsgd_status_string(int status);
@@ -259,7 +291,8 @@ size_t qsgd_policy_workspace_bytes(const qsgd_policy* plan, uint32_t bucket, uin
  * Encode / Decode under the policy. Arguments as for qsgd_encode, qsgd_decode_accumulate and
  * qsgd_decode_sgd_step, with the plan in place of n; `plan` is a host pointer to a struct of device
  * pointers. msgs[k] points to the start of policy message k (its raw region), tables[k] to its
- * offset table (msgs[k] + out_bits[1]). acc (n floats) is overwritten at every coordinate; x is
+ * offset table (msgs[k] + out_bits[1]), payload_bytes[k] (optional, as for qsgd_decode_accumulate) is
+ * the padded payload length out_bits[1] - out_bits[3]. acc (n floats) is overwritten at every coordinate; x is
  * updated at every coordinate; fused and unfused results are equal bit for bit. Errors as for the
  * ordinary calls. Launches: the ordinary encode or decode kernels plus one small kernel for the
  * raw tensors.
@@ -268,12 +301,14 @@ int qsgd_policy_encode(const float* g, const qsgd_policy* plan, uint32_t bucket,
                        int code_kind, uint64_t seed, uint32_t step, uint32_t worker, void* out,
                        size_t out_capacity, uint64_t* out_bits, void* workspace, uint32_t* status_dev,
                        qsgd_stream_t stream);
-int qsgd_policy_decode_accumulate(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
-                                  const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind,
-                                  float* acc, uint32_t* status_dev, qsgd_stream_t stream);
-int qsgd_policy_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
-                                const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind,
-                                float* x, float eta, uint32_t* status_dev, qsgd_stream_t stream);
+int qsgd_policy_decode_accumulate(const void* const* msgs, const uint64_t* const* tables,
+                                  const uint64_t* payload_bytes, uint32_t K, const qsgd_policy* plan,
+                                  uint32_t bucket, uint32_t s, int code_kind, float* acc,
+                                  uint32_t* status_dev, qsgd_stream_t stream);
+int qsgd_policy_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables,
+                                const uint64_t* payload_bytes, uint32_t K, const qsgd_policy* plan,
+                                uint32_t bucket, uint32_t s, int code_kind, float* x, float eta,
+                                uint32_t* status_dev, qsgd_stream_t stream);
 
 /*
  * Per-kernel timing (measurement aid; the paper has no counterpart). While enabled, every

@@ -2,7 +2,7 @@
 (include/qsgd.h), with a thin ctypes binding. The library is loaded on first use."""
 from .binding import (CODE_ELIAS, CODE_ELIAS_DENSE, CODE_FIXED, NORM_L2, NORM_MAX,  # noqa: F401
                       QsgdError, encode_alloc, new_status, qsgd_decode_accumulate,
-                      qsgd_decode_sgd_step, qsgd_encode, qsgd_encode_elias_static, qsgd_fixed_layout, qsgd_launch_count,
+                      qsgd_decode_sgd_step, qsgd_decode_accumulate_packed, qsgd_decode_sgd_step_packed, qsgd_encode, qsgd_encode_elias_static, qsgd_fixed_layout, qsgd_launch_count,
                       qsgd_message_capacity, qsgd_profile_collect, qsgd_profile_enable,
                       qsgd_sgd_step, qsgd_static_scratch_bytes, qsgd_workspace_bytes,
                       Policy, qsgd_policy_decode_accumulate, qsgd_policy_decode_sgd_step,

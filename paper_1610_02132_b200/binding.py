@@ -17,6 +17,7 @@ DEV_CAPACITY, DEV_OVERRUN, DEV_POSITION, DEV_LEVEL, DEV_TABLE, DEV_TIMEOUT = 1, 
 
 EXPORTS = ["qsgd_message_capacity", "qsgd_workspace_bytes", "qsgd_fixed_layout", "qsgd_encode",
            "qsgd_decode_accumulate", "qsgd_sgd_step", "qsgd_decode_sgd_step",
+           "qsgd_decode_accumulate_packed", "qsgd_decode_sgd_step_packed",
            "qsgd_status_string", "qsgd_launch_count", "qsgd_profile_enable",
            "qsgd_profile_kernel_count", "qsgd_profile_kernel_name", "qsgd_profile_collect",
            "qsgd_static_scratch_bytes", "qsgd_encode_elias_static",
@@ -55,14 +56,18 @@ def lib():
         L.qsgd_encode.argtypes = [vp, u64, u32, u32, C.c_int, C.c_int, u64, u32, u32, vp, sz, vp,
                                   vp, vp, vp]
         L.qsgd_encode.restype = C.c_int
-        L.qsgd_decode_accumulate.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, u64, u32, u32,
+        L.qsgd_decode_accumulate.argtypes = [C.POINTER(vp), C.POINTER(vp), C.POINTER(u64), u32, u64, u32, u32,
                                              C.c_int, vp, vp, vp]
         L.qsgd_decode_accumulate.restype = C.c_int
+        L.qsgd_decode_accumulate_packed.argtypes = L.qsgd_decode_accumulate.argtypes
+        L.qsgd_decode_accumulate_packed.restype = C.c_int
         L.qsgd_sgd_step.argtypes = [vp, vp, C.c_float, u32, u64, vp]
         L.qsgd_sgd_step.restype = C.c_int
-        L.qsgd_decode_sgd_step.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, u64, u32, u32,
+        L.qsgd_decode_sgd_step.argtypes = [C.POINTER(vp), C.POINTER(vp), C.POINTER(u64), u32, u64, u32, u32,
                                            C.c_int, vp, C.c_float, vp, vp]
         L.qsgd_decode_sgd_step.restype = C.c_int
+        L.qsgd_decode_sgd_step_packed.argtypes = L.qsgd_decode_sgd_step.argtypes
+        L.qsgd_decode_sgd_step_packed.restype = C.c_int
         L.qsgd_status_string.argtypes = [C.c_int]
         L.qsgd_status_string.restype = C.c_char_p
         L.qsgd_static_scratch_bytes.argtypes = []
@@ -84,10 +89,10 @@ def lib():
         L.qsgd_policy_encode.argtypes = [vp, pp, u32, u32, C.c_int, C.c_int, u64, u32, u32, vp, sz, vp,
                                          vp, vp, vp]
         L.qsgd_policy_encode.restype = C.c_int
-        L.qsgd_policy_decode_accumulate.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, pp, u32, u32,
+        L.qsgd_policy_decode_accumulate.argtypes = [C.POINTER(vp), C.POINTER(vp), pu64, u32, pp, u32, u32,
                                                     C.c_int, vp, vp, vp]
         L.qsgd_policy_decode_accumulate.restype = C.c_int
-        L.qsgd_policy_decode_sgd_step.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, pp, u32, u32,
+        L.qsgd_policy_decode_sgd_step.argtypes = [C.POINTER(vp), C.POINTER(vp), pu64, u32, pp, u32, u32,
                                                   C.c_int, vp, C.c_float, vp, vp]
         L.qsgd_policy_decode_sgd_step.restype = C.c_int
         L.qsgd_test_set_wait_polls.argtypes = [u32]
@@ -207,14 +212,48 @@ def _ptr_array(tensors):
     return arr
 
 
-def qsgd_decode_accumulate(msgs, tables, n, bucket, s, code_kind, acc, status_dev, stream=None):
+def _u64_array(values):
+    if values is None:
+        return None
+    return (C.c_uint64 * len(values))(*[int(v) for v in values])
+
+
+def qsgd_decode_accumulate(msgs, tables, n, bucket, s, code_kind, acc, status_dev, stream=None,
+                           payload_bytes=None):
     """acc <- ascending-k sum of the decoded messages; msgs / tables: lists of CUDA tensors
-    (or raw device addresses)."""
+    (or raw device addresses); payload_bytes: optional list of payload lengths (read bound)."""
     _require_cuda(acc, "acc")
     mp = _ptr_array(msgs)
     tp = None if tables is None else _ptr_array(tables)
-    _check(lib().qsgd_decode_accumulate(mp, tp, len(msgs), n, bucket, s, code_kind,
+    _check(lib().qsgd_decode_accumulate(mp, tp, _u64_array(payload_bytes), len(msgs), n, bucket, s, code_kind,
                                         acc.data_ptr(), status_dev.data_ptr(), _stream(stream)))
+
+
+def _msg_bytes(msgs, msg_bytes):
+    if msg_bytes is not None:
+        return _u64_array(msg_bytes)
+    return _u64_array([m.numel() * m.element_size() for m in msgs])
+
+
+def qsgd_decode_accumulate_packed(msgs, infos, n, bucket, s, code_kind, acc, status_dev, stream=None,
+                                  msg_bytes=None):
+    """As qsgd_decode_accumulate, for messages as Encode left them: infos[k] is the CUDA tensor (or
+    device address) of message k's four info words; the tables are found on the device. msg_bytes
+    defaults to the sizes of the message tensors."""
+    _require_cuda(acc, "acc")
+    ip = None if infos is None else _ptr_array(infos)
+    _check(lib().qsgd_decode_accumulate_packed(_ptr_array(msgs), ip, _msg_bytes(msgs, msg_bytes), len(msgs), n,
+                                               bucket, s, code_kind, acc.data_ptr(), status_dev.data_ptr(),
+                                               _stream(stream)))
+
+
+def qsgd_decode_sgd_step_packed(msgs, infos, n, bucket, s, code_kind, x, eta, status_dev, stream=None,
+                                msg_bytes=None):
+    _require_cuda(x, "x")
+    ip = None if infos is None else _ptr_array(infos)
+    _check(lib().qsgd_decode_sgd_step_packed(_ptr_array(msgs), ip, _msg_bytes(msgs, msg_bytes), len(msgs), n,
+                                             bucket, s, code_kind, x.data_ptr(), eta, status_dev.data_ptr(),
+                                             _stream(stream)))
 
 
 def qsgd_sgd_step(x, acc, eta, K, stream=None):
@@ -223,12 +262,13 @@ def qsgd_sgd_step(x, acc, eta, K, stream=None):
     _check(lib().qsgd_sgd_step(x.data_ptr(), acc.data_ptr(), eta, K, x.numel(), _stream(stream)))
 
 
-def qsgd_decode_sgd_step(msgs, tables, n, bucket, s, code_kind, x, eta, status_dev, stream=None):
+def qsgd_decode_sgd_step(msgs, tables, n, bucket, s, code_kind, x, eta, status_dev, stream=None,
+                         payload_bytes=None):
     _require_cuda(x, "x")
     mp = _ptr_array(msgs)
     tp = None if tables is None else _ptr_array(tables)
-    _check(lib().qsgd_decode_sgd_step(mp, tp, len(msgs), n, bucket, s, code_kind, x.data_ptr(),
-                                      eta, status_dev.data_ptr(), _stream(stream)))
+    _check(lib().qsgd_decode_sgd_step(mp, tp, _u64_array(payload_bytes), len(msgs), n, bucket, s, code_kind,
+                                      x.data_ptr(), eta, status_dev.data_ptr(), _stream(stream)))
 
 
 # ------------------------------- per-tensor policy -------------------------------------------
@@ -284,23 +324,25 @@ def qsgd_policy_encode(g, plan, s, norm_kind, code_kind, seed, step, worker, out
                                     out_bits.data_ptr(), ws, status_dev.data_ptr(), _stream(stream)))
 
 
-def qsgd_policy_decode_accumulate(msgs, tables, plan, s, code_kind, acc, status_dev, stream=None):
+def qsgd_policy_decode_accumulate(msgs, tables, plan, s, code_kind, acc, status_dev, stream=None,
+                                  payload_bytes=None):
     _require_cuda(acc, "acc")
     if acc.numel() != plan.n:
         raise QsgdError("acc has %d elements, the plan covers %d" % (acc.numel(), plan.n))
     mp = _ptr_array(msgs)
     tp = None if tables is None else _ptr_array(tables)
-    _check(lib().qsgd_policy_decode_accumulate(mp, tp, len(msgs), C.byref(plan.struct), plan.bucket, s, code_kind,
+    _check(lib().qsgd_policy_decode_accumulate(mp, tp, _u64_array(payload_bytes), len(msgs), C.byref(plan.struct), plan.bucket, s, code_kind,
                                                acc.data_ptr(), status_dev.data_ptr(), _stream(stream)))
 
 
-def qsgd_policy_decode_sgd_step(msgs, tables, plan, s, code_kind, x, eta, status_dev, stream=None):
+def qsgd_policy_decode_sgd_step(msgs, tables, plan, s, code_kind, x, eta, status_dev, stream=None,
+                                payload_bytes=None):
     _require_cuda(x, "x")
     if x.numel() != plan.n:
         raise QsgdError("x has %d elements, the plan covers %d" % (x.numel(), plan.n))
     mp = _ptr_array(msgs)
     tp = None if tables is None else _ptr_array(tables)
-    _check(lib().qsgd_policy_decode_sgd_step(mp, tp, len(msgs), C.byref(plan.struct), plan.bucket, s, code_kind,
+    _check(lib().qsgd_policy_decode_sgd_step(mp, tp, _u64_array(payload_bytes), len(msgs), C.byref(plan.struct), plan.bucket, s, code_kind,
                                              x.data_ptr(), eta, status_dev.data_ptr(), _stream(stream)))
 
 

@@ -61,13 +61,18 @@ uint32_t host_elias_len(uint32_t k) {
   return len;
 }
 
-int resolve_peers(const void* const* msgs, const uint64_t* const* tables, uint32_t K, uint64_t n,
-                  uint32_t bucket, uint32_t s, int code_kind, PeerSet* ps) {
+// msgs / tables / bytes as the decode entry points receive them. packed: tables[k] points to the
+// four info words of message k and bytes[k] says how much of the message buffer may be read;
+// otherwise tables[k] is the offset table and bytes (optional) bounds the payload.
+int resolve_peers(const void* const* msgs, const uint64_t* const* tables, const uint64_t* bytes, bool packed,
+                  uint32_t K, uint64_t n, uint32_t bucket, uint32_t s, int code_kind, PeerSet* ps) {
   if (!msgs) return QSGD_ERR_NULL;
   if (K < 1 || K > QSGD_MAX_PEERS) return QSGD_ERR_PEERS;
-  if (code_kind != QSGD_CODE_FIXED && !tables) return QSGD_ERR_NULL;
+  if (code_kind != QSGD_CODE_FIXED && (!tables || (packed && !bytes))) return QSGD_ERR_NULL;
   const FixedLayout L = make_fixed_layout(n, bucket, s);
+  ps->packed = (packed && code_kind != QSGD_CODE_FIXED) ? 1u : 0u;
   for (uint32_t k = 0; k < K; ++k) {
+    ps->bound[k] = (bytes && code_kind != QSGD_CODE_FIXED) ? bytes[k] : 0ull;
     if (!msgs[k]) return QSGD_ERR_NULL;
     if (!aligned16(msgs[k])) return QSGD_ERR_ALIGN;
     const uint8_t* m = static_cast<const uint8_t*>(msgs[k]);
@@ -144,20 +149,38 @@ int qsgd_encode(const float* g, uint64_t n, uint32_t bucket, uint32_t s, int nor
                              static_cast<uint8_t*>(workspace), status_dev, no_map(), cs);
 }
 
-int qsgd_decode_accumulate(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
-                           uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* acc,
-                           uint32_t* status_dev, qsgd_stream_t stream) {
-  if (!acc || !status_dev) return QSGD_ERR_NULL;
+static int decode_any(const void* const* msgs, const uint64_t* const* tables, const uint64_t* bytes, bool packed,
+                      uint32_t K, uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* out, bool fused,
+                      float eta, uint32_t* status_dev, qsgd_stream_t stream) {
+  if (!out || !status_dev) return QSGD_ERR_NULL;
   int st = check_shape(n, bucket, s, code_kind);
   if (st) return st;
-  if (!aligned16(acc)) return QSGD_ERR_ALIGN;
+  if (!aligned16(out)) return QSGD_ERR_ALIGN;
   PeerSet ps;
-  st = resolve_peers(msgs, tables, K, n, bucket, s, code_kind, &ps);
+  st = resolve_peers(msgs, tables, bytes, packed, K, n, bucket, s, code_kind, &ps);
   if (st) return st;
   cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  if (code_kind == QSGD_CODE_FIXED) return launch_decode_fixed(ps, K, n, bucket, s, acc, false, 0.f, no_map(), cs);
-  return launch_decode_elias(ps, K, n, bucket, s, code_kind == QSGD_CODE_ELIAS_DENSE, acc, false, 0.f,
+  if (code_kind == QSGD_CODE_FIXED) return launch_decode_fixed(ps, K, n, bucket, s, out, fused, eta, no_map(), cs);
+  return launch_decode_elias(ps, K, n, bucket, s, code_kind == QSGD_CODE_ELIAS_DENSE, out, fused, eta,
                              status_dev, no_map(), cs);
+}
+
+int qsgd_decode_accumulate(const void* const* msgs, const uint64_t* const* tables, const uint64_t* payload_bytes,
+                           uint32_t K, uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* acc,
+                           uint32_t* status_dev, qsgd_stream_t stream) {
+  return decode_any(msgs, tables, payload_bytes, false, K, n, bucket, s, code_kind, acc, false, 0.f, status_dev, stream);
+}
+
+int qsgd_decode_accumulate_packed(const void* const* msgs, const uint64_t* const* infos, const uint64_t* msg_bytes,
+                                  uint32_t K, uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* acc,
+                                  uint32_t* status_dev, qsgd_stream_t stream) {
+  return decode_any(msgs, infos, msg_bytes, true, K, n, bucket, s, code_kind, acc, false, 0.f, status_dev, stream);
+}
+
+int qsgd_decode_sgd_step_packed(const void* const* msgs, const uint64_t* const* infos, const uint64_t* msg_bytes,
+                                uint32_t K, uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* x,
+                                float eta, uint32_t* status_dev, qsgd_stream_t stream) {
+  return decode_any(msgs, infos, msg_bytes, true, K, n, bucket, s, code_kind, x, true, eta, status_dev, stream);
 }
 
 int qsgd_sgd_step(float* x, const float* acc, float eta, uint32_t K, uint64_t n,
@@ -169,20 +192,10 @@ int qsgd_sgd_step(float* x, const float* acc, float eta, uint32_t K, uint64_t n,
   return launch_sgd_step(x, acc, eta, K, n, static_cast<cudaStream_t>(stream));
 }
 
-int qsgd_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
-                         uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* x,
+int qsgd_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables, const uint64_t* payload_bytes,
+                         uint32_t K, uint64_t n, uint32_t bucket, uint32_t s, int code_kind, float* x,
                          float eta, uint32_t* status_dev, qsgd_stream_t stream) {
-  if (!x || !status_dev) return QSGD_ERR_NULL;
-  int st = check_shape(n, bucket, s, code_kind);
-  if (st) return st;
-  if (!aligned16(x)) return QSGD_ERR_ALIGN;
-  PeerSet ps;
-  st = resolve_peers(msgs, tables, K, n, bucket, s, code_kind, &ps);
-  if (st) return st;
-  cudaStream_t cs = static_cast<cudaStream_t>(stream);
-  if (code_kind == QSGD_CODE_FIXED) return launch_decode_fixed(ps, K, n, bucket, s, x, true, eta, no_map(), cs);
-  return launch_decode_elias(ps, K, n, bucket, s, code_kind == QSGD_CODE_ELIAS_DENSE, x, true, eta,
-                             status_dev, no_map(), cs);
+  return decode_any(msgs, tables, payload_bytes, false, K, n, bucket, s, code_kind, x, true, eta, status_dev, stream);
 }
 
 // ---- per-tensor policy --------------------------------------------------------------------------
@@ -292,8 +305,8 @@ int qsgd_policy_encode(const float* g, const qsgd_policy* plan, uint32_t bucket,
   return launch_raw_gather(g, raw_of(plan), static_cast<float*>(out), out_bits, nc != 0, cs);
 }
 
-static int policy_decode(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
-                         const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind, float* out,
+static int policy_decode(const void* const* msgs, const uint64_t* const* tables, const uint64_t* payload_bytes,
+                         uint32_t K, const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind, float* out,
                          bool fused, float eta, uint32_t* status_dev, qsgd_stream_t stream) {
   if (!out || !status_dev || !msgs) return QSGD_ERR_NULL;
   int st = check_policy(plan, bucket, s, code_kind);
@@ -313,7 +326,7 @@ static int policy_decode(const void* const* msgs, const uint64_t* const* tables,
   const uint64_t nc = plan->n_buckets * bucket;
   if (nc) {
     PeerSet ps;
-    st = resolve_peers(body, tables, K, nc, bucket, s, code_kind, &ps);
+    st = resolve_peers(body, tables, payload_bytes, false, K, nc, bucket, s, code_kind, &ps);
     if (st) return st;
     if (code_kind == QSGD_CODE_FIXED) st = launch_decode_fixed(ps, K, nc, bucket, s, out, fused, eta, map_of(plan), cs);
     else st = launch_decode_elias(ps, K, nc, bucket, s, code_kind == QSGD_CODE_ELIAS_DENSE, out, fused, eta,
@@ -323,16 +336,16 @@ static int policy_decode(const void* const* msgs, const uint64_t* const* tables,
   return launch_raw_decode(raw, K, raw_of(plan), out, fused, eta, cs);
 }
 
-int qsgd_policy_decode_accumulate(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
-                                  const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind,
+int qsgd_policy_decode_accumulate(const void* const* msgs, const uint64_t* const* tables, const uint64_t* payload_bytes,
+                                  uint32_t K, const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind,
                                   float* acc, uint32_t* status_dev, qsgd_stream_t stream) {
-  return policy_decode(msgs, tables, K, plan, bucket, s, code_kind, acc, false, 0.f, status_dev, stream);
+  return policy_decode(msgs, tables, payload_bytes, K, plan, bucket, s, code_kind, acc, false, 0.f, status_dev, stream);
 }
 
-int qsgd_policy_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables, uint32_t K,
-                                const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind,
+int qsgd_policy_decode_sgd_step(const void* const* msgs, const uint64_t* const* tables, const uint64_t* payload_bytes,
+                                uint32_t K, const qsgd_policy* plan, uint32_t bucket, uint32_t s, int code_kind,
                                 float* x, float eta, uint32_t* status_dev, qsgd_stream_t stream) {
-  return policy_decode(msgs, tables, K, plan, bucket, s, code_kind, x, true, eta, status_dev, stream);
+  return policy_decode(msgs, tables, payload_bytes, K, plan, bucket, s, code_kind, x, true, eta, status_dev, stream);
 }
 
 const char* qsgd_status_string(int status) {

@@ -17,7 +17,7 @@ int launch_decode_elias(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d
   // kernels are launched and exactly one does the work. Either decoder is correct on any input;
   // the choice is about speed only.
   const uint64_t B = (n + d - 1) / d;
-  bool sizes_known = !dense && K <= 32u;
+  bool sizes_known = !dense && K <= 32u && !peers.packed;
   uint64_t payload_bits = 0;
   for (uint32_t k = 0; k < K && sizes_known; ++k) {
     const uint8_t* w = reinterpret_cast<const uint8_t*>(peers.payload[k]);

@@ -48,6 +48,59 @@ inline SparseShape sparse_shape(uint32_t K, uint32_t d, uint64_t B, uint32_t sms
   return sh;
 }
 
+// Where peer k's offset table is and how many payload bits may be read. Ordinary form: the caller
+// gave the table pointer; the payload is bounded by the byte count the caller gave, else by the
+// table's own address when it sits behind the payload (as Encode writes it), else not at all.
+// Packed form: the table sits at byte info[1] of the message, which also is the padded payload
+// length; the place must be 16-byte aligned and the whole table must lie inside the bytes the
+// caller declared readable. Returns false (nothing may be read) when the packed place is bad.
+struct PeerTable {
+  const uint64_t* table;
+  uint64_t cap_bits;
+};
+
+__device__ __forceinline__ bool peer_table(const PeerSet& ps, uint32_t k, uint64_t B, PeerTable* out) {
+  const uint8_t* words = reinterpret_cast<const uint8_t*>(ps.payload[k]);
+  if (ps.packed) {
+    const uint64_t off = __ldg(ps.table[k] + 1);
+    const uint64_t need = 8ull * (B + 1ull);
+    out->table = nullptr;
+    out->cap_bits = 0;
+    if ((off & 15ull) || off > ps.bound[k] || ps.bound[k] - off < need) return false;
+    out->table = reinterpret_cast<const uint64_t*>(words + off);
+    out->cap_bits = 8ull * off;
+    return true;
+  }
+  const uint8_t* t = reinterpret_cast<const uint8_t*>(ps.table[k]);
+  out->table = ps.table[k];
+  out->cap_bits = ps.bound[k] ? 8ull * ps.bound[k] : (t > words ? 8ull * (uint64_t)(t - words) : ~0ull);
+  return true;
+}
+
+// First bit and length of bucket b's string of peer k, after every check that can be made before
+// the payload is touched: table entries ascending, at least the 32 bits of the scale, the end
+// inside the payload (table's last entry, and that entry inside the bound of peer_table), not
+// longer than any legal string of db coordinates. err != 0 means: read nothing.
+struct StringRef {
+  const uint32_t* words;
+  uint64_t lo;        // first bit (the scale)
+  uint32_t total;     // bits after the scale
+  uint32_t err;
+};
+
+__device__ __forceinline__ StringRef string_ref(const PeerSet& ps, uint32_t k, uint64_t b, uint64_t B, uint32_t db) {
+  StringRef r;
+  r.words = ps.payload[k];
+  r.lo = 0; r.total = 0; r.err = 0;
+  PeerTable pt;
+  if (!peer_table(ps, k, B, &pt)) { r.err = QSGD_DEV_TABLE; return r; }
+  const uint64_t lo = __ldg(pt.table + b), hi = __ldg(pt.table + b + 1), all = __ldg(pt.table + B);
+  if (hi < lo || hi - lo < 32 || hi > all || all > pt.cap_bits) r.err = QSGD_DEV_TABLE;
+  else if (hi - lo > 32ull + (uint64_t)db * 40ull) r.err = QSGD_DEV_OVERRUN;
+  else { r.lo = lo; r.total = (uint32_t)(hi - lo) - 32u; }
+  return r;
+}
+
 // Strings short enough for the entry-list decoder? True when the K payloads average less than a
 // quarter of a bit per coordinate beyond the scales: an entry of a sparse bucket costs 11 to 14
 // bits, so a list with room for one entry per 32 positions then fills to about 60 % on average and
@@ -55,7 +108,11 @@ inline SparseShape sparse_shape(uint32_t K, uint32_t d, uint64_t B, uint32_t sms
 __device__ __forceinline__ bool sparse_regime(const PeerSet& peers, uint32_t K, uint64_t B, uint32_t d) {
   if (K > 32u) return false;
   uint64_t bits = 0;
-  for (uint32_t k = 0; k < K; ++k) bits += __ldg(peers.table[k] + B);
+  for (uint32_t k = 0; k < K; ++k) {
+    PeerTable pt;
+    if (!peer_table(peers, k, B, &pt)) return false;        // the field decoders report the bad place
+    bits += __ldg(pt.table + B);
+  }
   return bits < (uint64_t)K * B * (32ull + d / 4u);
 }
 

@@ -18,20 +18,16 @@ namespace qsgd {
 namespace {
 
 template <int LB, bool DENSE>
-__device__ __forceinline__ uint32_t parse_to_fields(const uint32_t* __restrict__ words,
-                                                    const uint64_t* __restrict__ table, uint64_t b,
+__device__ __forceinline__ uint32_t parse_to_fields(const PeerSet& peers, uint32_t k, uint64_t b,
                                                     uint64_t B, uint32_t db, uint32_t d, uint32_t s,
                                                     const uint16_t* lut, uint32_t* __restrict__ row,
                                                     float* A_out) {
-  const uint64_t lo = __ldg(table + b), hi = __ldg(table + b + 1), all = __ldg(table + B);
   *A_out = 0.f;
-  if (hi < lo || hi - lo < 32 || hi > all) return QSGD_DEV_TABLE;
-  const uint64_t cap_bits = (uint64_t)((const uint8_t*)table - (const uint8_t*)words) * 8ull;
-  if ((const uint8_t*)table > (const uint8_t*)words && all > cap_bits) return QSGD_DEV_TABLE;
-  if (hi - lo > 32ull + (uint64_t)db * 40ull) return QSGD_DEV_OVERRUN;   // longer than any legal string
-  const uint32_t total = (uint32_t)(hi - lo) - 32u;
+  const StringRef ref = string_ref(peers, k, b, B, db);
+  if (ref.err) return ref.err;
+  const uint32_t total = ref.total;
   BitSrc src;
-  src.open(words, lo);
+  src.open(ref.words, ref.lo);
   *A_out = __uint_as_float(src.take(32));
   uint32_t* srow = row + ((d * LB) >> 5);            // sign bitmap of this peer row
   uint32_t used = 0, err = 0;
@@ -131,7 +127,7 @@ __global__ void __launch_bounds__(320) decode_elias_fields_kernel(const __grid_c
         const uint64_t base = b * p.d;
         const uint32_t db = (uint32_t)min((uint64_t)p.d, p.n - base);
         float A;
-        const uint32_t st = parse_to_fields<LB, DENSE>(p.peers.payload[k], p.peers.table[k], b, p.B, db, p.d,
+        const uint32_t st = parse_to_fields<LB, DENSE>(p.peers, k, b, p.B, db, p.d,
                                                        p.s, elias_lut, bucket + k * p.row_words, &A);
         reinterpret_cast<float*>(bucket + p.K * p.row_words)[k] = A;
         if (st) atomicOr(p.status, st);
@@ -285,17 +281,11 @@ __global__ void __launch_bounds__(128) decode_elias_ranged_kernel(const __grid_c
     if (pg < p.G && b0 + pg < p.B) db = (uint32_t)min((uint64_t)p.d, p.n - (b0 + pg) * p.d);
     const bool parsing = db != 0u && pk < p.K;
     if (parsing) {
-      const uint64_t b = b0 + pg;
-      const uint32_t* words = p.peers.payload[pk];
-      const uint64_t* table = p.peers.table[pk];
-      const uint64_t lo = __ldg(table + b), hi = __ldg(table + b + 1), all = __ldg(table + p.B);
-      const uint64_t cap_bits = (uint64_t)((const uint8_t*)table - (const uint8_t*)words) * 8ull;
-      if (hi < lo || hi - lo < 32 || hi > all) st.err = QSGD_DEV_TABLE;
-      else if ((const uint8_t*)table > (const uint8_t*)words && all > cap_bits) st.err = QSGD_DEV_TABLE;
-      else if (hi - lo > 32ull + (uint64_t)db * 40ull) st.err = QSGD_DEV_OVERRUN;   // longer than any legal string
-      else {
-        st.total = (uint32_t)(hi - lo) - 32u;
-        st.src.open(words, lo);
+      const StringRef ref = string_ref(p.peers, pk, b0 + pg, p.B, db);
+      st.err = ref.err;
+      if (!ref.err) {
+        st.total = ref.total;
+        st.src.open(ref.words, ref.lo);
         A = __uint_as_float(st.src.take(32));
       }
     }

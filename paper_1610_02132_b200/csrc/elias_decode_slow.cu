@@ -16,16 +16,14 @@ template <> struct CodeTraits<uint16_t> { static constexpr uint32_t kSignBit = 0
 
 // Parses one bucket string of one peer into codes[0..db). Returns a QSGD_DEV_* mask.
 template <typename CodeT, bool DENSE>
-__device__ __forceinline__ uint32_t parse_bucket(const uint32_t* __restrict__ words,
-                                                 const uint64_t* __restrict__ table, uint64_t b,
+__device__ __forceinline__ uint32_t parse_bucket(const PeerSet& peers, uint32_t k, uint64_t b,
                                                  uint64_t B, uint32_t db, uint32_t s,
                                                  CodeT* __restrict__ codes, float* A_out) {
-  const uint64_t lo = __ldg(table + b), hi = __ldg(table + b + 1), all = __ldg(table + B);
   *A_out = 0.f;
-  if (hi < lo || hi - lo < 32 || hi > all) return QSGD_DEV_TABLE;
-  // the table sits directly behind the payload: its address bounds the payload length
-  const uint64_t cap_bits = (uint64_t)((const uint8_t*)table - (const uint8_t*)words) * 8ull;
-  if ((const uint8_t*)table > (const uint8_t*)words && all > cap_bits) return QSGD_DEV_TABLE;
+  const StringRef ref = string_ref(peers, k, b, B, db);
+  if (ref.err) return ref.err;
+  const uint32_t* __restrict__ words = ref.words;
+  const uint64_t lo = ref.lo, hi = ref.lo + 32ull + ref.total;
   uint64_t pos = lo;
   *A_out = __uint_as_float(peek32(words, pos));
   pos += 32;
@@ -89,8 +87,8 @@ __global__ void __launch_bounds__(kThreads) decode_elias_slow_kernel(const __gri
       // phase 1: one lane per peer
       for (uint32_t kk = lane; kk < kc; kk += 32) {
         float A;
-        const uint32_t st = parse_bucket<CodeT, DENSE>(p.peers.payload[k0 + kk], p.peers.table[k0 + kk],
-                                                       b, p.B, db, p.s, codes + (size_t)kk * p.d, &A);
+        const uint32_t st = parse_bucket<CodeT, DENSE>(p.peers, k0 + kk, b, p.B, db, p.s,
+                                                       codes + (size_t)kk * p.d, &A);
         sA[kk] = A;
         if (st) atomicOr(p.status, st);
       }

@@ -63,17 +63,11 @@ __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __gri
     }
     const bool parsing = db != 0u && pk < p.K;
     if (parsing) {
-      const uint64_t b = b0 + pg;
-      const uint32_t* words = p.peers.payload[pk];
-      const uint64_t* table = p.peers.table[pk];
-      const uint64_t lo = __ldg(table + b), hi = __ldg(table + b + 1), all = __ldg(table + p.B);
-      const uint64_t cap_bits = (uint64_t)((const uint8_t*)table - (const uint8_t*)words) * 8ull;
-      if (hi < lo || hi - lo < 32 || hi > all) st.err = QSGD_DEV_TABLE;
-      else if ((const uint8_t*)table > (const uint8_t*)words && all > cap_bits) st.err = QSGD_DEV_TABLE;
-      else if (hi - lo > 32ull + (uint64_t)db * 40ull) st.err = QSGD_DEV_OVERRUN;   // longer than any legal string
-      else {
-        st.total = (uint32_t)(hi - lo) - 32u;
-        st.src.open(words, lo);
+      const StringRef ref = string_ref(p.peers, pk, b0 + pg, p.B, db);
+      st.err = ref.err;
+      if (!ref.err) {
+        st.total = ref.total;
+        st.src.open(ref.words, ref.lo);
         A = __uint_as_float(st.src.take(32));
       }
     }

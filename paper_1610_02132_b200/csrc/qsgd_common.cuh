@@ -91,7 +91,10 @@ struct PeerSet {                 // K messages, resolved to region pointers on t
   const uint32_t* sign[QSGD_MAX_PEERS];    // fixed: sign bitmaps
   const uint32_t* level[QSGD_MAX_PEERS];   // fixed: level fields
   const uint32_t* payload[QSGD_MAX_PEERS]; // Elias: payload words
-  const uint64_t* table[QSGD_MAX_PEERS];   // Elias: offset tables
+  const uint64_t* table[QSGD_MAX_PEERS];   // Elias: offset tables; packed form: the message's four info words
+  uint64_t bound[QSGD_MAX_PEERS];          // Elias: bytes of payload the caller vouches for (0 = not given);
+                                           // packed form: bytes readable from the start of the message
+  uint32_t packed;                         // Elias: tables are found on the device, at byte info[1] of each message
 };
 
 // Per-tensor policy (Section 5, "Protocol"): the coordinates that get quantized form a "compact"

@@ -104,6 +104,18 @@ def decode_parity(msgs_dev, infos, n, d, s, code_kind, eta=0.1, x0=None, tables_
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     assert bool((acc[n:] == 7.0).all()) and bool((xf[n:] == 3.0).all())
+    if not tables_first:
+        # the packed form (tables found on the device from the info words) gives the same bits
+        info_dev = [torch.tensor([int(v) for v in i], dtype=torch.int64, device=dev) for i in infos]
+        acc_p = torch.full((n + 64,), 7.0, dtype=torch.float32, device=dev)
+        xp = torch.full((n + 64,), 3.0, dtype=torch.float32, device=dev)
+        xp[:n] = torch.from_numpy(x0).cuda()
+        Q.qsgd_decode_accumulate_packed(msgs_dev, info_dev, n, d, s, code_kind, acc_p[:n], status)
+        Q.qsgd_decode_sgd_step_packed(msgs_dev, info_dev, n, d, s, code_kind, xp[:n], eta, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert torch.equal(acc_p.view(torch.int32), acc.view(torch.int32))
+        assert torch.equal(xp.view(torch.int32), xf.view(torch.int32))
     msgs = [m.cpu().numpy() for m in msgs_dev]
     tabs = None if tables is None else [t.cpu().numpy().view(np.uint64) for t in tables]
     st, acc_ref = O.decode_accumulate(msgs, tabs, n, d, s, code_kind)

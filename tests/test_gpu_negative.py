@@ -32,7 +32,7 @@ def good_message(shape, code_kind=O.CODE_ELIAS, seed=5):
     return m, info
 
 
-def run_decode(shape, msg_np, info, code_kind=O.CODE_ELIAS, table_np=None, s=None, n=None):
+def run_decode(shape, msg_np, info, code_kind=O.CODE_ELIAS, table_np=None, s=None, n=None, payload_bytes=None):
     """Decode one (possibly corrupted) message on the GPU; returns (status, acc, guard ok)."""
     d = shape[1]
     s = shape[2] if s is None else s
@@ -45,10 +45,11 @@ def run_decode(shape, msg_np, info, code_kind=O.CODE_ELIAS, table_np=None, s=Non
         table = torch.from_numpy(table_np.view(np.int64)).cuda()
     acc = torch.full((n + 256,), 7.0, dtype=torch.float32, device="cuda")
     status = Q.new_status()
-    Q.qsgd_decode_accumulate([buf], [table], n, d, s, code_kind, acc[:n], status)
+    pb = None if payload_bytes is None else [payload_bytes]
+    Q.qsgd_decode_accumulate([buf], [table], n, d, s, code_kind, acc[:n], status, payload_bytes=pb)
     x = torch.full((n + 256,), 3.0, dtype=torch.float32, device="cuda")
     status2 = Q.new_status()
-    Q.qsgd_decode_sgd_step([buf], [table], n, d, s, code_kind, x[:n], 0.5, status2)
+    Q.qsgd_decode_sgd_step([buf], [table], n, d, s, code_kind, x[:n], 0.5, status2, payload_bytes=pb)
     torch.cuda.synchronize()
     guard = bool((acc[n:] == 7.0).all()) and bool((x[n:] == 3.0).all())
     assert (int(status.item()) != 0) == (int(status2.item()) != 0)
@@ -84,6 +85,39 @@ def test_offsets_not_ascending_and_short_bucket(shape):
     t[1] = t[0] + 8                              # shorter than the 32-bit scale
     st, _, guard = run_decode(shape, m, info, table_np=t)
     assert st != 0 and guard
+
+
+def test_table_claiming_more_payload_than_there_is(shape):
+    """A table kept apart from its message whose last entry overstates the payload: with the payload
+    length given, every string of that message is refused before a single payload bit is read."""
+    n, d, s, _ = shape
+    m, info = good_message(shape)
+    t = O.message_table(m, info, n, d).copy()
+    t[-1] += 1 << 33                              # the last bucket now "ends" a gigabyte past the buffer
+    st, acc, guard = run_decode(shape, m, info, table_np=t, payload_bytes=info[1])
+    assert st & Q.binding.DEV_TABLE and guard
+    # the honest table with the same bound decodes cleanly
+    st, acc, guard = run_decode(shape, m, info, table_np=O.message_table(m, info, n, d).copy(), payload_bytes=info[1])
+    ref = O.decode(m, O.message_table(m, info, n, d), n, d, s, O.CODE_ELIAS)[1]
+    assert st == 0 and guard and np.array_equal(acc.view(np.uint32), ref.view(np.uint32))
+
+
+def test_packed_form_rejects_bad_table_places(shape):
+    """Packed decode reads the table's place from the info words on the device: a place that is
+    misaligned, or whose table would not fit in the bytes declared readable, is refused."""
+    n, d, s, _ = shape
+    m, info = good_message(shape)
+    buf = torch.from_numpy(np.concatenate([m, np.zeros(64, np.uint8)])).cuda()
+    for bad_info, nbytes in (([info[0], info[1] + 8, info[2], 0], buf.numel()),       # not 16-byte aligned
+                             ([info[0], info[1], info[2], 0], info[2] - 16),            # table cut off
+                             ([info[0], 1 << 40, info[2], 0], buf.numel())):           # far outside
+        iw = torch.tensor(bad_info, dtype=torch.int64, device="cuda")
+        acc = torch.full((n + 256,), 7.0, dtype=torch.float32, device="cuda")
+        status = Q.new_status()
+        Q.qsgd_decode_accumulate_packed([buf], [iw], n, d, s, O.CODE_ELIAS, acc[:n], status, msg_bytes=[nbytes])
+        torch.cuda.synchronize()
+        assert int(status.item()) & Q.binding.DEV_TABLE
+        assert bool((acc[n:] == 7.0).all())
 
 
 def test_level_above_s_is_flagged(shape):

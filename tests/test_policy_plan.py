@@ -73,6 +73,6 @@ def test_policy_entry_points_validate_before_launching():
     assert L.qsgd_policy_workspace_bytes(C.byref(good), 512, 15, 0) == 0                         # fixed-width: none
     assert L.qsgd_policy_workspace_bytes(C.byref(good), 512, 15, 1) == Q.qsgd_workspace_bytes(pl.n_buckets * 512, 512, 15, 1)
     msgs = (C.c_void_p * 1)(16)
-    assert L.qsgd_policy_decode_sgd_step(msgs, None, 0, C.byref(good), 512, 15, 0, 16, 0.1, 16, None) == -7   # K = 0
-    assert L.qsgd_policy_decode_sgd_step(msgs, None, 1, C.byref(good), 512, 15, 0, 8, 0.1, 16, None) == -5    # x misaligned
-    assert L.qsgd_policy_decode_sgd_step(msgs, None, 1, C.byref(good), 512, 15, 1, 16, 0.1, 16, None) == -1   # Elias needs tables
+    assert L.qsgd_policy_decode_sgd_step(msgs, None, None, 0, C.byref(good), 512, 15, 0, 16, 0.1, 16, None) == -7   # K = 0
+    assert L.qsgd_policy_decode_sgd_step(msgs, None, None, 1, C.byref(good), 512, 15, 0, 8, 0.1, 16, None) == -5    # x misaligned
+    assert L.qsgd_policy_decode_sgd_step(msgs, None, None, 1, C.byref(good), 512, 15, 1, 16, 0.1, 16, None) == -1   # Elias needs tables
