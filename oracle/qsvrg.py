@@ -2,7 +2,8 @@
 
 TEST INFRASTRUCTURE ONLY, like oracle.py. Written step by step in the paper's order:
 
-  epoch p:   every processor i quantizes the gradient of its share h_i at y^(p) and broadcasts it,
+  epoch p:   x_1 = y^(p) (appendix, "Background on SVRG": every epoch starts from its own average);
+             every processor i quantizes the gradient of its share h_i at y^(p) and broadcasts it,
              H_p = sum_i Q~(grad h_i(y^(p)))                                   (appendix form);
   t = 1..T:  processor i draws j, broadcasts u_i = Q~(grad f_j(x_t) - grad f_j(y^(p)) + H_p),
              x_(t+1) = x_t - eta * (1 / K) * sum_i u_i;
@@ -47,6 +48,7 @@ def qsvrg(grad_share, grad_sample, n, K, P, T, eta, indices, x0, code_kind=O.COD
 
     for p in range(P):
         step0 = p * (T + 1)
+        x = y.copy()                                                           # x_1^(p) = y^(p)
         shares = [np.asarray(grad_share(i, y), dtype=np.float32) for i in range(K)]
         if quantize_full:
             msgs, tabs = broadcast(shares, step0)

@@ -1,5 +1,6 @@
 """QSVRG (Section 3.3 and its appendix): the variance-reduced variant, orchestrated on the host around
-the library's Encode / Decode. Every broadcast vector is encoded by `qsgd_encode` with one bucket
+the library's Encode / Decode. Every epoch starts its iterate at the epoch's own point, x_1 = y^(p)
+(appendix, "Background on SVRG"). Every broadcast vector is encoded by `qsgd_encode` with one bucket
 spanning the whole vector (bucket = n <= 4096), s = floor(sqrt(n)) levels and the 2-norm, and the K
 messages of an iteration are decoded, averaged and applied by one `qsgd_decode_sgd_step`
 (x <- x - (eta / K) * sum_i u_i is exactly the paper's x_(t+1) = x_t - eta * u_t). The per-epoch sum
@@ -77,6 +78,7 @@ def qsvrg(grad_share, grad_sample, n, K, P, T, eta, indices, x0, code_kind=Q.COD
 
     for p in range(P):
         step0 = p * (T + 1)
+        x.copy_(y)                                                # every epoch starts at x_1 = y^(p)
         shares = [grad_share(i, y) for i in range(K)]
         if quantize_full:
             tables = broadcast(shares, step0)

@@ -92,6 +92,7 @@ def test_fine_quantization_tracks_plain_svrg():
     x = np.zeros(n)
     y = x.copy()
     for p in range(P):
+        x = y.copy()                          # SVRG as the appendix states it: x_1^(p) = y^(p)
         H = sum(gs(i, y).astype(np.float64) for i in range(k))
         xs = np.zeros(n)
         for t in range(T):
