@@ -28,7 +28,7 @@ NORM = {"l2": 0, "max": 1}
 CODE = {"fixed": 0, "elias": 1, "elias_dense": 2}
 
 WORKLOADS = {
-    # BASELINE configs: name -> (n, d, s, norm, codes, K, generator)
+    # the five workloads the metric is defined on: name -> (n, d, s, norm, codes, K, generator)
     "tiny": dict(n=2 ** 20, d=512, s=15, norm="l2", codes=["fixed"], K=4, gen="gauss0.01",
                  desc="tiny ref: N(0,0.01^2), n=2^20"),
     "sparse_elias": dict(n=2 ** 24, d=4096, s=1, norm="l2", codes=["elias"], K=8, gen="sparse_laplace",
@@ -215,27 +215,38 @@ class HotPath:
                 Q.qsgd_encode(g[w], self.d, self.s, self.norm, code, PHILOX_SEED, step, w,
                               self.msgs[code][w], self.bits[code][w], self.ws[code], self.status)
 
+    def read_info(self, code):
+        """Message sizes of the last encode (a host read-back; outside the timed step except under
+        the per-tensor policy, whose decode takes host-resolved table pointers)."""
+        if code != 0:
+            self.info[code] = self.bits[code].cpu().numpy().view(np.uint64)        # synchronises the stream
+
     def resolve_tables(self, code):
-        """Elias: the sender reads the message length back (it needs it to send the message);
-        the offset table sits at byte out_bits[1] of each message."""
+        """Elias under the per-tensor policy: the offset table sits at byte out_bits[1] of each message."""
         if code == 0:
             return None
-        info = self.bits[code].cpu().numpy().view(np.uint64)        # synchronises the stream
-        self.info[code] = info
+        self.read_info(code)
+        info = self.info[code]
         nb = 8 * (self.B + 1)
         return [self.msgs[code][w][int(info[w, 1]): int(info[w, 1]) + nb].view(self.torch.int64)
                 for w in range(self.K)]
 
+    def decode(self, code):
+        """Fused decode + aggregate + SGD step of the K messages of `code`. Ordinary workloads use
+        the packed form: the kernels find each offset table from the message's info words on the
+        device, so nothing is read back between Encode and Decode."""
+        if self.plan is not None:
+            self.Q.qsgd_policy_decode_sgd_step(self.msgs[code], self.resolve_tables(code), self.plan, self.s, code,
+                                               self.x, ETA, self.status)
+        else:
+            infos = None if code == 0 else [self.bits[code][w] for w in range(self.K)]
+            self.Q.qsgd_decode_sgd_step_packed(self.msgs[code], infos, self.n, self.d, self.s, code, self.x, ETA,
+                                               self.status)
+
     def step(self, step_idx, src=None):
         for code in self.codes:
             self.encode_all(code, step_idx, src)
-            tables = self.resolve_tables(code)
-            if self.plan is not None:
-                self.Q.qsgd_policy_decode_sgd_step(self.msgs[code], tables, self.plan, self.s, code, self.x,
-                                                   ETA, self.status)
-            else:
-                self.Q.qsgd_decode_sgd_step(self.msgs[code], tables, self.n, self.d, self.s, code, self.x,
-                                            ETA, self.status)
+            self.decode(code)
 
     def message_bytes(self, code):
         if code == 0:
@@ -352,14 +363,13 @@ def run_cuda(args):
         e[0].record()
         hp.encode_all(code, 1000)
         e[1].record()
-        tables = hp.resolve_tables(code)
+        hp.read_info(code)
         torch.cuda.synchronize()
         e[1].record()
-        Q.qsgd_decode_sgd_step(hp.msgs[code], tables, hp.n, hp.d, hp.s, code, hp.x, ETA, hp.status)
+        hp.decode(code)
         e[2].record()
         torch.cuda.synchronize()
-        t_enc, t_dec = e[0].elapsed_time(e[1]) * 1e-3 / K, e[1].elapsed_time(e[2]) * 1e-3
-        # encode time above includes the table read-back for Elias; re-time encode alone
+        t_dec = e[1].elapsed_time(e[2]) * 1e-3
         torch.cuda.synchronize(); e[0].record(); hp.encode_all(code, 1001); e[1].record()
         torch.cuda.synchronize()
         t_enc = e[0].elapsed_time(e[1]) * 1e-3 / K
@@ -404,16 +414,25 @@ def run_cuda(args):
             pinned[w].copy_(hp.g[w])
         x_host = torch.empty(n, dtype=torch.float32).pin_memory()
         stage = [torch.empty(n, dtype=torch.float32, device=device) for _ in range(2)]
+        copy_stream = torch.cuda.Stream(device=device)
+        landed = [torch.cuda.Event() for _ in range(2)]       # staging buffer holds worker w's gradient
+        taken = [torch.cuda.Event() for _ in range(2)]        # the encode that read it has finished
+        main = torch.cuda.current_stream(device)
 
         def e2e_step(i):
+            # the copy of worker w + 1 (copy stream) overlaps the encode of worker w (main stream)
             for code in hp.codes:
                 for w in range(K):
-                    buf = stage[w & 1]
-                    buf.copy_(pinned[w], non_blocking=True)
-                    Q.qsgd_encode(buf, hp.d, hp.s, hp.norm, code, PHILOX_SEED, i, w, hp.msgs[code][w],
+                    b = w & 1
+                    with torch.cuda.stream(copy_stream):
+                        copy_stream.wait_event(taken[b])
+                        stage[b].copy_(pinned[w], non_blocking=True)
+                        landed[b].record(copy_stream)
+                    main.wait_event(landed[b])
+                    Q.qsgd_encode(stage[b], hp.d, hp.s, hp.norm, code, PHILOX_SEED, i, w, hp.msgs[code][w],
                                   hp.bits[code][w], hp.ws[code], hp.status)
-                tables = hp.resolve_tables(code)
-                Q.qsgd_decode_sgd_step(hp.msgs[code], tables, hp.n, hp.d, hp.s, code, hp.x, ETA, hp.status)
+                    taken[b].record(main)
+                hp.decode(code)
                 x_host.copy_(hp.x, non_blocking=True)
             torch.cuda.synchronize()
 
@@ -430,13 +449,16 @@ def run_cuda(args):
         e2e_ms = float(t.item()) / e2e_steps
         e2e = {"value": grad_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": e2e_ms,
                "steps": e2e_steps, "h2d_bytes_per_step": len(hp.codes) * K * 4 * n,
-               "d2h_bytes_per_step": len(hp.codes) * (4 * n + 32 * K * (1 if 1 in hp.codes else 0))}
+               "d2h_bytes_per_step": len(hp.codes) * 4 * n,
+               "overlap": "H2D copy of worker w+1 on a second stream under the encode of worker w"}
         del pinned, x_host, stage
 
     # ---- CPU baseline: the oracle on a bounded sample -----------------------------------------
     cpu = None
     if rank == 0 and not args.no_cpu:
         cpu = run_oracle_sample(wl, steps=1)
+        cpu["host_cores"] = os.cpu_count()
+        cpu["all_cores"] = run_oracle_parallel(wl)
 
     if rank == 0:
         line = {
@@ -447,7 +469,8 @@ def run_cuda(args):
             "config": {"workload": args.workload + ": " + wl["desc"], "n": n, "bucket": hp.d, "s": hp.s,
                        "norm": wl["norm"], "codes": wl["codes"], "K": K,
                        "l2": "inputs larger than L2 (K gradients = %.0f MB rotate through 126 MB)" % (K * 4 * n / 1e6),
-                       "step": "per code kind: K encodes, message-size read-back (Elias), fused decode+aggregate+SGD"},
+                       "step": "per code kind: K encodes, fused decode+aggregate+SGD (tables found on the device; "
+                               "no host read-back inside a step)"},
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "roofline": roofline, "cpu_baseline": cpu, "phases": phases, "kernels": kern_tab,
         }
@@ -547,9 +570,12 @@ def run_sweep(args):
         "points": points}))
 
 
-def run_exchange(args):
-    """Algorithm 1 across GPUs: rank = worker. Per step and code kind: encode the local gradient,
-    all-gather the K = world-size messages over NCCL, fused decode + aggregate + SGD step."""
+def run_multi(args):
+    """Algorithm 1 across GPUs, K workers on N ranks (N divides K): rank r plays workers
+    r * K / N ... and, per step and code kind, encodes their gradients into its slots, all-gathers
+    the K messages (NCCL; they land in this GPU's own memory) and runs the same fused decode +
+    aggregate + SGD step over all K as the one-GPU bench does. Beside it, timed the same way, the
+    uncompressed arm: local sum of the rank's gradients, fp32 all-reduce, plain step."""
     import torch
     import torch.distributed as dist
     import paper_1610_02132_b200 as Q
@@ -560,65 +586,123 @@ def run_exchange(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
     os.environ.setdefault("MASTER_PORT", "29533")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
     dist.init_process_group("nccl", rank=rank, world_size=world, device_id=device)
     wl = dict(WORKLOADS[args.workload])
-    for k in ("n", "d", "s"):
+    for k in ("n", "d", "s", "K"):
         if getattr(args, k) is not None:
             wl[k] = getattr(args, k)
+    if args.norm:
+        wl["norm"] = args.norm
     if args.codes:
         wl["codes"] = args.codes.split(",")
-    n, d, s, K = wl["n"], wl["d"], wl["s"], world
-    norm = NORM[args.norm or wl["norm"]]
-    g = device_gradient(wl, rank, device)
+    if wl.get("policy"):
+        raise SystemExit("the per-tensor policy workloads run on one GPU")
+    n, d, s, K = wl["n"], wl["d"], wl["s"], wl["K"]
+    if K % world:
+        raise SystemExit("--gpus %d must divide the workload's K = %d workers" % (world, K))
+    W = K // world
+    norm = NORM[wl["norm"]]
+    B = (n + d - 1) // d
+    g = [device_gradient(wl, rank * W + w, device) for w in range(W)]
     x = torch.zeros(n, dtype=torch.float32, device=device)
+    x_ref = torch.zeros(n, dtype=torch.float32, device=device)
+    gsum = torch.empty(n, dtype=torch.float32, device=device)
     status = Q.new_status(device)
-    bufs = {}
+    ex, ws = {}, {}
     for cname in wl["codes"]:
         code = CODE[cname]
         cap = Q.qsgd_message_capacity(n, d, s, code)
-        if code != 0:
-            cap = min(cap, 2 * fixed_bytes(n, d, s) + 8 * ((n + d - 1) // d + 1))
-        cap = X.slot_bytes(cap)
-        bufs[code] = (torch.zeros(cap, dtype=torch.uint8, device=device),
-                      torch.zeros(4, dtype=torch.int64, device=device),
-                      torch.empty(max(Q.qsgd_workspace_bytes(n, d, s, code), 16), dtype=torch.uint8, device=device))
+        if code != 0:        # an Elias message longer than twice the fixed-width one is not worth sending
+            cap = min(cap, 2 * fixed_bytes(n, d, s) + 8 * (B + 1))
+        ex[code] = X.Exchange(cap, W, device)
+        ws[code] = torch.empty(max(Q.qsgd_workspace_bytes(n, d, s, code), 16), dtype=torch.uint8, device=device)
+    exact = not args.capacity_slots
 
     def step(i):
         for cname in wl["codes"]:
             code = CODE[cname]
-            out, info, ws = bufs[code]
-            Q.qsgd_encode(g, d, s, norm, code, PHILOX_SEED, i, rank, out, info, ws, status)
-            msgs, tables, _ = X.exchange(out, info, n, d, code != 0, fixed_bytes=fixed_bytes(n, d, s))
-            Q.qsgd_decode_sgd_step(msgs, tables, n, d, s, code, x, ETA, status)
+            e = ex[code]
+            for w in range(W):
+                out, info = e.local_slot(w)
+                Q.qsgd_encode(g[w], d, s, norm, code, PHILOX_SEED, i, rank * W + w, out, info, ws[code], status)
+            msgs, infos, nbytes = e.run(exact=exact and code != 0, with_info=code != 0)
+            Q.qsgd_decode_sgd_step_packed(msgs, infos if code != 0 else None, n, d, s, code, x, ETA, status,
+                                          msg_bytes=nbytes)
+
+    def step_allreduce():
+        for _ in wl["codes"]:
+            torch.add(g[0], g[1], out=gsum) if W > 1 else gsum.copy_(g[0])
+            for w in range(2, W):
+                gsum.add_(g[w])
+            dist.all_reduce(gsum)
+            x_ref.add_(gsum, alpha=-ETA / K)
+
+    def timed(fn, steps):
+        dist.barrier(); torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for i in range(steps):
+            fn(i)
+        ev1.record()
+        dist.barrier(); torch.cuda.synchronize()
+        t = torch.tensor([ev0.elapsed_time(ev1)], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item()) / steps
 
     for i in range(args.warmup):
         step(i)
-    dist.barrier(); torch.cuda.synchronize()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        step_allreduce()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
     l0 = Q.qsgd_launch_count()
-    ev0.record()
-    for i in range(args.steps):
-        step(args.warmup + i)
-    ev1.record()
-    dist.barrier(); torch.cuda.synchronize()
-    t = torch.tensor([ev0.elapsed_time(ev1)], dtype=torch.float64, device=device)
-    dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    assert int(status.item()) == 0
-    ms_step = float(t.item()) / args.steps
-    grad_bytes = len(wl["codes"]) * (world * 4 * n + world * K * 4 * n)
+    ms_step = timed(lambda i: step(args.warmup + i), args.steps)
+    launches = Q.qsgd_launch_count() - l0
+    clocks = sampler.stop() if rank == 0 else None
+    ms_allreduce = timed(lambda i: step_allreduce(), args.steps)
+    assert int(status.item()) == 0, "device status %d" % int(status.item())
+    sizes = {c: ex[CODE[c]].infos[:, 2].double().mean().item() if CODE[c] != 0 else float(fixed_bytes(n, d, s))
+             for c in wl["codes"]}
+    # fp32 gradient bytes through Encode (each worker once) plus through Decode (all K on every rank)
+    grad_bytes = len(wl["codes"]) * (K * 4 * n + world * K * 4 * n)
     if rank == 0:
         print(json.dumps({
             "metric": "QSGD encode + decode+aggregate throughput, fp32 gradient GB/s",
             "value": grad_bytes / (ms_step * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": args.workload + " (exchange): " + wl["desc"], "n": n, "bucket": d, "s": s,
-                       "norm": args.norm or wl["norm"], "codes": wl["codes"], "K": K,
-                       "parallelism": "rank = worker, NCCL all-gather of messages"},
-            "gpu_launches": int(Q.qsgd_launch_count() - l0)}))
+            "config": {"workload": args.workload + ": " + wl["desc"], "n": n, "bucket": d, "s": s,
+                       "norm": wl["norm"], "codes": wl["codes"], "K": K,
+                       "parallelism": "rank plays K/N = %d workers; NCCL all-gather of the K messages into local "
+                                      "memory; every rank decodes all K" % W,
+                       "slots": "exact (one 32-byte-per-message read-back per Elias exchange)" if exact
+                                else "capacity (no host synchronisation)",
+                       "l2": "inputs larger than L2 between steps"},
+            "gpu_launches": int(launches), "clocks": clocks,
+            "message_bytes": sizes,
+            "allreduce_fp32": {"ms_per_step": ms_allreduce, "what": "per code kind: local sum of the rank's "
+                               "gradients, dist.all_reduce of n fp32 values, x -= (eta/K) sum",
+                               "speedup_of_qsgd_step": ms_allreduce / ms_step}}))
     dist.destroy_process_group()
+
+
+def spawn_ranks(n_gpus):
+    """`python bench.py --gpus N` without a launcher: start N ranks on this node, one per GPU."""
+    import socket
+    sock = socket.socket()
+    sock.bind(("127.0.0.1", 0))
+    port = sock.getsockname()[1]
+    sock.close()
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "VERSION")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n_gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd, env=env))
 
 
 # ------------------------------------------------------------------------------------------------
@@ -664,6 +748,41 @@ def run_oracle_sample(wl, steps=1, workers=2):
             "seconds": t_total,
             "sample": "%d of %d workers, first %d of %d coordinates, codes %s, %d step(s)" % (
                 workers, wl["K"], n, wl["n"], ",".join(wl["codes"]), steps)}
+
+
+def run_oracle_parallel(wl, n_cap=2 ** 23):
+    """Second CPU figure: min(K, host cores) independent oracle instances, one thread each (the
+    oracle itself is single-threaded; its C calls release the interpreter lock). An instance encodes
+    one worker's gradient (first n_cap coordinates) under every code kind of the workload and decodes
+    that message into a step."""
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import oracle as O
+    if wl.get("policy"):
+        return None
+    T = max(1, min(wl["K"], os.cpu_count() or 1))
+    n = min(wl["n"], n_cap)
+    n -= n % wl["d"] if n > wl["d"] else 0
+    d, s, norm = wl["d"], wl["s"], NORM[wl["norm"]]
+    gs = [host_gradient(wl, w, n) for w in range(T)]
+
+    def instance(w):
+        x = np.zeros(n, dtype=np.float32)
+        for code_name in wl["codes"]:
+            code = CODE[code_name]
+            m, info = O.encode(gs[w], d, s, norm, code, PHILOX_SEED, 0, w)
+            tabs = None if code == 0 else [O.message_table(m, info, n, d)]
+            st, acc = O.decode_accumulate([m], tabs, n, d, s, code)
+            x = O.sgd_step(x, acc, ETA, 1)
+        return x[0]
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(T) as pool:
+        list(pool.map(instance, range(T)))
+    dt = time.perf_counter() - t0
+    return {"value": T * len(wl["codes"]) * 2 * 4 * n / dt / 1e9, "unit": "GB/s", "cores": T,
+            "host_cores": os.cpu_count(), "kind": "oracle, %d independent instances on %d threads" % (T, T),
+            "seconds": dt, "sample": "each instance: 1 worker, first %d of %d coordinates, codes %s" % (
+                n, wl["n"], ",".join(wl["codes"]))}
 
 
 def run_qsvrg(args):
@@ -750,9 +869,12 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--exchange", action="store_true",
-                    help="rank = worker: encode own gradient, NCCL all-gather of the messages, decode all "
-                         "K = world-size messages (Algorithm 1 across GPUs) instead of independent replicas")
+    ap.add_argument("--replicas", action="store_true",
+                    help="with more than one GPU: independent replicas of the one-GPU workload (no collective) "
+                         "instead of Algorithm 1 across the GPUs")
+    ap.add_argument("--capacity-slots", action="store_true",
+                    help="multi-GPU: all-gather whole capacity slots (no host synchronisation) instead of slots "
+                         "cut to the longest message of the step")
     ap.add_argument("--capture", action="store_true",
                     help="for runs under a profiler: keep --warmup as given, skip e2e and the CPU baseline")
     args = ap.parse_args()
@@ -760,6 +882,9 @@ def main():
         args.steps = 1 if args.steps is None else min(args.steps, 4)
         run_reference(args)
         return
+    world = int(os.environ.get("WORLD_SIZE", "0"))
+    if world == 0 and args.gpus > 1:
+        spawn_ranks(args.gpus)
     if args.steps is None:
         args.steps = 10
     if args.capture:
@@ -770,8 +895,8 @@ def main():
         run_sweep(args)
     elif args.workload == "qsvrg":
         run_qsvrg(args)
-    elif args.exchange:
-        run_exchange(args)
+    elif max(world, 1) > 1 and not args.replicas:
+        run_multi(args)
     else:
         run_cuda(args)
 

@@ -1,11 +1,18 @@
-"""Message exchange for the data-parallel step of Algorithm 1 ("broadcast M^i to all peers"):
-rank = worker, every rank contributes one encoded message and receives all K of them.
+"""Message exchange for the data-parallel step of Algorithm 1 ("broadcast M^i to all peers",
+"receive M^l"): every rank contributes the messages of the workers it plays and receives all K.
 
 Only plumbing lives here (torch.distributed collectives and slot arithmetic); encoding and
-decoding stay in the kernels. Fixed-width messages all have the same, statically known size, so
-one all-gather into a K-slot buffer suffices. Elias messages differ in length: the ranks first
-all-gather their four info words, then all-gather the messages padded to the longest one. The
-gathered slots sit in this GPU's own memory before any decode kernel reads them.
+decoding stay in the kernels. A rank encodes its W workers' messages into W slots of one buffer
+(slot pitch = the message capacity rounded up to SLOT_ALIGN); one all-gather puts the K = world * W
+slots, in worker order, into this GPU's own memory, and a second small all-gather does the same
+for the four info words of each message. The decode entry points of the packed form
+(qsgd_decode_*_packed) take exactly that: slot pointers, info-word pointers and the slot pitch as
+the readable size; they find each offset table on the device, so the exchange needs no host
+synchronisation at all.
+
+Elias messages are shorter than their capacity. `exact=True` sends only as many bytes per slot
+as the longest message of the step needs; that costs one host read-back of the gathered sizes
+(32 bytes per message), which a sender of variable-length messages cannot avoid.
 """
 import torch
 import torch.distributed as dist
@@ -18,53 +25,45 @@ def slot_bytes(max_message_bytes):
     return (int(max_message_bytes) + SLOT_ALIGN - 1) // SLOT_ALIGN * SLOT_ALIGN
 
 
-def gather_info(info, group=None):
-    """All-gathers the per-rank info words (int64[4]: payload bits, table offset, message bytes,
-    0). Returns an int64 tensor [K, 4] on the same device."""
-    world = dist.get_world_size(group)
-    out = torch.empty(world, 4, dtype=torch.int64, device=info.device)
-    dist.all_gather_into_tensor(out.view(-1), info.contiguous().view(-1), group=group)
-    return out
+class Exchange:
+    """Buffers of one rank for a fixed message capacity: W local slots, K gathered slots, the info
+    words of both. Allocated once; every step reuses them (slot and info addresses stay put, so a
+    step's launches can be replayed)."""
 
+    def __init__(self, capacity, workers_per_rank, device, group=None):
+        self.group = group
+        self.world = dist.get_world_size(group)
+        self.W = int(workers_per_rank)
+        self.K = self.world * self.W
+        self.pitch = slot_bytes(capacity)
+        self.local = torch.zeros(self.W * self.pitch, dtype=torch.uint8, device=device)
+        self.local_info = torch.zeros(self.W, 4, dtype=torch.int64, device=device)
+        self.gathered = torch.zeros(self.K * self.pitch, dtype=torch.uint8, device=device)
+        self.infos = torch.zeros(self.K, 4, dtype=torch.int64, device=device)
+        self._exact = None
 
-def gather_messages(msg, pitch, group=None, out=None):
-    """All-gathers one message per rank into K slots of `pitch` bytes. `msg` is a uint8 tensor
-    holding at least `pitch` bytes (bytes past the message length are transmitted but ignored)."""
-    world = dist.get_world_size(group)
-    if msg.numel() < pitch:
-        raise ValueError("message buffer shorter than the slot pitch")
-    if out is None:
-        out = torch.empty(world * pitch, dtype=torch.uint8, device=msg.device)
-    dist.all_gather_into_tensor(out, msg[:pitch].contiguous(), group=group)
-    return out
+    def local_slot(self, w):
+        """Message buffer of local worker w (encode into this), and its info words."""
+        return self.local[w * self.pitch: (w + 1) * self.pitch], self.local_info[w]
 
-
-def slots(gathered, pitch, infos, n, bucket, elias):
-    """Per-rank views into the gathered buffer: (messages, tables). tables is None for the
-    fixed-width code; for the Elias codes table k starts at byte infos[k][1] of slot k."""
-    world = infos.shape[0]
-    B = (n + bucket - 1) // bucket
-    msgs, tables = [], []
-    info_host = infos.cpu().tolist()
-    for k in range(world):
-        base = k * pitch
-        total = int(info_host[k][2])
-        msgs.append(gathered[base: base + total])
-        if elias:
-            off = base + int(info_host[k][1])
-            tables.append(gathered[off: off + 8 * (B + 1)].view(torch.int64))
-    return msgs, (tables if elias else None)
-
-
-def exchange(msg, info, n, bucket, elias, fixed_bytes=None, group=None):
-    """One exchange step. Returns (msgs, tables, infos) ready for the decode entry points."""
-    if elias:
-        infos = gather_info(info, group)
-        pitch = slot_bytes(int(infos[:, 2].max().item()))
-    else:
-        world = dist.get_world_size(group)
-        infos = info.view(1, 4).repeat(world, 1)          # same size on every rank
-        pitch = slot_bytes(fixed_bytes)
-    gathered = gather_messages(msg, pitch, group)
-    msgs, tables = slots(gathered, pitch, infos, n, bucket, elias)
-    return msgs, tables, infos
+    def run(self, exact=False, with_info=True):
+        """All-gathers the info words (Elias kinds need them; with_info=False skips it for the
+        fixed-width code) and the slots. Returns (msgs, infos, msg_bytes): K slot views in worker
+        order, K info-word views, and the readable bytes of each slot."""
+        if with_info or exact:
+            dist.all_gather_into_tensor(self.infos.view(-1), self.local_info.view(-1), group=self.group)
+        pitch = self.pitch
+        if exact:
+            pitch = min(slot_bytes(int(self.infos[:, 2].max().item())), self.pitch)    # the one host read-back
+        if pitch == self.pitch:
+            gathered = self.gathered
+            dist.all_gather_into_tensor(gathered, self.local, group=self.group)
+        else:
+            if self._exact is None or self._exact.numel() < self.K * pitch:
+                self._exact = torch.empty(self.K * pitch, dtype=torch.uint8, device=self.local.device)
+            gathered = self._exact[: self.K * pitch]
+            send = self.local.view(self.W, self.pitch)[:, :pitch].contiguous().view(-1)
+            dist.all_gather_into_tensor(gathered, send, group=self.group)
+        msgs = [gathered[k * pitch: (k + 1) * pitch] for k in range(self.K)]
+        infos = [self.infos[k] for k in range(self.K)]
+        return msgs, infos, [pitch] * self.K

@@ -1,7 +1,7 @@
-"""World-size-2 test of the message exchange (rank = worker) on CPU with the gloo backend: each
-rank encodes its own gradient (with the oracle, as there is no GPU here), the ranks exchange
-messages through paper_1610_02132_b200.exchange, every rank decodes all of them, and both must
-end with the same parameters as a single process that holds both messages."""
+"""World-size-2 test of the message exchange on CPU with the gloo backend: each rank encodes the
+gradients of the workers it plays (with the oracle, as there is no GPU here), the ranks exchange
+slots and info words through paper_1610_02132_b200.exchange, every rank decodes all K messages,
+and all must end with the same parameters as a single process that holds every message."""
 import os
 import socket
 import sys
@@ -23,59 +23,68 @@ def _free_port():
     return port
 
 
-def _worker(rank, world, port, code_kind, n, d, s, result_dir):
+def _worker(rank, world, port, code_kind, n, d, s, W, exact, result_dir):
     sys.path.insert(0, ROOT)
     os.environ["MASTER_ADDR"] = "127.0.0.1"
     os.environ["MASTER_PORT"] = str(port)
     dist.init_process_group("gloo", rank=rank, world_size=world)
     from oracle import oracle as O
     from paper_1610_02132_b200 import exchange as X, inputs as I
-    g = I.gaussian_mixture(n, seed=1 + rank)
-    m, info = O.encode(g, d, s, O.NORM_L2, code_kind, 7, 0, rank)
     elias = code_kind != O.CODE_FIXED
-    cap = O.message_capacity(n, d, s, code_kind) + X.SLOT_ALIGN
-    buf = torch.zeros(cap, dtype=torch.uint8)
-    buf[: m.size] = torch.from_numpy(m)
-    info_t = torch.tensor(info, dtype=torch.int64)
-    msgs, tables, infos = X.exchange(buf, info_t, n, d, elias, fixed_bytes=info[2])
-    assert len(msgs) == world and infos.shape == (world, 4)
-    assert torch.equal(msgs[rank], torch.from_numpy(m))                 # own slot holds own message
-    msgs_np = [x.numpy() for x in msgs]
-    tabs_np = None if tables is None else [t.numpy().view(np.uint64) for t in tables]
-    st, acc = O.decode_accumulate(msgs_np, tabs_np, n, d, s, code_kind)
+    ex = X.Exchange(O.message_capacity(n, d, s, code_kind), W, torch.device("cpu"))
+    assert ex.K == world * W and ex.pitch % X.SLOT_ALIGN == 0
+    mine = []
+    for w in range(W):
+        worker = rank * W + w
+        m, info = O.encode(I.gaussian_mixture(n, seed=1 + worker), d, s, O.NORM_L2, code_kind, 7, 0, worker)
+        buf, iw = ex.local_slot(w)
+        buf[: m.size] = torch.from_numpy(m)
+        iw.copy_(torch.tensor(info, dtype=torch.int64))
+        mine.append(m)
+    msgs, infos, nbytes = ex.run(exact=exact, with_info=elias)
+    assert len(msgs) == ex.K and len(infos) == ex.K and len(nbytes) == ex.K
+    if exact:
+        assert nbytes[0] <= ex.pitch and nbytes[0] % X.SLOT_ALIGN == 0
+    for w in range(W):                                                   # own slots hold own messages
+        k = rank * W + w
+        assert torch.equal(msgs[k][: mine[w].size], torch.from_numpy(mine[w]))
+    msgs_np, tabs_np = [], []
+    for k in range(ex.K):
+        total = int(infos[k][2]) if elias else O.message_capacity(n, d, s, code_kind)
+        assert total <= nbytes[k]
+        m = msgs[k][:total].numpy()
+        msgs_np.append(m)
+        if elias:
+            info = [int(v) for v in infos[k]]
+            tabs_np.append(O.message_table(m, info, n, d))
+    st, acc = O.decode_accumulate(msgs_np, tabs_np if elias else None, n, d, s, code_kind)
     assert st == 0
-    x = O.sgd_step(np.zeros(n, np.float32), acc, 0.1, world)
+    x = O.sgd_step(np.zeros(n, np.float32), acc, 0.1, ex.K)
     np.save(os.path.join(result_dir, "x%d.npy" % rank), x)
     dist.barrier()
     dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("code_kind", [0, 1])
-def test_two_rank_exchange_matches_single_process(tmp_path, code_kind):
+@pytest.mark.parametrize("code_kind,W,exact", [(0, 1, False), (1, 1, False), (1, 2, True), (2, 1, True), (0, 2, False)])
+def test_two_rank_exchange_matches_single_process(tmp_path, code_kind, W, exact):
     sys.path.insert(0, ROOT)
     from oracle import oracle as O
     from paper_1610_02132_b200 import inputs as I
     n, d, s, world = 5000, 512, 15, 2
     port = _free_port()
-    mp.spawn(_worker, args=(world, port, code_kind, n, d, s, str(tmp_path)), nprocs=world, join=True)
+    mp.spawn(_worker, args=(world, port, code_kind, n, d, s, W, exact, str(tmp_path)), nprocs=world, join=True)
     msgs, tabs = [], []
-    for w in range(world):
+    for w in range(world * W):
         m, info = O.encode(I.gaussian_mixture(n, seed=1 + w), d, s, O.NORM_L2, code_kind, 7, 0, w)
         msgs.append(m)
         tabs.append(None if code_kind == 0 else O.message_table(m, info, n, d))
     st, acc = O.decode_accumulate(msgs, None if code_kind == 0 else tabs, n, d, s, code_kind)
-    ref = O.sgd_step(np.zeros(n, np.float32), acc, 0.1, world)
-    for w in range(world):
-        x = np.load(os.path.join(str(tmp_path), "x%d.npy" % w))
+    ref = O.sgd_step(np.zeros(n, np.float32), acc, 0.1, world * W)
+    for r in range(world):
+        x = np.load(os.path.join(str(tmp_path), "x%d.npy" % r))
         assert np.array_equal(x.view(np.uint32), ref.view(np.uint32))
 
 
 def test_slot_arithmetic():
     from paper_1610_02132_b200 import exchange as X
     assert X.slot_bytes(1) == 256 and X.slot_bytes(256) == 256 and X.slot_bytes(257) == 512
-    infos = torch.tensor([[100, 16, 16 + 8 * 3, 0], [70, 16, 16 + 8 * 3, 0]], dtype=torch.int64)
-    pitch = X.slot_bytes(40)
-    buf = torch.arange(2 * pitch, dtype=torch.int64).to(torch.uint8)
-    msgs, tables = X.slots(buf, pitch, infos, n=64, bucket=32, elias=True)
-    assert msgs[1].data_ptr() - buf.data_ptr() == pitch and msgs[0].numel() == 40
-    assert tables[1].data_ptr() - buf.data_ptr() == pitch + 16 and tables[0].numel() == 3
