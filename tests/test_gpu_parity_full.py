@@ -1,8 +1,10 @@
-"""GPU parity at the full BASELINE sizes, in the launch configuration bench.py times. Small
-configs are compared whole; the 60M-coordinate and 2^28-coordinate configs are compared on
-sampled buckets (first, last / tail, and random ones) that the oracle recomputes one by one from
-the same gradient bytes, plus properties that hold at any size (fused == unfused, table
-arithmetic, code-length bound)."""
+"""GPU parity at the full sizes of the five workloads, in the launch configuration bench.py times.
+The small configs are compared whole. The two 60M-coordinate model-shaped configs are compared
+whole as well -- the complete messages of the first and the last worker against the oracle's
+encoder, and the complete stepped x against the oracle's decoder over all K messages -- and, like
+the 2^28-coordinate sweep points, on sampled buckets (first, last / tail, and random ones) that
+the oracle recomputes one by one from the same gradient bytes, plus properties that hold at any
+size (fused == unfused, table arithmetic, code-length bound)."""
 import math
 
 import numpy as np
@@ -13,7 +15,7 @@ import paper_1610_02132_b200 as Q
 from oracle import oracle as O
 from paper_1610_02132_b200 import inputs as I
 
-from parity_util import decode_parity, encode_parity, gpu_encode, table_view
+from parity_util import check_scales, decode_parity, encode_parity, gpu_encode, scales_from_message, table_view
 
 pytestmark = pytest.mark.gpu
 
@@ -124,6 +126,60 @@ def run_sampled_config(gs, n, d, s, norm_kind, code_kind, step, nsample, eta=0.1
         xr = O.sgd_step(x0[lo:hi].cpu().numpy(), ref, eta, K)
         assert np.array_equal(x_fus[lo:hi].cpu().numpy().view(np.uint32), xr.view(np.uint32)), b
     return infos
+
+
+def run_whole_config(gs, n, d, s, norm_kind, code_kind, step, eta=0.1):
+    """Whole-message, whole-vector compare at full size: every byte of the first and the last
+    worker's message equals the oracle's encoding (given the GPU's scales, which are checked
+    against the oracle's fp64 norms), and every coordinate of the fused step over all K messages
+    equals the oracle's decode + aggregate + step of those messages."""
+    K = len(gs)
+    B = O.n_buckets(n, d)
+    cap = min(Q.qsgd_message_capacity(n, d, s, code_kind),
+              2 * Q.qsgd_message_capacity(n, d, s, O.CODE_FIXED) + 8 * (B + 1))
+    msgs, infos = [], []
+    for w in range(K):
+        big, info, st, _ = gpu_encode(gs[w], d, s, norm_kind, code_kind, SEED, step, w, capacity=cap)
+        assert st == 0
+        msgs.append(big[: info[2]])
+        infos.append(info)
+    for w in (0, K - 1):
+        g = gs[w].cpu().numpy()
+        msg = msgs[w].cpu().numpy()
+        A_gpu = scales_from_message(msg, infos[w], n, d, s, code_kind)
+        check_scales(A_gpu, g, d, norm_kind)
+        ref, ref_info = O.encode(g, d, s, norm_kind, code_kind, SEED, step, w, A_ext=A_gpu)
+        assert infos[w] == ref_info
+        assert np.array_equal(msg, ref), "message of worker %d differs from the oracle's" % w
+        del g, ref
+    x0 = I.gaussian_device(n, 1.0, seed=99)
+    x = x0.clone()
+    status = Q.new_status()
+    info_dev = [torch.tensor(i, dtype=torch.int64, device="cuda") for i in infos]
+    Q.qsgd_decode_sgd_step_packed(msgs, None if code_kind == O.CODE_FIXED else info_dev, n, d, s, code_kind, x, eta,
+                                  status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    msgs_np = [m.cpu().numpy() for m in msgs]
+    tabs = None if code_kind == O.CODE_FIXED else [O.message_table(m, i, n, d) for m, i in zip(msgs_np, infos)]
+    st, acc = O.decode_accumulate(msgs_np, tabs, n, d, s, code_kind)
+    assert st == 0
+    x_ref = O.sgd_step(x0.cpu().numpy(), acc, eta, K)
+    assert np.array_equal(x.cpu().numpy().view(np.uint32), x_ref.view(np.uint32)), "stepped x differs from the oracle's"
+
+
+def test_config3_alexnet_whole():
+    shapes = I.alexnet_shapes()
+    n = I.numel(shapes)
+    gs = [I.layered_gaussian_device(shapes, seed=1 + w) for w in range(16)]
+    run_whole_config(gs, n, 512, 255, O.NORM_MAX, O.CODE_FIXED, step=0)
+
+
+@pytest.mark.parametrize("code_kind", [O.CODE_FIXED, O.CODE_ELIAS])
+def test_config4_resnet152_whole(code_kind):
+    n = I.numel(I.resnet152_shapes())
+    gs = [I.gaussian_mixture_device(n, seed=1 + w) for w in range(16)]
+    run_whole_config(gs, n, 512, 15, O.NORM_L2, code_kind, step=0)
 
 
 def test_config1_tiny_whole():
