@@ -21,7 +21,8 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kChunk = 512;            // coordinates per warp iteration
 
 struct DecodeParams {
-  PeerSet peers;
+  const uint8_t* msg[QSGD_MAX_PEERS];   // the K messages; all share one layout, so the three regions
+  uint64_t off_sign, off_level;         // of every message sit at the same byte offsets
   uint32_t K;
   uint64_t n;
   uint32_t d;
@@ -32,6 +33,10 @@ struct DecodeParams {
   uint64_t chunks;
   BucketMap map;
 };
+
+// Peers per unrolled group of the k loop: enough loads in flight to cover their latency, few
+// enough that the 16 running sums and the group's words stay in registers (measured per width).
+template <int LB> struct PeerUnroll { static constexpr int value = LB == 1 ? 3 : 4; };
 
 template <int LB, bool FUSED, bool SINGLE>
 __global__ void __launch_bounds__(kThreads, 4) decode_fixed_kernel(const __grid_constant__ DecodeParams p) {
@@ -57,24 +62,28 @@ __global__ void __launch_bounds__(kThreads, 4) decode_fixed_kernel(const __grid_
 #pragma unroll
     for (int e = 0; e < 16; ++e) acc[e] = 0.f;
 
-#pragma unroll 8
+    // byte offsets of this lane's scale, 16 sign bits and 16 level fields inside any message
+    const uint64_t slot = i0 >> 4;
+    const uint64_t off_a = 4ull * b, off_s = p.off_sign + 2ull * slot, off_l = p.off_level + (uint64_t)(2 * LB) * slot;
+#pragma unroll PeerUnroll<LB>::value
     for (uint32_t k = 0; k < p.K; ++k) {
       uint32_t w[4] = {0u, 0u, 0u, 0u};
       uint32_t sb = 0;
       float A = 0.f;
       if (live) {
-        A = __ldg(p.peers.A[k] + b);
-        sb = __ldg(reinterpret_cast<const uint16_t*>(p.peers.sign[k]) + (i0 >> 4));
+        const uint8_t* m = p.msg[k];
+        A = __ldg(reinterpret_cast<const float*>(m + off_a));
+        sb = __ldg(reinterpret_cast<const uint16_t*>(m + off_s));
         if (LB == 8) {
-          const uint4 t = __ldg(reinterpret_cast<const uint4*>(p.peers.level[k]) + (i0 >> 4));
+          const uint4 t = __ldg(reinterpret_cast<const uint4*>(m + off_l));
           w[0] = t.x; w[1] = t.y; w[2] = t.z; w[3] = t.w;
         } else if (LB == 4) {
-          const uint2 t = __ldg(reinterpret_cast<const uint2*>(p.peers.level[k]) + (i0 >> 4));
+          const uint2 t = __ldg(reinterpret_cast<const uint2*>(m + off_l));
           w[0] = t.x; w[1] = t.y;
         } else if (LB == 2) {
-          w[0] = __ldg(p.peers.level[k] + (i0 >> 4));
+          w[0] = __ldg(reinterpret_cast<const uint32_t*>(m + off_l));
         } else {
-          w[0] = __ldg(reinterpret_cast<const uint16_t*>(p.peers.level[k]) + (i0 >> 4));
+          w[0] = __ldg(reinterpret_cast<const uint16_t*>(m + off_l));
         }
       }
       if (LB == 8) add_peer_tab(acc, w, sb, tab_lane, A);
@@ -136,7 +145,10 @@ int launch_lb(const DecodeParams& p, bool fused, bool single, cudaStream_t strea
 int launch_decode_fixed(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d, uint32_t s,
                         float* acc_or_x, bool fused, float eta, const BucketMap& map, cudaStream_t stream) {
   DecodeParams p;
-  p.peers = peers; p.K = K; p.n = n; p.d = d; p.s = s; p.out = acc_or_x; p.map = map;
+  const FixedLayout L = make_fixed_layout(n, d, s);
+  for (uint32_t k = 0; k < K; ++k) p.msg[k] = reinterpret_cast<const uint8_t*>(peers.A[k]);   // the scales open a message
+  p.off_sign = L.off_sign; p.off_level = L.off_level;
+  p.K = K; p.n = n; p.d = d; p.s = s; p.out = acc_or_x; p.map = map;
   p.c = eta / (float)K;
   p.chunks = (n + kChunk - 1) / kChunk;
   // one scale per chunk when the bucket size is 512 * 2^j

@@ -1,7 +1,6 @@
-// Decode-and-aggregate, Elias path, optionally fused with the SGD step (Section 3.1: "read off
-// 32 bits to construct the norm, then iteratively ... read off the positions and values of the
-// nonzeros"; Appendix A.2 decoder; Algorithm 1 for the sum and the step): the choice among the
-// decoders. Whole-bucket and ranged field rebuilding live in elias_decode_fields.cu, the
+// Decode-and-aggregate, Elias path, optionally fused with the SGD step (Section 3.1, end of
+// "Efficient Coding of Gradients": scale first, then the codes of the nonzeros in index order;
+// Appendix A.2 decoder; Algorithm 1 for the sum and the step): the choice among the decoders. Whole-bucket and ranged field rebuilding live in elias_decode_fields.cu, the
 // nonzero-driven decoder of the sparse regime in elias_decode_sparse.cu, the general fallback in
 // elias_decode_slow.cu; what they share is in elias_decode.cuh.
 #include "elias_decode.cuh"

@@ -130,6 +130,7 @@ struct FieldParams {
   uint32_t* status;
   uint32_t row_words;   // per peer row: d * lb / 32 level words, then d / 32 sign words (padded to 4)
   uint32_t bucket_words;  // K rows + K scales, padded to 4
+  uint32_t range;         // byte-code decoder: positions per range
   uint32_t defer_sparse;  // a sparse-regime kernel was launched beside this one
   BucketMap map;          // where the buckets live in `out` (per-tensor policy), or no map
 };

@@ -1,6 +1,7 @@
-// Decode-and-aggregate, Elias path, optionally fused with the SGD step (Section 3.1: "read off
-// 32 bits to construct the norm, then iteratively ... read off the positions and values of the
-// nonzeros"; Appendix A.2 decoder; Algorithm 1 for the sum and the step).
+// Decode-and-aggregate, Elias path, optionally fused with the SGD step (Section 3.1, end of
+// "Efficient Coding of Gradients": the receiver takes the 32-bit scale off the front of a string and
+// then walks the (gap, sign, level) codes; Appendix A.2 for the integer decoder; Algorithm 1 for the
+// sum and the step).
 //
 // A string S can only be parsed front to back, but buckets and peers are independent once the
 // per-bucket offset table gives each string's first bit. A warp owns a group of G buckets.
@@ -405,8 +406,272 @@ int launch_ranged(FieldParams& p, bool fused, cudaStream_t stream, bool* handled
   return (int)cudaGetLastError();
 }
 
+// ------------------------------------------------------------------------------------------------
+// Byte-code decoder for s <= 15 (every field width up to 4 bits), Code_s, d < 1024, K <= 32. Same two
+// phases as above, with three changes that matter because this decoder is bound by shared-memory
+// traffic (table lookups, field writes, shuffles):
+//   * the parse writes one byte per nonzero coordinate -- level | negative << 4, which is the lane
+//     index of +-A * (level / s) in the shuffle table -- with a plain byte store: no read-modify-write
+//     of packed fields, and phase 2 feeds the bytes to the shuffles as they are, with no sign bits to
+//     merge into level fields;
+//   * a bucket is walked in ranges of 256 positions (a lane keeps its place in its string between
+//     ranges: bit window, position, one decoded entry that lies past the range), so the rows of one
+//     range are what sits in shared memory and twice as many warps are resident;
+//   * sign and level come from one lookup in a 256-entry table (the next 8 stream bits), and the
+//     per-entry checks are reduced to one comparison: an entry at or past min(range end, bucket
+//     length) is held back, and one that no range takes is a position error at the end.
+// Rows are kByteRange + 16 bytes apart so that lanes parsing different strings at similar positions
+// spread over the banks.
+// ------------------------------------------------------------------------------------------------
+constexpr uint32_t kRowPad = 16;
+constexpr uint32_t kByteRange = 256;
+
+// value | length << 8 of the Elias code that the 12 bits i start with, 0 when none is complete
+__device__ __forceinline__ uint32_t elias_table_entry(uint32_t i) {
+  uint32_t w = i << (32 - kLutBits), N = 1, used = 0;
+  bool ok = true;
+  for (int it = 0; it < 3 && (w >> 31); ++it) {
+    const uint32_t nb = N + 1;
+    if (used + nb > kLutBits) { ok = false; break; }
+    N = w >> (32 - nb);
+    w <<= nb;
+    used += nb;
+  }
+  ok = ok && !(w >> 31) && used + 1 <= kLutBits;
+  return ok ? (N | ((used + 1) << 8)) : 0u;
+}
+
+template <bool FUSED, bool SINGLE>
+__global__ void __launch_bounds__(512) decode_elias_bytes_kernel(const __grid_constant__ FieldParams p) {
+  extern __shared__ __align__(16) uint32_t fsm[];
+  __shared__ uint16_t elias_lut[1u << kLutBits];
+  __shared__ uint16_t level_lut[256];
+  if (p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const float sf = (float)p.s;
+  fill_elias_lut(elias_lut);
+  // sign + level in one lookup: entry i (the next 8 stream bits) = level | negative << 4 | length << 8 when
+  // the bits hold a sign and a complete code of a level <= min(s, 15), else 0
+  for (uint32_t i = tid; i < 256; i += blockDim.x) {
+    const uint32_t e = elias_table_entry((i & 0x7Fu) << 5);
+    const uint32_t level = e & 0xFFu, len = e >> 8;
+    level_lut[i] = (e && len <= 7u && level <= p.s && level <= 15u) ? (uint16_t)(level | ((i >> 7) << 4) | ((len + 1u) << 8))
+                                                                    : (uint16_t)0;
+  }
+  __syncthreads();
+  float lut0;
+  {
+    const uint32_t level = lane & 15u, neg = lane >> 4;
+    const float q = __fdiv_rn((float)level, sf);
+    lut0 = neg ? -q : q;
+  }
+  const uint32_t R = p.range;                                   // positions per range (multiple of 32)
+  const uint32_t row_bytes = R + kRowPad;
+  const uint32_t rows_bytes = p.G * p.K * row_bytes;            // per warp: G * K rows, then 32 scales
+  uint8_t* mine = reinterpret_cast<uint8_t*>(fsm) + (size_t)warp * (rows_bytes + 128u);
+  float* scales = reinterpret_cast<float*>(mine + rows_bytes);
+  const uint32_t pg = lane / p.Kpad, pk = lane % p.Kpad;      // parse role: bucket in group, peer
+  uint8_t* row = mine + (pg * p.K + pk) * row_bytes;           // this lane's row (when it parses)
+  const uint64_t groups = (p.B + p.G - 1) / p.G;
+  constexpr uint32_t kNone = 0xFFFFFFFFu;
+
+  for (uint64_t grp = (uint64_t)blockIdx.x * nwarps + warp; grp < groups; grp += (uint64_t)gridDim.x * nwarps) {
+    const uint64_t b0 = grp * p.G;
+    // ---- open this lane's string ---------------------------------------------------------------
+    BitSrc src;
+    uint32_t used = 0, total = 0, err = 0, at = 0xFFFFFFFFu, pend = kNone, db = 0;
+    float A = 0.f;
+    if (pg < p.G && b0 + pg < p.B) db = (uint32_t)min((uint64_t)p.d, p.n - (b0 + pg) * p.d);
+    const bool parsing = db != 0u && pk < p.K;
+    if (parsing) {
+      const StringRef ref = string_ref(p.peers, pk, b0 + pg, p.B, db);
+      err = ref.err;
+      if (!err) {
+        total = ref.total;
+        src.open(ref.words, ref.lo);
+        A = __uint_as_float(src.take(32));
+      }
+    }
+    scales[lane] = A;
+    bool readable = parsing && err == 0u;
+
+    for (uint32_t rbeg = 0; rbeg < p.d; rbeg += R) {
+      const uint32_t rend = min(rbeg + R, p.d);
+      for (uint32_t q = lane; q < (rows_bytes >> 4); q += 32) reinterpret_cast<uint4*>(mine)[q] = make_uint4(0u, 0u, 0u, 0u);
+      __syncwarp();
+      // ---- phase 1: this lane's nonzeros of the range, one byte each ----------------------------
+      if (readable) {
+        const uint32_t lim = min(rend, db);                 // entries at or past it wait (or are errors)
+        if (pend != kNone && (pend & 0xFFFFu) < lim) {
+          row[(pend & 0xFFFFu) - rbeg] = (uint8_t)(pend >> 16);
+          pend = kNone;
+        }
+        if (pend == kNone) {
+          while (used < total) {
+            src.refill();                                   // >= 33 bits: a table-decoded triple takes <= 20
+            uint32_t gap, l1 = 0, code, l2 = 0;
+            const uint32_t e1 = elias_lut[src.hi >> (32 - kLutBits)];
+            if (e1) {
+              gap = e1 & 0xFFu;
+              l1 = e1 >> 8;
+            } else {
+              if (!src.elias(gap, used)) { err = QSGD_DEV_OVERRUN; break; }
+              src.refill();
+            }
+            const uint32_t e2 = level_lut[__funnelshift_lc(src.lo, src.hi, l1) >> 24];
+            if (e2) {
+              code = e2;                                    // the byte store keeps level | negative << 4
+              l2 = e2 >> 8;
+            } else {
+              src.drop(l1);
+              used += l1;
+              l1 = 0;
+              const uint32_t neg = src.hi >> 31;
+              src.drop(1);
+              used += 1;
+              uint32_t level;
+              if (!src.elias(level, used)) { err = QSGD_DEV_OVERRUN; break; }
+              if (level - 1u >= p.s) { err = QSGD_DEV_LEVEL; break; }
+              code = level | (neg << 4);
+            }
+            src.drop(l1 + l2);
+            used += l1 + l2;
+            at += gap;
+            if (at >= lim) { pend = at | ((code & 0x1Fu) << 16); break; }     // a later range's, or past the bucket
+            row[at - rbeg] = (uint8_t)code;
+          }
+          if (err) readable = false;
+        }
+      }
+      __syncwarp();
+      // ---- phase 2: ascending-k sum; a lane takes 8 coordinates per pass --------------------------
+      const uint32_t slots_per_bucket = (rend - rbeg) >> 3;
+      const uint32_t total_slots = p.G * slots_per_bucket;
+      for (uint32_t s0 = 0; s0 < total_slots; s0 += 32) {
+        const uint32_t slot = s0 + lane;
+        const uint32_t g = slot / slots_per_bucket, cl = (slot - g * slots_per_bucket) << 3, c = rbeg + cl;
+        const uint64_t b = b0 + g;
+        const uint64_t i0 = b * p.d + c;
+        const bool in_tile = slot < total_slots;               // rows and scales of bucket g exist in the tile
+        const bool live = in_tile && b < p.B && i0 < p.n;
+        // a lane past the end of its bucket still holds its share of the bucket's shuffle table
+        const uint32_t gg = in_tile ? g : 0u;
+        const uint8_t* rows = mine + gg * p.K * row_bytes + cl;
+        const float* sc = scales + gg * p.Kpad;
+        float acc[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+#pragma unroll 4
+        for (uint32_t k = 0; k < p.K; ++k) {
+          const uint2 cw = in_tile ? *reinterpret_cast<const uint2*>(rows + k * row_bytes) : make_uint2(0u, 0u);
+          const float Ak = sc[k];
+          const uint32_t w[2] = {cw.x, cw.y};
+          if (SINGLE) {
+            const float lutk = __fmul_rn(Ak, lut0);            // every lane of this pass is in bucket g
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                acc[4 * h + j] = __fadd_rn(acc[4 * h + j], shfl_f(lutk, w[h] >> (8 * j)));
+          } else {
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+                acc[4 * h + j] = __fadd_rn(acc[4 * h + j], __fmul_rn(Ak, shfl_f(lut0, w[h] >> (8 * j))));
+          }
+        }
+        if (live) {
+          float* o;
+          uint32_t valid;
+          if (p.map.src) {
+            const OutSpan sp = out_span(p.out, p.map, b, c, p.d, p.n, 8u);
+            o = sp.ptr; valid = sp.valid;
+          } else {
+            o = p.out + i0;
+            valid = (uint32_t)min((uint64_t)8u, p.n - i0);
+          }
+          if (valid == 8u && (reinterpret_cast<uintptr_t>(o) & 15u) == 0) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+              float4 r = make_float4(acc[4 * j], acc[4 * j + 1], acc[4 * j + 2], acc[4 * j + 3]);
+              if (FUSED) {
+                const float4 x = *reinterpret_cast<const float4*>(o + 4 * j);
+                r.x = __fsub_rn(x.x, __fmul_rn(p.c, r.x)); r.y = __fsub_rn(x.y, __fmul_rn(p.c, r.y));
+                r.z = __fsub_rn(x.z, __fmul_rn(p.c, r.z)); r.w = __fsub_rn(x.w, __fmul_rn(p.c, r.w));
+              }
+              *reinterpret_cast<float4*>(o + 4 * j) = r;
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              if ((uint32_t)e < valid) o[e] = FUSED ? __fsub_rn(o[e], __fmul_rn(p.c, acc[e])) : acc[e];
+          }
+        }
+      }
+      __syncwarp();
+    }
+    // a string must end exactly where the table says
+    // a string must end exactly where the table says, with no entry left over (one that no range took
+    // lies past the bucket)
+    if (parsing && err == 0u && pend != kNone) err = QSGD_DEV_POSITION;
+    if (parsing && err == 0u && used != total) err = QSGD_DEV_OVERRUN;
+    if (err) atomicOr(p.status, err);
+    __syncwarp();
+  }
+}
+
+int launch_bytes(FieldParams& p, bool fused, cudaStream_t stream, bool* handled) {
+  *handled = false;
+  if (p.K > 32u) return 0;
+  int dev = 0, max_smem = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  uint32_t kpad = 1;
+  while (kpad < p.K) kpad <<= 1;
+  p.Kpad = kpad;
+  p.G = 32u / kpad;
+  const uint32_t R = p.d <= kByteRange ? p.d : kByteRange;
+  p.range = R;
+  const size_t per_warp = (size_t)p.G * p.K * (R + kRowPad) + 128u;
+  const size_t per_cta = 8192 + 512 + 1024;                     // the two code tables + slack
+  const size_t budget = (size_t)max_smem - per_cta;
+  const size_t per_sm = 227u << 10;
+  int warps = 0, best = 0;
+  for (int w = 1; w <= 16; ++w) {
+    if ((size_t)w * per_warp > budget) break;
+    const int resident = (int)(per_sm / ((size_t)w * per_warp + per_cta)) * w;
+    if (resident > best) { best = resident; warps = w; }
+  }
+  if (warps == 0) return 0;
+  const bool single = (R & 255u) == 0;                          // a pass of 32 lanes x 8 stays inside one bucket
+  void (*kern)(FieldParams);
+  if (fused) kern = single ? decode_elias_bytes_kernel<true, true> : decode_elias_bytes_kernel<true, false>;
+  else kern = single ? decode_elias_bytes_kernel<false, true> : decode_elias_bytes_kernel<false, false>;
+  const size_t smem = (size_t)warps * per_warp;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return (int)e;
+  int occ = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, warps * 32, smem);
+  if (e != cudaSuccess) return (int)e;
+  if (occ < 1) occ = 1;
+  const uint64_t groups = (p.B + p.G - 1) / p.G;
+  const uint64_t want = (groups + warps - 1) / warps;
+  const uint64_t cap = (uint64_t)sms * occ;
+  const uint32_t grid = (uint32_t)(want < cap ? want : cap);
+  {
+    ScopedKernel sk(kKernDecodeElias, stream);
+    kern<<<grid, warps * 32, smem, stream>>>(p);
+  }
+  *handled = true;
+  return (int)cudaGetLastError();
+}
+
+
 template <int LB>
 int launch_fields_lb(FieldParams& p, bool dense, bool fused, cudaStream_t stream, bool* handled) {
+  if (!dense && LB != 8 && p.d < 1024u && p.K <= 32u) return launch_bytes(p, fused, stream, handled);
   if (p.d >= 1024u && p.K <= 32u)       // long buckets: fields of one range at a time
     return dense ? launch_ranged<LB, true>(p, fused, stream, handled) : launch_ranged<LB, false>(p, fused, stream, handled);
   return dense ? launch_fields<LB, true>(p, fused, stream, handled) : launch_fields<LB, false>(p, fused, stream, handled);

@@ -126,6 +126,22 @@ def test_elias_peer_counts(K, code_kind):
     decode_parity(msgs, infos, n, d, s, code_kind, eta=0.05, x0=I.gaussian(n, 1.0, seed=9), tables_first=True)
 
 
+@pytest.mark.parametrize("K", [1, 2, 3, 5, 8])
+@pytest.mark.parametrize("d,tail", [(512, 188), (512, 300), (256, 100), (96, 40), (992, 500)])
+def test_elias_few_peers_high_levels_ragged_tail(K, d, tail):
+    """Few peers (a warp then owns many buckets), max-norm scaling at s = 15 (negative levels of 8 and
+    more occur, the codes whose value sits in the upper lanes of the decoder's shuffle table) and a
+    last bucket that is shorter than a decoding range."""
+    n, s = 9 * d + tail, 15
+    msgs, infos = [], []
+    for w in range(K):
+        g = make(n, "mix", seed=500 + w)
+        m, info = encode_parity(g, d, s, O.NORM_MAX, O.CODE_ELIAS, seed=9, step=2, worker=w)
+        msgs.append(m)
+        infos.append(info)
+    decode_parity(msgs, infos, n, d, s, O.CODE_ELIAS, eta=0.3, x0=I.gaussian(n, 1.0, seed=2))
+
+
 @pytest.mark.parametrize("d,s", [(4096, 255), (4096, 1), (2048, 15), (1024, 3), (64, 15), (32, 1)])
 def test_elias_bucket_shapes(d, s):
     n, K = 5 * d + 123, 4
