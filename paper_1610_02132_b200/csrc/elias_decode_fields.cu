@@ -645,7 +645,7 @@ int launch_bytes(FieldParams& p, bool fused, cudaStream_t stream, bool* handled)
     if (resident > best) { best = resident; warps = w; }
   }
   if (warps == 0) return 0;
-  const bool single = (R & 255u) == 0;                          // a pass of 32 lanes x 8 stays inside one bucket
+  const bool single = (p.d & 255u) == 0;                        // every range is 256 long: a pass of 32 lanes x 8 stays inside one bucket
   void (*kern)(FieldParams);
   if (fused) kern = single ? decode_elias_bytes_kernel<true, true> : decode_elias_bytes_kernel<true, false>;
   else kern = single ? decode_elias_bytes_kernel<false, true> : decode_elias_bytes_kernel<false, false>;
