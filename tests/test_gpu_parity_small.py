@@ -142,6 +142,22 @@ def test_elias_few_peers_high_levels_ragged_tail(K, d, tail):
     decode_parity(msgs, infos, n, d, s, O.CODE_ELIAS, eta=0.3, x0=I.gaussian(n, 1.0, seed=2))
 
 
+@pytest.mark.parametrize("d", [32, 64, 160, 256, 288, 480, 512, 736, 1000 // 32 * 32])
+@pytest.mark.parametrize("K,s,norm_kind", [(1, 15, O.NORM_MAX), (2, 3, O.NORM_L2), (4, 7, O.NORM_MAX), (7, 1, O.NORM_L2),
+                                           (16, 15, O.NORM_L2), (17, 2, O.NORM_MAX), (32, 15, O.NORM_MAX)])
+def test_elias_decoder_shapes_below_1024(d, K, s, norm_kind):
+    """Bucket sizes around the decoder's range length (256), peer counts around the powers of two that
+    set how many buckets a warp owns, every field width up to 4 bits, a ragged tail."""
+    n = 11 * d + d // 2 + 3
+    msgs, infos = [], []
+    for w in range(K):
+        g = make(n, ["gauss", "sparse", "mix"][w % 3], seed=700 + w)
+        m, info = encode_parity(g, d, s, norm_kind, O.CODE_ELIAS, seed=3, step=5, worker=w)
+        msgs.append(m)
+        infos.append(info)
+    decode_parity(msgs, infos, n, d, s, O.CODE_ELIAS, eta=0.2, x0=I.gaussian(n, 1.0, seed=4))
+
+
 @pytest.mark.parametrize("d,s", [(4096, 255), (4096, 1), (2048, 15), (1024, 3), (64, 15), (32, 1)])
 def test_elias_bucket_shapes(d, s):
     n, K = 5 * d + 123, 4
