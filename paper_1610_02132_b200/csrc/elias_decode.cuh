@@ -104,23 +104,22 @@ __device__ __forceinline__ StringRef string_ref(const PeerSet& ps, uint32_t k, u
 // Strings short enough for the entry-list decoder? True when the K payloads average less than a
 // quarter of a bit per coordinate beyond the scales: an entry of a sparse bucket costs 11 to 14
 // bits, so a list with room for one entry per 32 positions then fills to about 60 % on average and
-// rarely overflows. Called by every thread of a CTA (it holds a CTA barrier): thread 0 reads the K
-// payload lengths and the answer goes round through shared memory, so a kernel that only has to
-// stand down costs K loads per CTA. Same answer in every kernel that asks.
+// rarely overflows. Called by every thread of a CTA (it holds CTA barriers): K threads read the K
+// payload lengths side by side and add them up in shared memory, so a kernel that only has to stand
+// down costs one round of loads per CTA. Same answer in every kernel that asks.
 __device__ __forceinline__ bool sparse_regime(const PeerSet& peers, uint32_t K, uint64_t B, uint32_t d) {
-  __shared__ uint32_t verdict;
-  if (threadIdx.x == 0) {
-    bool sparse = K <= 32u;
-    uint64_t bits = 0;
-    for (uint32_t k = 0; k < K && sparse; ++k) {
-      PeerTable pt;
-      if (!peer_table(peers, k, B, &pt)) sparse = false;     // the field decoders report the bad place
-      else bits += __ldg(pt.table + B);
-    }
-    verdict = (sparse && bits < (uint64_t)K * B * (32ull + d / 4u)) ? 1u : 0u;
+  __shared__ unsigned long long total_bits;
+  __shared__ uint32_t bad_place;
+  if (threadIdx.x == 0) { total_bits = 0ull; bad_place = 0u; }
+  __syncthreads();
+  // thread k reads peer k's payload length: the K pairs of dependent loads run side by side
+  for (uint32_t k = threadIdx.x; k < K; k += blockDim.x) {
+    PeerTable pt;
+    if (!peer_table(peers, k, B, &pt)) atomicOr(&bad_place, 1u);     // the field decoders report the bad place
+    else atomicAdd(&total_bits, (unsigned long long)__ldg(pt.table + B));
   }
   __syncthreads();
-  return verdict != 0u;
+  return K <= 32u && bad_place == 0u && total_bits < (uint64_t)K * B * (32ull + d / 4u);
 }
 
 struct FieldParams {
