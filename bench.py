@@ -872,6 +872,9 @@ def main():
     ap.add_argument("--replicas", action="store_true",
                     help="with more than one GPU: independent replicas of the one-GPU workload (no collective) "
                          "instead of Algorithm 1 across the GPUs")
+    ap.add_argument("--exchange", action="store_true",
+                    help="run the multi-GPU path (encode into slots, NCCL all-gather, packed decode, all-reduce arm) "
+                         "even with a single rank: exercises that path on one GPU")
     ap.add_argument("--capacity-slots", action="store_true",
                     help="multi-GPU: all-gather whole capacity slots (no host synchronisation) instead of slots "
                          "cut to the longest message of the step")
@@ -895,7 +898,7 @@ def main():
         run_sweep(args)
     elif args.workload == "qsvrg":
         run_qsvrg(args)
-    elif max(world, 1) > 1 and not args.replicas:
+    elif (max(world, 1) > 1 and not args.replicas) or args.exchange:
         run_multi(args)
     else:
         run_cuda(args)

@@ -763,7 +763,7 @@ int qsgd_encode_elias_static(const float* g, uint64_t n, uint32_t bucket, uint32
                              qsgd_stream_t stream) {
   using namespace qsgd;
   if (!g || !out || !out_bits || !status_dev) return QSGD_ERR_NULL;
-  if (n == 0) return QSGD_ERR_SIZE;
+  if (n == 0 || n > QSGD_MAX_COORDS) return QSGD_ERR_SIZE;
   if (bucket < 32 || bucket > QSGD_MAX_BUCKET || (bucket & 31u)) return QSGD_ERR_BUCKET;
   if (s < 1 || s > QSGD_MAX_LEVELS) return QSGD_ERR_LEVELS;
   if (code_kind != QSGD_CODE_ELIAS && code_kind != QSGD_CODE_ELIAS_DENSE) return QSGD_ERR_KIND;
