@@ -44,6 +44,9 @@ WORKLOADS = {
     "resnet152_policy": dict(n=60192808, d=512, s=15, norm="l2", codes=["fixed", "elias"], K=16, gen="mixture",
                              policy="resnet152",
                              desc="ResNet-152-shaped gradient under the per-tensor policy (313 small tensors raw)"),
+    # Corollary 3.3's regime: the dense code Code'_s at s = sqrt(d)
+    "dense_elias": dict(n=2 ** 24, d=4096, s=64, norm="l2", codes=["elias_dense"], K=8, gen="gauss1",
+                        desc="dense Elias regime: N(0,1), n=2^24, s = sqrt(d), every coordinate coded"),
     "sweep_point": dict(n=2 ** 28, d=512, s=15, norm="l2", codes=["fixed"], K=16, gen="gauss1",
                         desc="bandwidth sweep point: N(0,1), n=2^28"),
 }
@@ -459,6 +462,11 @@ def run_cuda(args):
         cpu = run_oracle_sample(wl, steps=1)
         cpu["host_cores"] = os.cpu_count()
         cpu["all_cores"] = run_oracle_parallel(wl)
+
+    if clocks and clocks.get("sm_mhz"):
+        # time x median SM clock: how a kernel's duration would move with the clock, were it core-bound
+        for k in kern_tab:
+            kern_tab[k]["kcycles_at_median_sm_clock"] = kern_tab[k]["avg_us"] * clocks["sm_mhz"] / 1e3
 
     if rank == 0:
         line = {

@@ -3,11 +3,11 @@
 //
 // Two streaming kernels for power-of-two bucket sizes, both persistent and fed by 1-D TMA bulk
 // copies (cp.async.bulk + mbarrier), so no thread spends instructions on global loads:
-//   * quantize_warp_kernel (d <= 512, no bucket map): every warp runs its own pipeline over
+//   * quantize_warp_kernel (d <= 512, with or without a bucket map): every warp runs its own pipeline over
 //     chunks of 512 coordinates (whole buckets) with a private ring of shared-memory stages that
 //     its lane 0 refills as soon as the warp has taken a stage into registers. No CTA-wide
 //     barrier and no separate "empty" barrier exist, and every decision is warp-uniform.
-//   * quantize_pow2_kernel (d >= 1024, or buckets fetched through a bucket map): the CTA walks
+//   * quantize_pow2_kernel (d >= 1024): the CTA walks
 //     tiles of 4096 coordinates through a shared ring; scales of buckets that span several
 //     warps meet in shared memory.
 // A thread owns 16 consecutive coordinates: it pulls them into registers once, the bucket scale
@@ -351,12 +351,12 @@ __device__ __forceinline__ void issue_tile(const FastParams& p, float* tile, uin
   if (lane < nb && L) bulk_load(tile + lane * d, p.g + src, 4u * L, full_bar);
 }
 
-// CROSS: a bucket spans several warps (d >= 1024); otherwise a bucket is d / 16 <= 32 lanes.
-// CTAs 0 .. main_ctas - 1 stream the complete tiles; one optional extra CTA runs the ragged last
-// tile and the region padding through the generic tile code (its operands alias the tile ring).
-// MAPPED: buckets are fetched through a bucket map (per-tensor policy); a separate instantiation, so
-// that the ordinary kernel carries none of that code.
-template <int LB, int NORM, bool CROSS, bool MAPPED>
+// CTA-wide streaming kernel for d >= 1024, where a bucket spans 2^(log2d - 9) warps and the scales
+// meet in shared memory. CTAs 0 .. main_ctas - 1 stream the complete tiles; one optional extra CTA
+// runs the ragged last tile and the region padding through the generic tile code (its operands alias
+// the tile ring). MAPPED: buckets are fetched through a bucket map (per-tensor policy); a separate
+// instantiation, so that the ordinary kernel carries none of that code.
+template <int LB, int NORM, bool MAPPED>
 __global__ void __launch_bounds__(kThreads, 4)
 quantize_pow2_kernel(const __grid_constant__ FastParams p) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -389,9 +389,8 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
 
   const float sf = (float)p.s;
   const float cap = kTwo23 + sf;
-  const uint32_t team_w = CROSS ? 32u : (1u << (p.log2d - 4));   // lanes per bucket (<= 32)
-  const uint32_t wpb = CROSS ? (1u << (p.log2d - 9)) : 1u;       // warps per bucket
-  const bool leader = CROSS ? ((tid & (32u * wpb - 1u)) == 0) : ((lane & (team_w - 1u)) == 0);
+  const uint32_t wpb = 1u << (p.log2d - 9);                      // warps per bucket
+  const bool leader = (tid & (32u * wpb - 1u)) == 0;
   const uint32_t my_bucket = (tid * 16u) >> p.log2d;             // bucket of this thread in a tile
   const uint32_t buckets_per_tile_log2 = 12u - p.log2d;
 
@@ -416,24 +415,21 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
 #pragma unroll
     for (uint32_t o = 16; o > 0; o >>= 1) {
       const float q = __shfl_xor_sync(0xffffffffu, part, o);
-      const float merged = (NORM == QSGD_NORM_L2) ? part + q : fmaxf(part, q);
-      part = (o < team_w) ? merged : part;
+      part = (NORM == QSGD_NORM_L2) ? part + q : fmaxf(part, q);
     }
     // 2-norm: an fp32 sum of squares outside [8e-28, 1e30] may have lost bits to underflow or
-    // overflowed; such buckets are redone in fp64 (rare, the warp / CTA branches together)
+    // overflowed; such buckets are redone in fp64 (rare, the CTA branches together)
     bool shaky = false;
     if (NORM == QSGD_NORM_L2) shaky = !(part >= 8.0e-28f && part <= 1.0e30f) && part != 0.f;
-    if (CROSS && lane == 0) sm.wsum[it & 1][warp] = part;
+    if (lane == 0) sm.wsum[it & 1][warp] = part;
 
     // ---- release the stage: every warp signals that its values are in registers; the producer
     // thread refills the stage that was released one iteration ago (its arrivals are long in) ----
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.empty[stage]);
-    // a wait that ran out ends the loop; the decision is taken per CTA (CROSS: the scales meet
-    // in shared memory) or per warp (its lanes meet in shuffles), never per lane
-    int flags = arrived ? 0 : 1;
-    if (CROSS) flags = __syncthreads_or(flags | (shaky ? 2 : 0));
-    else flags = __any_sync(0xffffffffu, flags != 0) ? 1 : 0;
+    // a wait that ran out ends the loop; the decision is taken per CTA (the scales meet in
+    // shared memory), never per lane
+    const int flags = __syncthreads_or((arrived ? 0 : 1) | (shaky ? 2 : 0));
     if (flags & 1) {
       if (lane == 0) atomicOr(p.status, QSGD_DEV_TIMEOUT);
       break;
@@ -460,7 +456,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
       }
     }
     float A;
-    if (CROSS) {
+    {
       const uint32_t w0 = warp & ~(wpb - 1u);
       float acc = 0.f;
       for (uint32_t w = 0; w < wpb; ++w) {
@@ -485,21 +481,6 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
       } else {
         A = acc;
       }
-    } else if (NORM == QSGD_NORM_L2) {
-      A = __fsqrt_rn(part);
-      if (__any_sync(0xffffffffu, shaky)) {
-        double wide = 0.0;
-#pragma unroll
-        for (int e = 0; e < 16; ++e) wide = fma((double)v[e], (double)v[e], wide);
-#pragma unroll
-        for (uint32_t o = 16; o > 0; o >>= 1) {
-          const double q = __shfl_xor_sync(0xffffffffu, wide, o);
-          wide = (o < team_w) ? wide + q : wide;
-        }
-        if (shaky) A = __double2float_rn(sqrt(wide));
-      }
-    } else {
-      A = part;
     }
     if (!(A >= FLT_MIN)) A = 0.f;                      // zero bucket: Q(0) = 0
     const float r = A > 0.f ? __frcp_rn(A) : 0.f;
@@ -712,7 +693,7 @@ __device__ __forceinline__ void quantize_generic_tile(const QuantizeParams& p, u
 }
 
 // ---------------------------------------------------------------------------------------------
-// Per-warp streaming kernel: d <= 512 (a bucket never leaves a warp), no bucket map.
+// Per-warp streaming kernel: d <= 512 (a bucket never leaves a warp).
 // Warp w of CTA b takes chunks b * 8 + w, + 8 * main_ctas, ... of 512 coordinates. Its ring of
 // kWarpStages stages is private: lane 0 arms a stage (expect-tx + bulk copy), all lanes wait on
 // the stage's barrier, pull their 16 values into registers, and after the shuffle reduction of
@@ -728,7 +709,66 @@ struct __align__(16) WarpRings {
   uint64_t full[kThreads / 32][kWarpStages];
 };
 
-template <int LB, int NORM>
+// How the per-warp kernel finds its chunks. The streaming loop is sensitive to every warp-wide step
+// added to it (a shuffle and a vote on the map entries cost 8 % of the kernel's time with nothing
+// else changed), so with a map every lane that owns a bucket of the chunk starts that bucket's copy
+// by itself, and the zeros behind a short bucket are one more copy, from a block of zeros in global
+// memory: no loop, no call, no common step. Buckets of 512 -- one per chunk, lane 0 alone at work --
+// are an instantiation of their own. What is left of the map's cost (about 8 % against the same
+// buckets without a map) is not the two loads, which cost nothing when their results go unused, but
+// handing a loaded address and length to the bulk copy, whose operands sit in uniform registers.
+enum MapMode { kNoMap = 0, kMapOnePerChunk = 1, kMapSeveralPerChunk = 2 };
+
+__device__ __align__(128) float g_zero_chunk[kChunk];      // never written
+
+// What lane j < 512 / d knows of bucket j of a chunk when buckets come through a bucket map.
+struct MappedBucket {
+  uint64_t src;   // first coordinate of the bucket in g
+  uint32_t len;   // coordinates it holds (<= d; zeros stand behind a short one)
+};
+
+template <int MAP>
+__device__ __forceinline__ MappedBucket fetch_bucket(const FastParams& p, uint32_t chunk, uint32_t chunks,
+                                                     uint32_t lane) {
+  MappedBucket mb{0ull, 0u};
+  if (MAP != kNoMap) {
+    const uint32_t nb = (uint32_t)kChunk >> p.log2d;
+    if (chunk < chunks && lane < nb) {
+      const uint64_t b = ((uint64_t)chunk << (9u - p.log2d)) + lane;
+      mb.src = __ldg(p.map.src + b);
+      mb.len = min(__ldg(p.map.len + b), 1u << p.log2d);
+    }
+  }
+  return mb;
+}
+
+// Arm one stage for `chunk` (called by the whole warp; its reads of the stage are already done).
+// The stage always receives kChunk * 4 bytes: lane 0 announces them, and the copies may complete
+// before or after that (the barrier's transaction count is signed). The map guarantees 16-byte
+// aligned places and lengths.
+template <int MAP>
+__device__ __forceinline__ void arm_chunk(const FastParams& p, float* dst, uint64_t* bar, uint32_t chunk,
+                                          uint32_t lane, const MappedBucket mb) {
+  if (MAP == kNoMap) {
+    if (lane == 0) {
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");     // our reads before the copy's writes
+      mbar_expect_tx(bar, kChunk * 4);
+      bulk_load(dst, p.g + (size_t)chunk * kChunk, kChunk * 4, bar);
+    }
+    return;
+  }
+  const uint32_t d = MAP == kMapOnePerChunk ? (uint32_t)kChunk : 1u << p.log2d;
+  const uint32_t nb = MAP == kMapOnePerChunk ? 1u : (uint32_t)kChunk >> p.log2d;
+  if (lane < nb) {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (lane == 0) mbar_expect_tx(bar, kChunk * 4);
+    float* mine = dst + lane * d;
+    if (mb.len) bulk_load(mine, p.g + mb.src, 4u * mb.len, bar);
+    if (mb.len != d) bulk_load(mine + mb.len, g_zero_chunk, 4u * (d - mb.len), bar);
+  }
+}
+
+template <int LB, int NORM, int MAP>
 __global__ void __launch_bounds__(kThreads, 4)
 quantize_warp_kernel(const __grid_constant__ FastParams p) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
@@ -737,7 +777,7 @@ quantize_warp_kernel(const __grid_constant__ FastParams p) {
   const uint32_t grid = p.main_ctas;
   if (blockIdx.x >= grid) {                     // the extra CTA: ragged tail + padding
     float* scratch = &sm.chunk[0][0][0];
-    quantize_generic_tile<LB, NORM, false>(p.tail, 0u, 1u, scratch, scratch + kTile, scratch + kTile + 1024);
+    quantize_generic_tile<LB, NORM, MAP != kNoMap>(p.tail, 0u, 1u, scratch, scratch + kTile, scratch + kTile + 1024);
     return;
   }
   const uint32_t chunks = p.full_tiles * (kTile / kChunk), stride = grid * (kThreads / 32);
@@ -749,15 +789,17 @@ quantize_warp_kernel(const __grid_constant__ FastParams p) {
       p.info[0] = 8 * p.total_bytes; p.info[1] = 0; p.info[2] = p.total_bytes; p.info[3] = 0;
     }
     if (tid == 0 && blockIdx.x == 0 && p.clear_word) *p.clear_word = 0u;
-    for (int s = 0; s < kWarpStages; ++s) {
-      const uint32_t cs = c + (uint32_t)s * stride;
-      if (cs < chunks) {
-        mbar_expect_tx(&sm.full[warp][s], kChunk * 4);
-        bulk_load(sm.chunk[warp][s], p.g + (size_t)cs * kChunk, kChunk * 4, &sm.full[warp][s]);
-      }
-    }
   }
   __syncwarp();
+  for (int s = 0; s < kWarpStages; ++s) {
+    const uint32_t cs = c + (uint32_t)s * stride;
+    if (cs < chunks) {
+      const MappedBucket mb = fetch_bucket<MAP>(p, cs, chunks, lane);
+      arm_chunk<MAP>(p, sm.chunk[warp][s], &sm.full[warp][s], cs, lane, mb);
+    }
+  }
+  // the map entries of the next chunk to arm are fetched one round ahead of their use
+  MappedBucket ahead = fetch_bucket<MAP>(p, c + (uint32_t)kWarpStages * stride, chunks, lane);
 
   const float sf = (float)p.s;
   const float cap = kTwo23 + sf;
@@ -808,13 +850,10 @@ quantize_warp_kernel(const __grid_constant__ FastParams p) {
 
     // ---- the stage is in registers: refill it with the chunk kWarpStages rounds ahead --------
     __syncwarp();
-    if (lane == 0) {
+    {
       const uint32_t cn = c + (uint32_t)kWarpStages * stride;
-      if (cn < chunks) {
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // our reads before the copy's writes
-        mbar_expect_tx(&sm.full[warp][stage], kChunk * 4);
-        bulk_load(sm.chunk[warp][stage], p.g + (size_t)cn * kChunk, kChunk * 4, &sm.full[warp][stage]);
-      }
+      if (cn < chunks) arm_chunk<MAP>(p, sm.chunk[warp][stage], &sm.full[warp][stage], cn, lane, ahead);
+      ahead = fetch_bucket<MAP>(p, cn + stride, chunks, lane);
     }
 
     // ---- scale ---------------------------------------------------------------------------------
@@ -895,23 +934,34 @@ PhiloxConsts make_philox_consts(uint64_t seed, uint32_t step, uint32_t worker) {
 
 std::atomic<uint32_t> g_poll_limit{kDrainPolls};
 
-template <int LB, int NORM, bool CROSS, bool MAPPED>
-int launch_fast(FastParams& fp, bool with_tail, cudaStream_t stream) {
-  constexpr bool kPerWarp = !CROSS && !MAPPED;
+template <int LB, int NORM, int MAP>
+int launch_warp(FastParams& fp, bool with_tail, cudaStream_t stream) {
   static KernelSite site;
-  const size_t smem = (kPerWarp ? sizeof(WarpRings) : sizeof(TileSmem)) + 128;
+  const size_t smem = sizeof(WarpRings) + 128;
   int sms = 0, ctas_per_sm = 0;
-  int st;
-  if (kPerWarp) st = site.lookup(quantize_warp_kernel<LB, NORM>, kThreads, smem, &sms, &ctas_per_sm);
-  else st = site.lookup(quantize_pow2_kernel<LB, NORM, CROSS, MAPPED>, kThreads, smem, &sms, &ctas_per_sm);
+  const int st = site.lookup(quantize_warp_kernel<LB, NORM, MAP>, kThreads, smem, &sms, &ctas_per_sm);
   if (st) return st;
   const uint32_t cap = (uint32_t)(sms * ctas_per_sm);
   fp.main_ctas = fp.full_tiles < cap ? fp.full_tiles : cap;
   fp.poll_limit = g_poll_limit.load(std::memory_order_relaxed);
   ScopedKernel sk(kKernQuantize, stream);
-  const uint32_t grid = fp.main_ctas + (with_tail ? 1u : 0u);
-  if (kPerWarp) quantize_warp_kernel<LB, NORM><<<grid, kThreads, smem, stream>>>(fp);
-  else quantize_pow2_kernel<LB, NORM, CROSS, MAPPED><<<grid, kThreads, smem, stream>>>(fp);
+  quantize_warp_kernel<LB, NORM, MAP><<<fp.main_ctas + (with_tail ? 1u : 0u), kThreads, smem, stream>>>(fp);
+  return (int)cudaGetLastError();
+}
+
+// d >= 1024: the CTA-wide ring.
+template <int LB, int NORM, bool MAPPED>
+int launch_cross(FastParams& fp, bool with_tail, cudaStream_t stream) {
+  static KernelSite site;
+  const size_t smem = sizeof(TileSmem) + 128;
+  int sms = 0, ctas_per_sm = 0;
+  const int st = site.lookup(quantize_pow2_kernel<LB, NORM, MAPPED>, kThreads, smem, &sms, &ctas_per_sm);
+  if (st) return st;
+  const uint32_t cap = (uint32_t)(sms * ctas_per_sm);
+  fp.main_ctas = fp.full_tiles < cap ? fp.full_tiles : cap;
+  fp.poll_limit = g_poll_limit.load(std::memory_order_relaxed);
+  ScopedKernel sk(kKernQuantize, stream);
+  quantize_pow2_kernel<LB, NORM, MAPPED><<<fp.main_ctas + (with_tail ? 1u : 0u), kThreads, smem, stream>>>(fp);
   return (int)cudaGetLastError();
 }
 
@@ -920,9 +970,8 @@ int launch_one(QuantizeParams& p, uint64_t seed, cudaStream_t stream) {
   const uint32_t d = p.d;
   const bool pow2 = (d & (d - 1)) == 0;
   uint32_t full_tiles = 0;
-  // with a bucket map the bulk copies need 16-byte aligned places and lengths, and one copy per
-  // bucket is only worth issuing from a single thread when buckets are not tiny
-  const bool map_ok = !p.map.src || (p.map.quads != 0u && d >= 256);
+  // with a bucket map the bulk copies need 16-byte aligned places and lengths
+  const bool map_ok = !p.map.src || p.map.quads != 0u;
   if (pow2 && p.n <= (1ull << 32) && map_ok) full_tiles = (uint32_t)(p.n / kTile);
   if (full_tiles > 0) {
     FastParams fp;
@@ -941,10 +990,11 @@ int launch_one(QuantizeParams& p, uint64_t seed, cudaStream_t stream) {
     fp.tail = p;
     fp.tail.info = nullptr;
     fp.tail.clear_word = nullptr;
-    if (fp.map.src) return d >= 1024 ? launch_fast<LB, NORM, true, true>(fp, with_tail, stream)
-                                     : launch_fast<LB, NORM, false, true>(fp, with_tail, stream);
-    return d >= 1024 ? launch_fast<LB, NORM, true, false>(fp, with_tail, stream)
-                     : launch_fast<LB, NORM, false, false>(fp, with_tail, stream);
+    if (d >= 1024) return fp.map.src ? launch_cross<LB, NORM, true>(fp, with_tail, stream)
+                                     : launch_cross<LB, NORM, false>(fp, with_tail, stream);
+    if (!fp.map.src) return launch_warp<LB, NORM, kNoMap>(fp, with_tail, stream);
+    return d == (uint32_t)kChunk ? launch_warp<LB, NORM, kMapOnePerChunk>(fp, with_tail, stream)
+                                 : launch_warp<LB, NORM, kMapSeveralPerChunk>(fp, with_tail, stream);
   }
   // the fast path does not apply: everything through the generic kernel
   p.coord_base = 0;

@@ -116,6 +116,16 @@ def test_policy_many_tiles_and_sparse_regime(code_kind):
     run_case(sizes, 4096, 1, O.NORM_L2, code_kind, K=8, kind="sparse")
 
 
+@pytest.mark.parametrize("d", [32, 128, 256, 512])
+@pytest.mark.parametrize("norm_kind", [O.NORM_L2, O.NORM_MAX])
+def test_policy_short_buckets_inside_the_stream(d, norm_kind):
+    # every place and length a multiple of 4 (bulk copies), most tensors ending in a short bucket that
+    # lies among the complete tiles of the streaming encoder: of 4, of d - 4 and of d / 2 coordinates
+    sizes = [4096 * 5 + 4, 8192 + d - 4, 20, 20480 + d // 2, 4096 * 9, 12288 + 36, 65536 + 8]
+    run_case(sizes, d, 15, norm_kind, O.CODE_FIXED, K=2, tau=4096)
+    run_case(sizes, d, 3, norm_kind, O.CODE_ELIAS, K=2, tau=4096)
+
+
 def test_policy_many_peers():
     run_case(RAGGED, 256, 7, O.NORM_L2, O.CODE_ELIAS, K=33, tau=4096)
 
