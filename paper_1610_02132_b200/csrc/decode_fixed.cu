@@ -44,6 +44,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_fixed_kernel(const __grid_
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float sf = (float)p.s;
   float lut0 = 0.f;                                  // this lane's +-(level / s)
+  chain_release();
   if (LB == 8) {
     for (uint32_t i = tid; i < 256 * 32; i += kThreads) xi_tab[i] = __fdiv_rn((float)(i >> 5), sf);
     __syncthreads();
@@ -53,6 +54,7 @@ __global__ void __launch_bounds__(kThreads, 4) decode_fixed_kernel(const __grid_
     lut0 = neg ? -q : q;
   }
   const uint8_t* tab_lane = reinterpret_cast<const uint8_t*>(xi_tab) + 4 * lane;
+  chain_wait();                                      // the messages come from the kernels ahead
 
   for (uint64_t ch = (uint64_t)blockIdx.x * kWarps + warp; ch < p.chunks; ch += (uint64_t)gridDim.x * kWarps) {
     const uint64_t i0 = ch * kChunk + (uint64_t)lane * 16;       // first coordinate of this lane
@@ -104,6 +106,8 @@ __global__ void __launch_bounds__(kThreads) sgd_step_kernel(float* __restrict__ 
                                                            const float* __restrict__ acc, float c,
                                                            uint64_t n) {
   const uint64_t i0 = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) * 4;
+  chain_release();
+  chain_wait();
   if (i0 + 4 <= n) {
     const float4 a = __ldcs(reinterpret_cast<const float4*>(acc + i0));
     float4 v = *reinterpret_cast<const float4*>(x + i0);
@@ -129,7 +133,8 @@ int launch_one(const DecodeParams& p, cudaStream_t stream) {
   const uint32_t grid = (uint32_t)(want < cap ? want : cap);
   {
     ScopedKernel sk(kKernDecodeFixed, stream);
-    kern<<<grid, kThreads, 0, stream>>>(p);
+    const cudaError_t e = launch_chained(kern, grid, kThreads, 0, stream, p);
+    if (e != cudaSuccess) return (int)e;
   }
   return (int)cudaGetLastError();
 }
@@ -170,7 +175,8 @@ int launch_sgd_step(float* x, const float* acc, float eta, uint32_t K, uint64_t 
   const uint32_t grid = (uint32_t)((quads + kThreads - 1) / kThreads);
   {
     ScopedKernel sk(kKernSgdStep, stream);
-    sgd_step_kernel<<<grid, kThreads, 0, stream>>>(x, acc, c, n);
+    const cudaError_t e = launch_chained(sgd_step_kernel, grid, kThreads, 0, stream, x, acc, c, n);
+    if (e != cudaSuccess) return (int)e;
   }
   return (int)cudaGetLastError();
 }

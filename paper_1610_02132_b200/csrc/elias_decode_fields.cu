@@ -92,6 +92,8 @@ __global__ void __launch_bounds__(320) decode_elias_fields_kernel(const __grid_c
   extern __shared__ __align__(16) uint32_t fsm[];
   __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
   __shared__ uint16_t elias_lut[1u << kLutBits];
+  chain_release();
+  chain_wait();                                   // the messages come from the kernels ahead
   if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const float sf = (float)p.s;
@@ -228,7 +230,8 @@ int launch_fields(FieldParams& p, bool fused, cudaStream_t stream, bool* handled
   const uint32_t grid = (uint32_t)(want < cap ? want : cap);
   {
     ScopedKernel sk(kKernDecodeElias, stream);
-    kern<<<grid, warps * 32, smem, stream>>>(p);
+    const cudaError_t le = launch_chained(kern, grid, warps * 32, smem, stream, p);
+    if (le != cudaSuccess) return (int)le;
   }
   *handled = true;
   return (int)cudaGetLastError();
@@ -247,6 +250,8 @@ __global__ void __launch_bounds__(128) decode_elias_ranged_kernel(const __grid_c
   constexpr uint32_t kLevelWords = kR * LB / 32, kRowWords = kLevelWords + kR / 32;
   extern __shared__ __align__(16) uint32_t fsm[];
   __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
+  chain_release();
+  chain_wait();                                   // the messages come from the kernels ahead
   if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const float sf = (float)p.s;
@@ -400,7 +405,8 @@ int launch_ranged(FieldParams& p, bool fused, cudaStream_t stream, bool* handled
   const uint32_t grid = (uint32_t)(want < cap ? want : cap);
   {
     ScopedKernel sk(kKernDecodeElias, stream);
-    kern<<<grid, warps * 32, smem, stream>>>(p);
+    const cudaError_t le = launch_chained(kern, grid, warps * 32, smem, stream, p);
+    if (le != cudaSuccess) return (int)le;
   }
   *handled = true;
   return (int)cudaGetLastError();
@@ -446,6 +452,8 @@ __global__ void __launch_bounds__(512) decode_elias_bytes_kernel(const __grid_co
   extern __shared__ __align__(16) uint32_t fsm[];
   __shared__ uint16_t elias_lut[1u << kLutBits];
   __shared__ uint16_t level_lut[256];
+  chain_release();
+  chain_wait();                                   // the messages come from the kernels ahead
   if (p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const float sf = (float)p.s;
@@ -662,7 +670,8 @@ int launch_bytes(FieldParams& p, bool fused, cudaStream_t stream, bool* handled)
   const uint32_t grid = (uint32_t)(want < cap ? want : cap);
   {
     ScopedKernel sk(kKernDecodeElias, stream);
-    kern<<<grid, warps * 32, smem, stream>>>(p);
+    const cudaError_t le = launch_chained(kern, grid, warps * 32, smem, stream, p);
+    if (le != cudaSuccess) return (int)le;
   }
   *handled = true;
   return (int)cudaGetLastError();

@@ -58,6 +58,8 @@ template <typename CodeT, bool DENSE, bool FUSED>
 __global__ void __launch_bounds__(kThreads) decode_elias_slow_kernel(const __grid_constant__ EliasDecodeParams p) {
   extern __shared__ __align__(16) uint8_t smem[];
   __shared__ float xi[256];
+  chain_release();
+  chain_wait();                                   // the messages come from the kernels ahead
   if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const float sf = (float)p.s;
   for (uint32_t l = threadIdx.x; l < 256; l += kThreads) xi[l] = __fdiv_rn((float)l, sf);
@@ -176,7 +178,8 @@ int launch_slow(EliasDecodeParams& p, bool fused, cudaStream_t stream) {
   const uint32_t grid = (uint32_t)(want < cap ? want : cap);
   {
     ScopedKernel sk(kKernDecodeElias, stream);
-    kern<<<grid, kThreads, smem, stream>>>(p);
+    const cudaError_t le = launch_chained(kern, grid, kThreads, smem, stream, p);
+    if (le != cudaSuccess) return (int)le;
   }
   return (int)cudaGetLastError();
 }

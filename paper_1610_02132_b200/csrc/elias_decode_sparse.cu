@@ -21,6 +21,8 @@ template <bool FUSED>
 __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __grid_constant__ SparseParams p) {
   extern __shared__ __align__(16) uint32_t ssm[];
   __shared__ float xi[256];
+  chain_release();
+  chain_wait();                                   // the messages come from the kernels ahead
   if (p.check_regime && !sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const uint32_t G = p.sh.G, Kpad = p.sh.Kpad, R = p.sh.R, C = p.sh.C;
@@ -258,7 +260,8 @@ int launch_elias_sparse(const PeerSet& peers, uint32_t K, uint64_t n, uint32_t d
   const uint32_t grid = (uint32_t)(want < cap ? want : cap);
   {
     ScopedKernel sk(kKernDecodeEliasSparse, stream);
-    kern<<<grid, warps * 32, smem, stream>>>(p);
+    const cudaError_t le = launch_chained(kern, grid, warps * 32, smem, stream, p);
+    if (le != cudaSuccess) return (int)le;
   }
   *launched = true;
   return (int)cudaGetLastError();

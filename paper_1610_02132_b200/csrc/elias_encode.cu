@@ -426,8 +426,10 @@ __global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketPara
   __shared__ uint32_t warp_sum[kWarps];
   __shared__ uint32_t is_last;
   __shared__ uint32_t tab[17];
+  chain_release();
   fill_code_table(tab);
   __syncthreads();
+  chain_wait();                                    // the fields come from the kernel ahead
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t tl = lane & (p.lpb - 1), team = lane / p.lpb, bpw = 32 / p.lpb;
   const uint64_t b = (uint64_t)blockIdx.x * p.nbc + warp * bpw + team;
@@ -498,7 +500,7 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
   // whole code words (code | length << 16) of the integers met most: every level, and gaps below 64
   __shared__ uint32_t level_code[1u << LB];
   __shared__ uint32_t gap_code[64];
-  if (!ctrl->ok) return;
+  chain_release();
   fill_code_table(tab);
   if (!DENSE) {
     for (uint32_t k = threadIdx.x; k < (1u << LB) + 64u; k += kThreads) {
@@ -508,6 +510,8 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
       (k < (1u << LB) ? level_code[v] : gap_code[v]) = code | (ln << 16);
     }
   }
+  chain_wait();                                    // ctrl, lengths and sums come from the kernel ahead
+  if (!ctrl->ok) return;
   const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t tl = lane & (p.lpb - 1), team = lane / p.lpb, bpw = 32 / p.lpb;
   const uint64_t b = (uint64_t)blockIdx.x * p.nbc + warp * bpw + team;
@@ -661,7 +665,9 @@ int run_pipeline(BucketParams& bp, const EliasWs& w, uint32_t s, uint8_t* out, s
     sa.ctas = ctas; sa.out_capacity = out_capacity; sa.ctrl = w.ctrl; sa.out_bits = out_bits;
     sa.status_dev = status_dev; sa.out = out;
     ScopedKernel sk(kKernEliasLength, stream);
-    elias_length_kernel<LB, DENSE><<<(uint32_t)ctas, kThreads, 0, stream>>>(bp, w.len, w.lane_rec, w.cta_sums, sa);
+    const cudaError_t e = launch_chained(elias_length_kernel<LB, DENSE>, (uint32_t)ctas, kThreads, 0, stream, bp, w.len,
+                                         w.lane_rec, w.cta_sums, sa);
+    if (e != cudaSuccess) return (int)e;
   }
   {
     // staging: the longest legal strings of a CTA's buckets, plus the shared lead-in word
@@ -674,9 +680,8 @@ int run_pipeline(BucketParams& bp, const EliasWs& w, uint32_t s, uint8_t* out, s
       if (e != cudaSuccess) return (int)e;
     }
     ScopedKernel sk(kKernEliasScatter, stream);
-    kern<<<(uint32_t)ctas, kThreads, smem, stream>>>(bp, w.len, w.lane_rec, w.cta_sums, w.ctrl, out);
+    return (int)launch_chained(kern, (uint32_t)ctas, kThreads, smem, stream, bp, w.len, w.lane_rec, w.cta_sums, w.ctrl, out);
   }
-  return (int)cudaGetLastError();
 }
 
 }  // namespace

@@ -3,6 +3,8 @@
 #pragma once
 
 #include <cuda_runtime.h>
+
+#include <utility>
 #include <stdint.h>
 
 #include <mutex>
@@ -197,6 +199,33 @@ struct KernelSite {
 // Test hook: bound (in polls) of the waits inside the streaming encoder's main loop.
 void set_quantize_poll_limit(uint32_t polls);
 uint32_t default_quantize_poll_limit();
+
+// Programmatic dependent launch. Every kernel of the library is launched so that its CTAs may be
+// placed while the kernel ahead of it in the stream drains (the launch latency and the ramp-up hide
+// behind that kernel's tail: about 2 us per launch), and keeps the stream's order itself: it calls
+// chain_release() first thing and touches no global memory before chain_wait(), which returns once
+// the kernel ahead has completed and its writes are visible. A kernel launched the ordinary way
+// ahead of or behind these keeps the ordinary order.
+#ifdef __CUDACC__
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chained(void (*kern)(KArgs...), uint32_t grid, uint32_t block, size_t smem,
+                                  cudaStream_t stream, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+#endif
 
 struct ScopedKernel {
   ScopedKernel(KernelId id, cudaStream_t stream);

@@ -364,7 +364,9 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
 
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t grid = p.main_ctas;
+  chain_release();
   if (blockIdx.x >= grid) {                     // the extra CTA: ragged tail + padding
+    chain_wait();
     quantize_generic_tile<LB, NORM, MAPPED>(p.tail, 0u, 1u, sm.tile[0], sm.tile[1], sm.tile[1] + 1024);
     return;
   }
@@ -375,6 +377,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  chain_wait();                                 // nothing above touches global memory
   __syncthreads();
   if (MAPPED ? warp == 0 : tid == 0) {
     if (tid == 0 && blockIdx.x == 0 && p.info) {
@@ -775,7 +778,9 @@ quantize_warp_kernel(const __grid_constant__ FastParams p) {
   WarpRings& sm = *reinterpret_cast<WarpRings*>(smem_raw);
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t grid = p.main_ctas;
+  chain_release();
   if (blockIdx.x >= grid) {                     // the extra CTA: ragged tail + padding
+    chain_wait();
     float* scratch = &sm.chunk[0][0][0];
     quantize_generic_tile<LB, NORM, MAP != kNoMap>(p.tail, 0u, 1u, scratch, scratch + kTile, scratch + kTile + 1024);
     return;
@@ -785,10 +790,11 @@ quantize_warp_kernel(const __grid_constant__ FastParams p) {
   if (lane == 0) {
     for (int s = 0; s < kWarpStages; ++s) mbar_init(&sm.full[warp][s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    if (tid == 0 && blockIdx.x == 0 && p.info) {
-      p.info[0] = 8 * p.total_bytes; p.info[1] = 0; p.info[2] = p.total_bytes; p.info[3] = 0;
-    }
-    if (tid == 0 && blockIdx.x == 0 && p.clear_word) *p.clear_word = 0u;
+  }
+  chain_wait();                                 // nothing above touches global memory
+  if (tid == 0 && blockIdx.x == 0) {
+    if (p.info) { p.info[0] = 8 * p.total_bytes; p.info[1] = 0; p.info[2] = p.total_bytes; p.info[3] = 0; }
+    if (p.clear_word) *p.clear_word = 0u;
   }
   __syncwarp();
   for (int s = 0; s < kWarpStages; ++s) {
@@ -912,6 +918,8 @@ __global__ void __launch_bounds__(kThreads) quantize_generic_kernel(const Quanti
   __shared__ __align__(16) float tile[kTile];
   __shared__ float part[kTile / 8];
   __shared__ float s_rcp[kMaxBucketsPerTile];
+  chain_release();
+  chain_wait();
   quantize_generic_tile<LB, NORM, MAPPED>(p, blockIdx.x, gridDim.x, tile, part, s_rcp);
 }
 
@@ -945,8 +953,8 @@ int launch_warp(FastParams& fp, bool with_tail, cudaStream_t stream) {
   fp.main_ctas = fp.full_tiles < cap ? fp.full_tiles : cap;
   fp.poll_limit = g_poll_limit.load(std::memory_order_relaxed);
   ScopedKernel sk(kKernQuantize, stream);
-  quantize_warp_kernel<LB, NORM, MAP><<<fp.main_ctas + (with_tail ? 1u : 0u), kThreads, smem, stream>>>(fp);
-  return (int)cudaGetLastError();
+  return (int)launch_chained(quantize_warp_kernel<LB, NORM, MAP>, fp.main_ctas + (with_tail ? 1u : 0u), kThreads, smem,
+                             stream, fp);
 }
 
 // d >= 1024: the CTA-wide ring.
@@ -961,8 +969,8 @@ int launch_cross(FastParams& fp, bool with_tail, cudaStream_t stream) {
   fp.main_ctas = fp.full_tiles < cap ? fp.full_tiles : cap;
   fp.poll_limit = g_poll_limit.load(std::memory_order_relaxed);
   ScopedKernel sk(kKernQuantize, stream);
-  quantize_pow2_kernel<LB, NORM, MAPPED><<<fp.main_ctas + (with_tail ? 1u : 0u), kThreads, smem, stream>>>(fp);
-  return (int)cudaGetLastError();
+  return (int)launch_chained(quantize_pow2_kernel<LB, NORM, MAPPED>, fp.main_ctas + (with_tail ? 1u : 0u), kThreads, smem,
+                             stream, fp);
 }
 
 template <int LB, int NORM>
@@ -1003,10 +1011,9 @@ int launch_one(QuantizeParams& p, uint64_t seed, cudaStream_t stream) {
   if (tiles == 0) tiles = 1;
   {
     ScopedKernel sk(kKernQuantizeTail, stream);
-    if (p.map.src) quantize_generic_kernel<LB, NORM, true><<<(uint32_t)tiles, kThreads, 0, stream>>>(p);
-    else quantize_generic_kernel<LB, NORM, false><<<(uint32_t)tiles, kThreads, 0, stream>>>(p);
+    if (p.map.src) return (int)launch_chained(quantize_generic_kernel<LB, NORM, true>, (uint32_t)tiles, kThreads, 0, stream, p);
+    return (int)launch_chained(quantize_generic_kernel<LB, NORM, false>, (uint32_t)tiles, kThreads, 0, stream, p);
   }
-  return (int)cudaGetLastError();
 }
 
 template <int LB>

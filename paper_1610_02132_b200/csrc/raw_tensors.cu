@@ -27,6 +27,8 @@ __global__ void __launch_bounds__(kThreads) raw_gather_kernel(const float* __res
                                                             float* __restrict__ out_raw, uint64_t padded,
                                                             uint64_t* info, int has_compact) {
   const uint64_t j = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
+  chain_release();
+  chain_wait();
   if (j < raw.n_raw) {
     const uint64_t sgm = find_segment(raw.start, raw.R, j);
     out_raw[j] = g[__ldg(raw.src + sgm) + (j - __ldg(raw.start + sgm))];
@@ -53,6 +55,8 @@ template <bool FUSED>
 __global__ void __launch_bounds__(kThreads) raw_decode_kernel(const __grid_constant__ RawPeers peers, uint32_t K,
                                                             const RawSegments raw, float* __restrict__ out, float c) {
   const uint64_t j = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
+  chain_release();
+  chain_wait();
   if (j >= raw.n_raw) return;
   float acc = 0.f;
   for (uint32_t k = 0; k < K; ++k) acc = __fadd_rn(acc, __ldg(peers.region[k] + j));
@@ -70,9 +74,9 @@ int launch_raw_gather(const float* g, const RawSegments& raw, float* out_raw, ui
   const uint32_t grid = (uint32_t)((threads + kThreads - 1) / kThreads);
   {
     ScopedKernel sk(kKernRawGather, stream);
-    raw_gather_kernel<<<grid, kThreads, 0, stream>>>(g, raw, out_raw, padded, info, has_compact ? 1 : 0);
+    return (int)launch_chained(raw_gather_kernel, grid, kThreads, 0, stream, g, raw, out_raw, padded, info,
+                               has_compact ? 1 : 0);
   }
-  return (int)cudaGetLastError();
 }
 
 int launch_raw_decode(const float* const* raw_regions, uint32_t K, const RawSegments& raw, float* acc_or_x,
@@ -85,10 +89,9 @@ int launch_raw_decode(const float* const* raw_regions, uint32_t K, const RawSegm
   const float c = eta / (float)K;
   {
     ScopedKernel sk(kKernRawDecode, stream);
-    if (fused) raw_decode_kernel<true><<<grid, kThreads, 0, stream>>>(peers, K, raw, acc_or_x, c);
-    else raw_decode_kernel<false><<<grid, kThreads, 0, stream>>>(peers, K, raw, acc_or_x, c);
+    if (fused) return (int)launch_chained(raw_decode_kernel<true>, grid, kThreads, 0, stream, peers, K, raw, acc_or_x, c);
+    return (int)launch_chained(raw_decode_kernel<false>, grid, kThreads, 0, stream, peers, K, raw, acc_or_x, c);
   }
-  return (int)cudaGetLastError();
 }
 
 }  // namespace qsgd
