@@ -292,6 +292,8 @@ def run_cuda(args):
     import torch
     import torch.distributed as dist
     import paper_1610_02132_b200 as Q
+    if getattr(args, 'no_chaining', False):
+        Q.qsgd_set_launch_chaining(False)
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -507,6 +509,8 @@ def run_sweep(args):
     of 3), GB/s of fp32 gradient, algorithmic GB/s and fraction of the HBM peak."""
     import torch
     import paper_1610_02132_b200 as Q
+    if getattr(args, 'no_chaining', False):
+        Q.qsgd_set_launch_chaining(False)
     from paper_1610_02132_b200 import inputs as I
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -600,6 +604,8 @@ def run_multi(args):
     import torch
     import torch.distributed as dist
     import paper_1610_02132_b200 as Q
+    if getattr(args, 'no_chaining', False):
+        Q.qsgd_set_launch_chaining(False)
     from paper_1610_02132_b200 import exchange as X
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -812,6 +818,8 @@ def run_qsvrg(args):
     gradient arithmetic). Vectors of 16 KB make this launch-bound; reported for completeness."""
     import torch
     import paper_1610_02132_b200 as Q
+    if getattr(args, 'no_chaining', False):
+        Q.qsgd_set_launch_chaining(False)
     from paper_1610_02132_b200 import inputs as I
     from paper_1610_02132_b200 import qsvrg as GV
     if not torch.cuda.is_available():
@@ -887,6 +895,8 @@ def main():
     ap.add_argument("--K", type=int, default=None)
     ap.add_argument("--norm", default=None, choices=["l2", "max"])
     ap.add_argument("--codes", default=None, help="comma list of fixed,elias,elias_dense")
+    ap.add_argument("--no-chaining", action="store_true",
+                    help="plain stream-ordered launches (no programmatic dependent launch)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")

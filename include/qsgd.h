@@ -192,6 +192,17 @@ const char* qsgd_status_string(int status);
 uint64_t qsgd_launch_count(void);
 
 /*
+ * Launch chaining (the paper has no counterpart). By default every kernel of the library is launched
+ * with programmatic stream serialization: its launch is prepared while the kernel ahead of it in the
+ * stream still runs, and the kernel itself waits for that kernel to complete before it touches global
+ * memory, so the stream's order of reads and writes is the ordinary one. qsgd_set_launch_chaining(0)
+ * makes later launches of this process plain stream-ordered launches (for a profiler or a debugger
+ * that wants kernels strictly one after the other); nonzero turns chaining back on. Returns the
+ * previous setting.
+ */
+int qsgd_set_launch_chaining(int on);
+
+/*
  * TEST HOOK, not part of the codec (the paper has no counterpart). The streaming encoder waits for
  * its bulk copies with bounded polling; when a wait runs out the warp (or CTA) raises
  * QSGD_DEV_TIMEOUT in status_dev, stops encoding, still waits -- with the full built-in bound --

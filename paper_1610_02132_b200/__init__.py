@@ -7,4 +7,4 @@ from .binding import (CODE_ELIAS, CODE_ELIAS_DENSE, CODE_FIXED, NORM_L2, NORM_MA
                       qsgd_sgd_step, qsgd_static_scratch_bytes, qsgd_workspace_bytes,
                       Policy, qsgd_policy_decode_accumulate, qsgd_policy_decode_sgd_step,
                       qsgd_policy_encode, qsgd_policy_message_capacity, qsgd_policy_workspace_bytes,
-                      qsgd_test_default_wait_polls, qsgd_test_set_wait_polls)
+                      qsgd_test_default_wait_polls, qsgd_test_set_wait_polls, qsgd_set_launch_chaining)

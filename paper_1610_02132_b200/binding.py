@@ -23,7 +23,8 @@ EXPORTS = ["qsgd_message_capacity", "qsgd_workspace_bytes", "qsgd_fixed_layout",
            "qsgd_static_scratch_bytes", "qsgd_encode_elias_static",
            "qsgd_policy_plan_sizes", "qsgd_policy_plan", "qsgd_policy_message_capacity",
            "qsgd_policy_workspace_bytes", "qsgd_policy_encode", "qsgd_policy_decode_accumulate",
-           "qsgd_policy_decode_sgd_step", "qsgd_test_set_wait_polls", "qsgd_test_default_wait_polls"]
+           "qsgd_policy_decode_sgd_step", "qsgd_test_set_wait_polls", "qsgd_test_default_wait_polls",
+           "qsgd_set_launch_chaining"]
 
 _lib = None
 
@@ -95,6 +96,8 @@ def lib():
         L.qsgd_policy_decode_sgd_step.argtypes = [C.POINTER(vp), C.POINTER(vp), pu64, u32, pp, u32, u32,
                                                   C.c_int, vp, C.c_float, vp, vp]
         L.qsgd_policy_decode_sgd_step.restype = C.c_int
+        L.qsgd_set_launch_chaining.argtypes = [C.c_int]
+        L.qsgd_set_launch_chaining.restype = C.c_int
         L.qsgd_test_set_wait_polls.argtypes = [u32]
         L.qsgd_test_set_wait_polls.restype = None
         L.qsgd_test_default_wait_polls.argtypes = []
@@ -143,6 +146,11 @@ def qsgd_fixed_layout(n, bucket, s):
 
 def qsgd_launch_count():
     return int(lib().qsgd_launch_count())
+
+
+def qsgd_set_launch_chaining(on):
+    """Turns programmatic dependent launch of the library's kernels on or off; returns the previous setting."""
+    return bool(lib().qsgd_set_launch_chaining(1 if on else 0))
 
 
 def qsgd_test_set_wait_polls(polls):

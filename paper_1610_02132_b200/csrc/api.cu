@@ -9,6 +9,10 @@
 namespace qsgd {
 
 static std::atomic<uint64_t> g_launches{0};
+static std::atomic<bool> g_chaining{true};
+
+bool launch_chaining_enabled() { return g_chaining.load(std::memory_order_relaxed); }
+bool set_launch_chaining(bool on) { return g_chaining.exchange(on, std::memory_order_relaxed); }
 static std::atomic<int> g_profile{0};
 static std::mutex g_prof_mu;
 struct TimedLaunch { KernelId id; cudaEvent_t a, b; };
@@ -364,6 +368,8 @@ const char* qsgd_status_string(int status) {
     default: return status > 0 ? cudaGetErrorString((cudaError_t)status) : "unknown status";
   }
 }
+
+int qsgd_set_launch_chaining(int on) { return set_launch_chaining(on != 0) ? 1 : 0; }
 
 void qsgd_test_set_wait_polls(uint32_t polls) { set_quantize_poll_limit(polls); }
 

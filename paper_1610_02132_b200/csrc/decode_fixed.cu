@@ -44,7 +44,6 @@ __global__ void __launch_bounds__(kThreads, 4) decode_fixed_kernel(const __grid_
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float sf = (float)p.s;
   float lut0 = 0.f;                                  // this lane's +-(level / s)
-  chain_release();
   if (LB == 8) {
     for (uint32_t i = tid; i < 256 * 32; i += kThreads) xi_tab[i] = __fdiv_rn((float)(i >> 5), sf);
     __syncthreads();
@@ -106,7 +105,6 @@ __global__ void __launch_bounds__(kThreads) sgd_step_kernel(float* __restrict__ 
                                                            const float* __restrict__ acc, float c,
                                                            uint64_t n) {
   const uint64_t i0 = ((uint64_t)blockIdx.x * kThreads + threadIdx.x) * 4;
-  chain_release();
   chain_wait();
   if (i0 + 4 <= n) {
     const float4 a = __ldcs(reinterpret_cast<const float4*>(acc + i0));

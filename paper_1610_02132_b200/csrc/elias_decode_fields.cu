@@ -92,7 +92,6 @@ __global__ void __launch_bounds__(320) decode_elias_fields_kernel(const __grid_c
   extern __shared__ __align__(16) uint32_t fsm[];
   __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
   __shared__ uint16_t elias_lut[1u << kLutBits];
-  chain_release();
   chain_wait();                                   // the messages come from the kernels ahead
   if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -250,7 +249,6 @@ __global__ void __launch_bounds__(128) decode_elias_ranged_kernel(const __grid_c
   constexpr uint32_t kLevelWords = kR * LB / 32, kRowWords = kLevelWords + kR / 32;
   extern __shared__ __align__(16) uint32_t fsm[];
   __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
-  chain_release();
   chain_wait();                                   // the messages come from the kernels ahead
   if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -452,7 +450,6 @@ __global__ void __launch_bounds__(512) decode_elias_bytes_kernel(const __grid_co
   extern __shared__ __align__(16) uint32_t fsm[];
   __shared__ uint16_t elias_lut[1u << kLutBits];
   __shared__ uint16_t level_lut[256];
-  chain_release();
   chain_wait();                                   // the messages come from the kernels ahead
   if (p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;

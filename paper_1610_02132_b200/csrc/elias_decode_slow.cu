@@ -58,7 +58,6 @@ template <typename CodeT, bool DENSE, bool FUSED>
 __global__ void __launch_bounds__(kThreads) decode_elias_slow_kernel(const __grid_constant__ EliasDecodeParams p) {
   extern __shared__ __align__(16) uint8_t smem[];
   __shared__ float xi[256];
-  chain_release();
   chain_wait();                                   // the messages come from the kernels ahead
   if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const float sf = (float)p.s;

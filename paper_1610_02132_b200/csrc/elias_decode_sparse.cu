@@ -21,7 +21,6 @@ template <bool FUSED>
 __global__ void __launch_bounds__(256, 2) decode_elias_sparse_kernel(const __grid_constant__ SparseParams p) {
   extern __shared__ __align__(16) uint32_t ssm[];
   __shared__ float xi[256];
-  chain_release();
   chain_wait();                                   // the messages come from the kernels ahead
   if (p.check_regime && !sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;

@@ -426,7 +426,6 @@ __global__ void __launch_bounds__(kThreads) elias_length_kernel(const BucketPara
   __shared__ uint32_t warp_sum[kWarps];
   __shared__ uint32_t is_last;
   __shared__ uint32_t tab[17];
-  chain_release();
   fill_code_table(tab);
   __syncthreads();
   chain_wait();                                    // the fields come from the kernel ahead
@@ -500,7 +499,6 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
   // whole code words (code | length << 16) of the integers met most: every level, and gaps below 64
   __shared__ uint32_t level_code[1u << LB];
   __shared__ uint32_t gap_code[64];
-  chain_release();
   fill_code_table(tab);
   if (!DENSE) {
     for (uint32_t k = threadIdx.x; k < (1u << LB) + 64u; k += kThreads) {

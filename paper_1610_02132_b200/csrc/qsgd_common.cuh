@@ -200,14 +200,19 @@ struct KernelSite {
 void set_quantize_poll_limit(uint32_t polls);
 uint32_t default_quantize_poll_limit();
 
-// Programmatic dependent launch. Every kernel of the library is launched so that its CTAs may be
-// placed while the kernel ahead of it in the stream drains (the launch latency and the ramp-up hide
-// behind that kernel's tail: about 2 us per launch), and keeps the stream's order itself: it calls
-// chain_release() first thing and touches no global memory before chain_wait(), which returns once
-// the kernel ahead has completed and its writes are visible. A kernel launched the ordinary way
-// ahead of or behind these keeps the ordinary order.
+// Programmatic dependent launch. Every kernel of the library is launched with programmatic stream
+// serialization, so the launch of the next kernel is prepared while the one ahead still runs and its
+// CTAs are placed as that kernel's CTAs leave, and it keeps the stream's order itself: it touches no
+// global memory before chain_wait(), which returns once the kernel ahead has completed and its
+// writes are visible. No kernel releases its dependents early (griddepcontrol.launch_dependents):
+// measured, CTAs of a dependent that sit waiting beside running CTAs slow those down (a third on the
+// dense-code encode, whose length and scatter kernels run long), while leaving the release to each
+// CTA's exit gains 2 us per launch (3 % on back-to-back encodes) and never loses. A kernel launched
+// the ordinary way ahead of or behind these keeps the ordinary order.
+bool launch_chaining_enabled();
+bool set_launch_chaining(bool on);      // returns the previous setting
+
 #ifdef __CUDACC__
-__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;"); }
 __device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 template <typename... KArgs, typename... Args>
@@ -222,7 +227,7 @@ inline cudaError_t launch_chained(void (*kern)(KArgs...), uint32_t grid, uint32_
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = launch_chaining_enabled() ? 1 : 0;
   return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 #endif

@@ -364,7 +364,6 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
 
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t grid = p.main_ctas;
-  chain_release();
   if (blockIdx.x >= grid) {                     // the extra CTA: ragged tail + padding
     chain_wait();
     quantize_generic_tile<LB, NORM, MAPPED>(p.tail, 0u, 1u, sm.tile[0], sm.tile[1], sm.tile[1] + 1024);
@@ -778,7 +777,6 @@ quantize_warp_kernel(const __grid_constant__ FastParams p) {
   WarpRings& sm = *reinterpret_cast<WarpRings*>(smem_raw);
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t grid = p.main_ctas;
-  chain_release();
   if (blockIdx.x >= grid) {                     // the extra CTA: ragged tail + padding
     chain_wait();
     float* scratch = &sm.chunk[0][0][0];
@@ -918,7 +916,6 @@ __global__ void __launch_bounds__(kThreads) quantize_generic_kernel(const Quanti
   __shared__ __align__(16) float tile[kTile];
   __shared__ float part[kTile / 8];
   __shared__ float s_rcp[kMaxBucketsPerTile];
-  chain_release();
   chain_wait();
   quantize_generic_tile<LB, NORM, MAPPED>(p, blockIdx.x, gridDim.x, tile, part, s_rcp);
 }

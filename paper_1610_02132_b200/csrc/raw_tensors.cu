@@ -27,7 +27,6 @@ __global__ void __launch_bounds__(kThreads) raw_gather_kernel(const float* __res
                                                             float* __restrict__ out_raw, uint64_t padded,
                                                             uint64_t* info, int has_compact) {
   const uint64_t j = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
-  chain_release();
   chain_wait();
   if (j < raw.n_raw) {
     const uint64_t sgm = find_segment(raw.start, raw.R, j);
@@ -55,7 +54,6 @@ template <bool FUSED>
 __global__ void __launch_bounds__(kThreads) raw_decode_kernel(const __grid_constant__ RawPeers peers, uint32_t K,
                                                             const RawSegments raw, float* __restrict__ out, float c) {
   const uint64_t j = (uint64_t)blockIdx.x * kThreads + threadIdx.x;
-  chain_release();
   chain_wait();
   if (j >= raw.n_raw) return;
   float acc = 0.f;
