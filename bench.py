@@ -55,6 +55,25 @@ ETA = 0.1
 PHILOX_SEED = 7
 
 
+# The one JSON line goes to the process's real standard output; whatever libraries print on file
+# descriptor 1 meanwhile (NCCL announces its version there) is sent to standard error.
+_REAL_STDOUT = None
+
+
+def claim_stdout():
+    global _REAL_STDOUT
+    if _REAL_STDOUT is None:
+        sys.stdout.flush()
+        _REAL_STDOUT = os.fdopen(os.dup(1), "w")
+        os.dup2(2, 1)
+
+
+def emit(text):
+    out = _REAL_STDOUT if _REAL_STDOUT is not None else sys.stdout
+    out.write(text + "\n")
+    out.flush()
+
+
 def elen(k):
     return 1 if k == 1 else k.bit_length() + elen(k.bit_length() - 1)
 
@@ -497,7 +516,7 @@ def run_cuda(args):
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "roofline": roofline, "cpu_baseline": cpu, "phases": phases, "kernels": kern_tab,
         }
-        print(json.dumps(line))
+        emit(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
 
@@ -586,7 +605,7 @@ def run_sweep(args):
                     del msgs, ws
     ref = [p for p in points if (p["d"], p["s"], p["norm"], p["code"]) == (512, 15, "l2", "fixed")][0]
     value = (2 * K * 4 * n) / (K * ref["encode_us"] * 1e-6 + ref["decode_sgd_us"] * 1e-6) / 1e9
-    print(json.dumps({
+    emit(json.dumps({
         "metric": "QSGD encode + decode+aggregate throughput, fp32 gradient GB/s", "value": value, "unit": "GB/s",
         "n_gpus": 1, "steps": 3, "warmup": 1, "ms_per_step": (K * ref["encode_us"] + ref["decode_sgd_us"]) * 1e-3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
@@ -698,7 +717,7 @@ def run_multi(args):
     # fp32 gradient bytes through Encode (each worker once) plus through Decode (all K on every rank)
     grad_bytes = len(wl["codes"]) * (K * 4 * n + world * K * 4 * n)
     if rank == 0:
-        print(json.dumps({
+        emit(json.dumps({
             "metric": "QSGD encode + decode+aggregate throughput, fp32 gradient GB/s",
             "value": grad_bytes / (ms_step * 1e-3) / 1e9, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -729,7 +748,7 @@ def spawn_ranks(n_gpus):
     env.setdefault("NCCL_DEBUG", "VERSION")
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n_gpus),
            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
-    raise SystemExit(subprocess.call(cmd, env=env))
+    raise SystemExit(subprocess.call(cmd, env=env, stdout=_REAL_STDOUT))     # the ranks' JSON line goes to our real stdout
 
 
 # ------------------------------------------------------------------------------------------------
@@ -851,7 +870,7 @@ def run_qsvrg(args):
         "bits_per_processor": int(out["bits"][0]), "bound_bits": float((32 + 2.8 * n) * (T + 1)),
         "f_start": float(f(np.zeros(n))), "f_after_epoch": float(f(out["y"][-1].astype(np.float64))),
     }
-    print(json.dumps(line))
+    emit(json.dumps(line))
 
 
 def run_reference(args):
@@ -879,10 +898,11 @@ def run_reference(args):
         "cpu_baseline": cpu,
         "e2e": {"value": cpu["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
-    print(json.dumps(line))
+    emit(json.dumps(line))
 
 
 def main():
+    claim_stdout()
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
