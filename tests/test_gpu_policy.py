@@ -126,6 +126,12 @@ def test_policy_short_buckets_inside_the_stream(d, norm_kind):
     run_case(sizes, d, 3, norm_kind, O.CODE_ELIAS, K=2, tau=4096)
 
 
+@pytest.mark.parametrize("code_kind", [O.CODE_FIXED, O.CODE_ELIAS])
+def test_policy_long_raw_tensors(code_kind):
+    # a large threshold leaves long tensors raw
+    run_case([20000, 9001, 4096 * 12, 30, 17000], 512, 15, O.NORM_L2, code_kind, K=3, tau=30000)
+
+
 def test_policy_many_peers():
     run_case(RAGGED, 256, 7, O.NORM_L2, O.CODE_ELIAS, K=33, tau=4096)
 
