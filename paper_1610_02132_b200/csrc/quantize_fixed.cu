@@ -430,8 +430,12 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.empty[stage]);
     // a wait that ran out ends the loop; the decision is taken per CTA (the scales meet in
-    // shared memory), never per lane
-    const int flags = __syncthreads_or((arrived ? 0 : 1) | (shaky ? 2 : 0));
+    // shared memory), never per lane. __syncthreads_or tells only whether any thread's value was
+    // nonzero, so the ordinary tile costs one barrier and an unusual one two more to tell a
+    // timeout (bit 0) from a bucket that needs the fp64 path (bit 1).
+    int flags = 0;
+    if (__syncthreads_or((arrived ? 0 : 1) | (shaky ? 1 : 0)))
+      flags = (__syncthreads_or(arrived ? 0 : 1) ? 1 : 0) | (__syncthreads_or(shaky ? 1 : 0) ? 2 : 0);
     if (flags & 1) {
       if (lane == 0) atomicOr(p.status, QSGD_DEV_TIMEOUT);
       break;

@@ -1,0 +1,61 @@
+"""Seeded random shapes through the whole path on the GPU against the oracle: the parametrised
+parity tests pick their shapes by hand; these draw them (n, bucket size, s, norm, code kind, number
+of peers, input family) from a fixed seed, so that a shape nobody thought of gets its turn. Every
+case is small enough for the oracle to finish in well under a second."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_1610_02132_b200 import inputs as I
+from parity_util import decode_parity, encode_parity
+
+pytestmark = pytest.mark.gpu
+
+
+def draw_case(rng):
+    # bucket sizes: the streaming kernels' powers of two, the generic kernel's other multiples of 32
+    d = int(rng.choice([32, 64, 128, 256, 512, 512, 1024, 2048, 4096, 4096,
+                        32 * int(rng.integers(1, 80))]))
+    buckets = int(rng.integers(1, 1 + max(1, 200000 // d)))
+    n = max(1, buckets * d - int(rng.integers(0, d)))            # ragged last bucket more often than not
+    s = int(rng.choice([1, 2, 3, 4, 7, 15, 15, 16, 31, 64, 200, 255]))
+    norm_kind = int(rng.choice([O.NORM_L2, O.NORM_MAX]))
+    code_kind = int(rng.choice([O.CODE_FIXED, O.CODE_ELIAS, O.CODE_ELIAS, O.CODE_ELIAS_DENSE]))
+    K = int(rng.choice([1, 2, 3, 4, 5, 8, 16, 17, 33]))
+    family = str(rng.choice(["mixture", "gauss", "sparse", "tiny_values", "huge_values", "zeros_inside"]))
+    return n, d, s, norm_kind, code_kind, K, family
+
+
+def make_input(family, n, seed):
+    if family == "mixture":
+        return I.gaussian_mixture(n, seed=seed)
+    if family == "gauss":
+        return I.gaussian(n, 1.0, seed=seed)
+    if family == "sparse":
+        return I.sparse_laplace(n, 1e-3, 0.3, seed=seed)
+    if family == "tiny_values":                       # sums of squares far below fp32's normal range
+        return (I.gaussian(n, 1.0, seed=seed) * np.float32(1e-22)).astype(np.float32)
+    if family == "huge_values":                       # sums of squares beyond fp32's range
+        return (I.gaussian(n, 1.0, seed=seed) * np.float32(3e19)).astype(np.float32)
+    g = I.gaussian(n, 1.0, seed=seed)                 # whole stretches of exact zeros (zero buckets)
+    z = np.random.default_rng(seed).integers(0, n, size=4)
+    for a in z:
+        g[a: a + 3000] = 0.0
+    return g
+
+
+CASES = [draw_case(np.random.default_rng(1000 + i)) for i in range(72)]
+
+
+@pytest.mark.parametrize("case", CASES, ids=["n%d_d%d_s%d_norm%d_code%d_K%d_%s" % c for c in CASES])
+def test_random_shape_matches_oracle(case):
+    n, d, s, norm_kind, code_kind, K, family = case
+    msgs, infos = [], []
+    for w in range(K):
+        g = make_input(family, n, seed=300 + 7 * w)
+        m, info = encode_parity(g, d, s, norm_kind, code_kind, 11, 5, w)
+        msgs.append(m)
+        infos.append(info)
+    decode_parity(msgs, infos, n, d, s, code_kind, eta=0.05, x0=I.gaussian(n, 1.0, seed=77))
+    torch.cuda.synchronize()

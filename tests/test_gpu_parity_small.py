@@ -71,6 +71,26 @@ def test_degenerate_buckets(code_kind):
             assert np.all(acc[1536:] == 3.0)
 
 
+@pytest.mark.parametrize("d", [64, 512, 1024, 4096, 96])
+@pytest.mark.parametrize("scale", [1e-22, 3e19])
+@pytest.mark.parametrize("code_kind", [O.CODE_FIXED, O.CODE_ELIAS])
+def test_two_norm_outside_fp32_range(d, scale, code_kind):
+    """Buckets whose fp32 sum of squares underflows (values around 1e-22) or overflows (3e19) take the
+    fp64 path of every encoder (per-warp, CTA-wide for d >= 1024, generic), inside the streamed tiles
+    and in the tail, next to ordinary buckets; the encode must finish with status 0 and match."""
+    n = 5 * 4096 + 3 * d + 17
+    g = I.gaussian(n, 1.0, seed=3)
+    g[: 2 * 4096] *= np.float32(scale)                 # whole tiles out of range
+    g[3 * 4096 + d: 3 * 4096 + 2 * d] *= np.float32(scale)   # one bucket among ordinary ones
+    g[5 * 4096:] *= np.float32(scale)                  # the tail
+    msgs, infos = [], []
+    for w in range(2):
+        m, info = encode_parity(np.roll(g, 5 * w), d, 15, O.NORM_L2, code_kind, seed=2, step=1, worker=w)
+        msgs.append(m)
+        infos.append(info)
+    decode_parity(msgs, infos, n, d, 15, code_kind)
+
+
 @pytest.mark.parametrize("d", [128, 512, 4096])
 @pytest.mark.parametrize("shape", ["equal", "ascending", "descending", "one_large"])
 def test_two_norm_tolerance_on_adversarial_inputs(d, shape):
