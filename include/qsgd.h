@@ -105,9 +105,10 @@ int qsgd_fixed_layout(uint64_t n, uint32_t bucket, uint32_t s, uint64_t* layout)
  * rounded square root of a sum of squares that the streaming kernels (power-of-two bucket, at
  * least 4096 coordinates) accumulate in fp32 -- a chain of 16 fused multiply-adds per thread,
  * then a shuffle tree over the bucket's lanes, then, for buckets of 1024 and more, up to 8
- * sequential adds across warps -- and redo in fp64 when that sum leaves [8e-28, 1e30]; the
- * generic kernel (other shapes, ragged tail) sums 8 squares in fp32 and those partial sums in
- * fp64. Either way A lies within 1e-6 relative of the exact norm (at most 29 roundings of 2^-24
+ * sequential adds across warps -- and redo in fp64 when that sum leaves [8e-28, 1e30] (a sum of
+ * exactly zero included: squares below 1.4e-45 vanish in fp32 although the norm is representable);
+ * the generic kernel (other shapes, ragged tail) sums 8 squares in fp32 and those partial sums in
+ * fp64, and redoes a bucket in fp64 likewise. Either way A lies within 1e-6 relative of the exact norm (at most 29 roundings of 2^-24
  * on the sum, halved by the root), but the two kernels may give last-place differences for the
  * same bucket, so a message is reproducible for a given (n, bucket), not across shapes. A scale
  * below the smallest normal fp32 makes a zero bucket (A = +0, all levels 0). Per coordinate i (global index): u = Philox4x32-10(counter = (i / 4 lo,

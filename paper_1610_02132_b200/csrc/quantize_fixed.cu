@@ -422,7 +422,8 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
     // 2-norm: an fp32 sum of squares outside [8e-28, 1e30] may have lost bits to underflow or
     // overflowed; such buckets are redone in fp64 (rare, the CTA branches together)
     bool shaky = false;
-    if (NORM == QSGD_NORM_L2) shaky = !(part >= 8.0e-28f && part <= 1.0e30f) && part != 0.f;
+    // (a zero sum counts: squares below 1.4e-45 vanish in fp32 while the values do not in fp64)
+    if (NORM == QSGD_NORM_L2) shaky = !(part >= 8.0e-28f && part <= 1.0e30f);
     if (lane == 0) sm.wsum[it & 1][warp] = part;
 
     // ---- release the stage: every warp signals that its values are in registers; the producer
@@ -599,7 +600,9 @@ __device__ __forceinline__ void quantize_generic_tile(const QuantizeParams& p, u
   for (uint32_t b = warp; b < nb; b += kThreads / 32) {
     float A;
     if (NORM == QSGD_NORM_L2) {
-      // fp32 partials of 8 squares each; redo in fp64 from the tile when they may have lost bits
+      // fp32 partials of 8 squares each; redo in fp64 from the tile when they may have lost bits:
+      // a nonzero partial outside [8e-28, 1e30], or a bucket total below that range (a zero total
+      // too: squares below 1.4e-45 vanish in fp32 while the values do not in fp64)
       double acc = 0.0;
       bool shaky = false;
       for (uint32_t j = lane; j < gpb; j += 32) {
@@ -607,15 +610,17 @@ __device__ __forceinline__ void quantize_generic_tile(const QuantizeParams& p, u
         shaky |= !(q >= 8.0e-28f && q <= 1.0e30f) && q != 0.f;
         acc += (double)q;
       }
-      if (__any_sync(0xffffffffu, shaky)) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if (__any_sync(0xffffffffu, shaky) || !(acc >= 8.0e-28)) {
         acc = 0.0;
         for (uint32_t i = lane; i < p.d; i += 32) {
           const double x = (double)tile[b * p.d + i];
           acc = fma(x, x, acc);
         }
-      }
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      }
       A = __double2float_rn(__dsqrt_rn(acc));
     } else {
       float acc = 0.f;
@@ -870,7 +875,7 @@ quantize_warp_kernel(const __grid_constant__ FastParams p) {
     float A;
     bool shaky = false;
     if (NORM == QSGD_NORM_L2) {
-      shaky = !(part >= 8.0e-28f && part <= 1.0e30f) && part != 0.f;
+      shaky = !(part >= 8.0e-28f && part <= 1.0e30f);   // a zero sum too: tiny squares vanish in fp32
       A = __fsqrt_rn(part);
       if (__any_sync(0xffffffffu, shaky)) {
         double wide = 0.0;

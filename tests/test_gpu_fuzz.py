@@ -2,6 +2,8 @@
 parity tests pick their shapes by hand; these draw them (n, bucket size, s, norm, code kind, number
 of peers, input family) from a fixed seed, so that a shape nobody thought of gets its turn. Every
 case is small enough for the oracle to finish in well under a second."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -45,7 +47,10 @@ def make_input(family, n, seed):
     return g
 
 
-CASES = [draw_case(np.random.default_rng(1000 + i)) for i in range(72)]
+# QSGD_FUZZ_CASES / QSGD_FUZZ_POLICY_CASES draw more cases from the same seeds (the defaults are a prefix)
+N_CASES = int(os.environ.get("QSGD_FUZZ_CASES", "72"))
+N_POLICY_CASES = int(os.environ.get("QSGD_FUZZ_POLICY_CASES", "40"))
+CASES = [draw_case(np.random.default_rng(1000 + i)) for i in range(N_CASES)]
 
 
 @pytest.mark.parametrize("case", CASES, ids=["n%d_d%d_s%d_norm%d_code%d_K%d_%s" % c for c in CASES])
@@ -59,3 +64,40 @@ def test_random_shape_matches_oracle(case):
         infos.append(info)
     decode_parity(msgs, infos, n, d, s, code_kind, eta=0.05, x0=I.gaussian(n, 1.0, seed=77))
     torch.cuda.synchronize()
+
+
+def draw_policy_case(rng):
+    d = int(rng.choice([32, 128, 256, 512, 512, 1024, 4096, 32 * int(rng.integers(1, 40))]))
+    aligned = bool(rng.integers(0, 2))                 # every size a multiple of 4: the bulk-copy paths
+    T = int(rng.integers(1, 12))
+    sizes = []
+    for _ in range(T):
+        kind = int(rng.integers(0, 4))
+        if kind == 0:
+            m = int(rng.integers(1, 300))                                  # stays raw
+        elif kind == 1:
+            m = int(rng.integers(1, 40)) * d                               # whole buckets
+        elif kind == 2:
+            m = int(rng.integers(4096, 60000))                             # ends in a short bucket
+        else:
+            m = 4096 * int(rng.integers(1, 12)) + int(rng.integers(0, 9))  # several tiles, tiny remainder
+        if aligned:
+            m = max(4, m // 4 * 4)
+        sizes.append(m)
+    s = int(rng.choice([1, 3, 7, 15, 64, 255]))
+    norm_kind = int(rng.choice([O.NORM_L2, O.NORM_MAX]))
+    code_kind = int(rng.choice([O.CODE_FIXED, O.CODE_ELIAS, O.CODE_ELIAS_DENSE]))
+    K = int(rng.choice([1, 2, 3, 5, 16]))
+    tau = int(rng.choice([1, 1000, 4096, 10000, 50000]))
+    return tuple(sizes), d, s, norm_kind, code_kind, K, tau
+
+
+POLICY_CASES = [draw_policy_case(np.random.default_rng(5000 + i)) for i in range(N_POLICY_CASES)]
+
+
+@pytest.mark.parametrize("case", POLICY_CASES,
+                         ids=["T%d_n%d_d%d_s%d_norm%d_code%d_K%d_tau%d" % (len(c[0]), sum(c[0]), *c[1:]) for c in POLICY_CASES])
+def test_random_policy_matches_oracle(case):
+    from test_gpu_policy import run_case
+    sizes, d, s, norm_kind, code_kind, K, tau = case
+    run_case(list(sizes), d, s, norm_kind, code_kind, K=K, tau=tau)

@@ -91,6 +91,26 @@ def test_two_norm_outside_fp32_range(d, scale, code_kind):
     decode_parity(msgs, infos, n, d, 15, code_kind)
 
 
+@pytest.mark.parametrize("d", [64, 512, 1024, 96])
+def test_two_norm_of_vanishing_squares(d):
+    """Values whose squares are below fp32's smallest subnormal (|v| < 3.7e-23) give an fp32 sum of
+    squares of exactly zero, yet their norm is far above FLT_MIN: such buckets are not zero buckets.
+    One among the streamed tiles, one in the tail, and a last bucket of a single coordinate."""
+    B = (3 * 4096) // d + 3                           # buckets, the last of one coordinate
+    n = (B - 1) * d + 1
+    g = I.gaussian(n, 1.0, seed=8)
+    sign = np.where(np.arange(d) % 3 == 0, -1.0, 1.0).astype(np.float32)
+    early, late = 4096 // d + 1, B - 2                # a bucket inside the streamed tiles, one in the tail
+    g[early * d: (early + 1) * d] = np.float32(2e-23) * sign
+    g[late * d: (late + 1) * d] = np.float32(3e-23) * sign
+    g[-1] = np.float32(1.5e-23)
+    for code_kind in (O.CODE_FIXED, O.CODE_ELIAS):
+        m, info = encode_parity(g, d, 15, O.NORM_L2, code_kind, seed=2, step=1, worker=0)
+        acc, _ = decode_parity([m], [info], n, d, 15, code_kind, eta=1.0)
+        assert acc[-1] != 0.0                         # a bucket of one value: level s, decoded to the value itself
+        assert np.any(acc[early * d: (early + 1) * d] != 0.0) and np.any(acc[late * d: (late + 1) * d] != 0.0)
+
+
 @pytest.mark.parametrize("d", [128, 512, 4096])
 @pytest.mark.parametrize("shape", ["equal", "ascending", "descending", "one_large"])
 def test_two_norm_tolerance_on_adversarial_inputs(d, shape):
