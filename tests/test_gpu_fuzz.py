@@ -63,6 +63,9 @@ def test_random_shape_matches_oracle(case):
         msgs.append(m)
         infos.append(info)
     decode_parity(msgs, infos, n, d, s, code_kind, eta=0.05, x0=I.gaussian(n, 1.0, seed=77))
+    if code_kind != O.CODE_FIXED and (n + K) % 2 == 0:
+        # offset tables kept in front of the payloads: the library cannot read sizes off the pointers
+        decode_parity(msgs, infos, n, d, s, code_kind, eta=0.05, x0=I.gaussian(n, 1.0, seed=77), tables_first=True)
     torch.cuda.synchronize()
 
 
@@ -101,3 +104,29 @@ def test_random_policy_matches_oracle(case):
     from test_gpu_policy import run_case
     sizes, d, s, norm_kind, code_kind, K, tau = case
     run_case(list(sizes), d, s, norm_kind, code_kind, K=K, tau=tau)
+
+
+def draw_mid_case(rng):
+    # enough tiles for every persistent warp / CTA of the streaming encoders to go round its ring
+    # of stages several times (2.4 M coordinates fill the grid once)
+    d = int(rng.choice([32, 128, 512, 1024, 4096]))
+    n = int(rng.integers(5_000_000, 14_000_000))
+    s = int(rng.choice([1, 3, 15, 255]))
+    norm_kind = int(rng.choice([O.NORM_L2, O.NORM_MAX]))
+    code_kind = int(rng.choice([O.CODE_FIXED, O.CODE_ELIAS, O.CODE_ELIAS_DENSE]))
+    family = str(rng.choice(["mixture", "sparse", "zeros_inside"]))
+    return n, d, s, norm_kind, code_kind, family
+
+
+MID_CASES = [draw_mid_case(np.random.default_rng(9000 + i)) for i in range(int(os.environ.get("QSGD_FUZZ_MID_CASES", "10")))]
+
+
+@pytest.mark.parametrize("case", MID_CASES, ids=["n%d_d%d_s%d_norm%d_code%d_%s" % c for c in MID_CASES])
+def test_random_mid_size_matches_oracle(case):
+    n, d, s, norm_kind, code_kind, family = case
+    msgs, infos = [], []
+    for w in range(2):
+        m, info = encode_parity(make_input(family, n, seed=40 + w), d, s, norm_kind, code_kind, 3, 9, w)
+        msgs.append(m)
+        infos.append(info)
+    decode_parity(msgs, infos, n, d, s, code_kind, eta=0.05, x0=I.gaussian(n, 1.0, seed=78))
