@@ -44,9 +44,11 @@ def test_wait_gives_up_and_kernel_returns(zero_polls, d, code_kind):
     encode_parity(g.cpu().numpy(), d, s, O.NORM_L2, code_kind, seed=7, step=0, worker=0)
 
 
-def test_wait_gives_up_under_policy(zero_polls):
+@pytest.mark.parametrize("bucket", [512, 128, 4096])
+def test_wait_gives_up_under_policy(zero_polls, bucket):
+    # one bucket per chunk, several per chunk (each lane starts its own copy), and the CTA-wide ring
     sizes = [30000, 700, 4096 * 6 + 8, 20000]
-    bucket, s = 512, 15
+    s = 15
     plan = Q.Policy(sizes, bucket)
     g = torch.from_numpy(I.gaussian(sum(sizes), 0.01, seed=4)).cuda()
     cap = Q.qsgd_policy_message_capacity(plan, s, O.CODE_FIXED)
