@@ -1,14 +1,17 @@
 // Encode, fixed-width path: bucket scale + Philox stochastic rounding + bit packing in one pass
 // over the gradient (Section 3.1, Eq. 2; Section 4 bucketing / max-norm; Section 5 bit widths).
 //
-// Two streaming kernels for power-of-two bucket sizes, both persistent and fed by 1-D TMA bulk
+// Three streaming kernels for power-of-two bucket sizes, all persistent and fed by 1-D TMA bulk
 // copies (cp.async.bulk + mbarrier), so no thread spends instructions on global loads:
 //   * quantize_warp_kernel (d <= 512, with or without a bucket map): every warp runs its own pipeline over
 //     chunks of 512 coordinates (whole buckets) with a private ring of shared-memory stages that
 //     its lane 0 refills as soon as the warp has taken a stage into registers. No CTA-wide
 //     barrier and no separate "empty" barrier exist, and every decision is warp-uniform.
-//   * quantize_pow2_kernel (d >= 1024): the CTA walks
-//     tiles of 4096 coordinates through a shared ring; scales of buckets that span several
+//   * quantize_group_kernel (d >= 1024, 2-norm, no bucket map): the same per-warp pipelines; the
+//     warps that share a bucket meet once per chunk at a named barrier of their own to exchange
+//     their partial sums.
+//   * quantize_pow2_kernel (d >= 1024, max-norm or bucket map, where it measures faster): the CTA
+//     walks tiles of 4096 coordinates through a shared ring; scales of buckets that span several
 //     warps meet in shared memory.
 // A thread owns 16 consecutive coordinates: it pulls them into registers once, the bucket scale
 // is reduced with shuffles, and the same registers are then quantized, so the gradient is read
@@ -414,6 +417,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
       if (NORM == QSGD_NORM_L2) part = fmaf(v[e], v[e], part);
       else part = fmaxf(part, fabsf(v[e]));
     }
+    const float mine = part;                                       // this thread's share of the scale
 #pragma unroll
     for (uint32_t o = 16; o > 0; o >>= 1) {
       const float q = __shfl_xor_sync(0xffffffffu, part, o);
@@ -463,6 +467,7 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
       }
     }
     float A;
+    bool clamp = true;
     {
       const uint32_t w0 = warp & ~(wpb - 1u);
       float acc = 0.f;
@@ -472,6 +477,9 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
       }
       if (NORM == QSGD_NORM_L2) {
         A = __fsqrt_rn(acc);
+        // no per-coordinate clamp where no thread of the warp holds (nearly) all of its bucket's
+        // sum of squares: see the per-warp kernel
+        clamp = (flags & 2) || __any_sync(0xffffffffu, !(mine <= 0.9f * acc));
         if (flags & 2) {                      // some bucket of this tile needs the fp64 path
           double wide = 0.0;
 #pragma unroll
@@ -497,7 +505,8 @@ quantize_pow2_kernel(const __grid_constant__ FastParams p) {
     float um[16];
     philox_uniforms16(t * (kTile / 4) + tid * 4, p.pc, um);
     uint32_t sw, lw[4];
-    quantize16<LB, true>(v, um, r, sf, cap, lw, sw);
+    if (clamp) quantize16<LB, true>(v, um, r, sf, cap, lw, sw);
+    else quantize16<LB, false>(v, um, r, sf, cap, lw, sw);
     if (LB != 8) sw &= nonzero_fields16<LB>(lw);          // canonical sign: 0 where the level is 0
 
     store_chunk<LB>(p.sign_out, p.level_out, t * (kTile / 512) + warp, lane, sw, lw);
@@ -920,6 +929,180 @@ quantize_warp_kernel(const __grid_constant__ FastParams p) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Per-warp pipelines for d >= 1024: a bucket is 2^(log2d - 9) consecutive chunks, taken by as
+// many neighbouring warps of one CTA (a group). Each warp streams its chunk exactly as in
+// quantize_warp_kernel; once per chunk the group's warps meet at a named barrier of their own to
+// exchange their partial sums (and the "my wait ran out" / "my sum left the fp32 range" flags, so
+// that the whole group takes the same path). No CTA-wide barrier, no producer thread.
+// ---------------------------------------------------------------------------------------------
+struct __align__(16) GroupRings {
+  WarpRings rings;
+  float wsum[2][kThreads / 32];
+  uint32_t wflag[2][kThreads / 32];
+  double wsum64[kThreads / 32];
+};
+
+__device__ __forceinline__ void group_barrier(uint32_t id, uint32_t threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// With a bucket map: the piece of bucket (chunk / chunks-per-bucket) that this chunk covers.
+template <bool MAPPED>
+__device__ __forceinline__ MappedBucket fetch_piece(const FastParams& p, uint32_t chunk, uint32_t chunks,
+                                                    uint32_t lane) {
+  MappedBucket mb{0ull, 0u};
+  if (MAPPED && chunk < chunks && lane == 0) {
+    const uint32_t sh = p.log2d - 9u;
+    const uint64_t b = chunk >> sh;
+    const uint32_t off = (chunk & ((1u << sh) - 1u)) << 9;
+    const uint32_t L = min(__ldg(p.map.len + b), 1u << p.log2d);
+    mb.src = __ldg(p.map.src + b) + off;
+    mb.len = L > off ? min(L - off, (uint32_t)kChunk) : 0u;
+  }
+  return mb;
+}
+
+template <int LB, int NORM, bool MAPPED>
+__global__ void __launch_bounds__(kThreads, 4)
+quantize_group_kernel(const __grid_constant__ FastParams p) {
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  GroupRings& gs = *reinterpret_cast<GroupRings*>(smem_raw);
+  WarpRings& sm = gs.rings;
+  constexpr int MAP = MAPPED ? kMapOnePerChunk : kNoMap;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t grid = p.main_ctas;
+  if (blockIdx.x >= grid) {                     // the extra CTA: ragged tail + padding
+    chain_wait();
+    float* scratch = &sm.chunk[0][0][0];
+    quantize_generic_tile<LB, NORM, MAPPED>(p.tail, 0u, 1u, scratch, scratch + kTile, scratch + kTile + 1024);
+    return;
+  }
+  const uint32_t chunks = p.full_tiles * (kTile / kChunk), stride = grid * (kThreads / 32);
+  uint32_t c = blockIdx.x * (kThreads / 32) + warp;
+  if (lane == 0) {
+    for (int s = 0; s < kWarpStages; ++s) mbar_init(&sm.full[warp][s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  chain_wait();                                 // nothing above touches global memory
+  if (tid == 0 && blockIdx.x == 0) {
+    if (p.info) { p.info[0] = 8 * p.total_bytes; p.info[1] = 0; p.info[2] = p.total_bytes; p.info[3] = 0; }
+    if (p.clear_word) *p.clear_word = 0u;
+  }
+  __syncwarp();
+  for (int s = 0; s < kWarpStages; ++s) {
+    const uint32_t cs = c + (uint32_t)s * stride;
+    if (cs < chunks) {
+      const MappedBucket mb = fetch_piece<MAPPED>(p, cs, chunks, lane);
+      arm_chunk<MAP>(p, sm.chunk[warp][s], &sm.full[warp][s], cs, lane, mb);
+    }
+  }
+  MappedBucket ahead = fetch_piece<MAPPED>(p, c + (uint32_t)kWarpStages * stride, chunks, lane);
+
+  const float sf = (float)p.s;
+  const float cap = kTwo23 + sf;
+  const uint32_t wpb = 1u << (p.log2d - 9);                      // warps per bucket = warps of a group
+  const uint32_t w0 = warp & ~(wpb - 1u);                        // first warp of this warp's group
+  const uint32_t bar_id = 1u + (w0 >> (p.log2d - 9));            // named barriers 1 .. 4
+  const bool leader = warp == w0 && lane == 0;
+
+  uint32_t stage = 0, phase = 0, it = 0;
+  for (; c < chunks; c += stride, ++it) {
+    const float* src = sm.chunk[warp][stage];
+    const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(&sm.full[warp][stage], phase, p.poll_limit));
+
+    float v[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float4 a = *reinterpret_cast<const float4*>(src + lane * 16 + j * 4);
+      v[4 * j] = a.x; v[4 * j + 1] = a.y; v[4 * j + 2] = a.z; v[4 * j + 3] = a.w;
+    }
+    float um[16];
+    philox_uniforms16(c * (kChunk / 4) + lane * 4, p.pc, um);
+    float part = 0.f;
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      if (NORM == QSGD_NORM_L2) part = fmaf(v[e], v[e], part);
+      else part = fmaxf(part, fabsf(v[e]));
+    }
+    const float mine = part;
+#pragma unroll
+    for (uint32_t o = 16; o > 0; o >>= 1) {
+      const float q = __shfl_xor_sync(0xffffffffu, part, o);
+      part = (NORM == QSGD_NORM_L2) ? part + q : fmaxf(part, q);
+    }
+    bool shaky = false;
+    if (NORM == QSGD_NORM_L2) shaky = !(part >= 8.0e-28f && part <= 1.0e30f);   // a zero sum too
+    const uint32_t par = it & 1u;
+    if (lane == 0) {
+      gs.wsum[par][warp] = part;
+      gs.wflag[par][warp] = (ok ? 0u : 1u) | (shaky ? 2u : 0u);
+    }
+
+    // ---- the stage is in registers: refill it (not after a wait that ran out: its copy may still land)
+    __syncwarp();
+    {
+      const uint32_t cn = c + (uint32_t)kWarpStages * stride;
+      if (ok && cn < chunks) arm_chunk<MAP>(p, sm.chunk[warp][stage], &sm.full[warp][stage], cn, lane, ahead);
+      ahead = fetch_piece<MAPPED>(p, cn + stride, chunks, lane);
+    }
+
+    // ---- the group's warps exchange their sums ---------------------------------------------------
+    group_barrier(bar_id, 32u * wpb);
+    float acc = 0.f;
+    uint32_t fl = 0u;
+    for (uint32_t w = 0; w < wpb; ++w) {
+      const float q = gs.wsum[par][w0 + w];
+      acc = (NORM == QSGD_NORM_L2) ? acc + q : fmaxf(acc, q);
+      fl |= gs.wflag[par][w0 + w];
+    }
+    float A;
+    if (NORM == QSGD_NORM_L2) {
+      A = __fsqrt_rn(acc);
+      if (fl & 2u) {                          // some warp's sum left the fp32 range: the bucket again in fp64
+        double wide = 0.0;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) wide = fma((double)v[e], (double)v[e], wide);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) wide += __shfl_xor_sync(0xffffffffu, wide, o);
+        if (lane == 0) gs.wsum64[warp] = wide;
+        group_barrier(bar_id, 32u * wpb);
+        wide = 0.0;
+        for (uint32_t w = 0; w < wpb; ++w) wide += gs.wsum64[w0 + w];
+        A = __double2float_rn(sqrt(wide));
+        group_barrier(bar_id, 32u * wpb);
+      }
+    } else {
+      A = acc;
+    }
+    if (!ok) {                                 // this warp's wait ran out: it leaves with its stage still armed
+      if (lane == 0) atomicOr(p.status, QSGD_DEV_TIMEOUT);
+      break;
+    }
+    if (!(A >= FLT_MIN)) A = 0.f;                      // zero bucket: Q(0) = 0
+    const float r = A > 0.f ? __frcp_rn(A) : 0.f;
+    if (leader) p.A_out[c >> (p.log2d - 9)] = A;
+
+    uint32_t sw, lw[4];
+    bool clamp = true;
+    if (NORM == QSGD_NORM_L2) clamp = (fl & 2u) || __any_sync(0xffffffffu, !(mine <= 0.9f * acc));
+    if (clamp) quantize16<LB, true>(v, um, r, sf, cap, lw, sw);
+    else quantize16<LB, false>(v, um, r, sf, cap, lw, sw);
+    if (LB != 8) sw &= nonzero_fields16<LB>(lw);          // canonical sign: 0 where the level is 0
+    store_chunk<LB>(p.sign_out, p.level_out, c, lane, sw, lw);
+    if (++stage == kWarpStages) { stage = 0; phase ^= 1; }
+    if (fl & 1u) { c += stride; break; }       // another warp of the group gave up: the group stops together
+  }
+
+  // Leave no bulk copy in flight: a warp that stopped early waits (bounded) for the stages it armed.
+  if (lane == 0 && c < chunks) {
+    for (uint32_t j = 0; j < (uint32_t)kWarpStages; ++j) {
+      if (c + j * stride < chunks) mbar_wait_bounded(&sm.full[warp][stage], phase, kDrainPolls);
+      if (++stage == kWarpStages) { stage = 0; phase ^= 1; }
+    }
+  }
+}
+
 template <int LB, int NORM, bool MAPPED>
 __global__ void __launch_bounds__(kThreads) quantize_generic_kernel(const QuantizeParams p) {
   __shared__ __align__(16) float tile[kTile];
@@ -963,7 +1146,22 @@ int launch_warp(FastParams& fp, bool with_tail, cudaStream_t stream) {
                              stream, fp);
 }
 
-// d >= 1024: the CTA-wide ring.
+template <int LB, int NORM, bool MAPPED>
+int launch_group(FastParams& fp, bool with_tail, cudaStream_t stream) {
+  static KernelSite site;
+  const size_t smem = sizeof(GroupRings) + 128;
+  int sms = 0, ctas_per_sm = 0;
+  const int st = site.lookup(quantize_group_kernel<LB, NORM, MAPPED>, kThreads, smem, &sms, &ctas_per_sm);
+  if (st) return st;
+  const uint32_t cap = (uint32_t)(sms * ctas_per_sm);
+  fp.main_ctas = fp.full_tiles < cap ? fp.full_tiles : cap;
+  fp.poll_limit = g_poll_limit.load(std::memory_order_relaxed);
+  ScopedKernel sk(kKernQuantize, stream);
+  return (int)launch_chained(quantize_group_kernel<LB, NORM, MAPPED>, fp.main_ctas + (with_tail ? 1u : 0u), kThreads, smem,
+                             stream, fp);
+}
+
+// d >= 1024, max-norm or bucket map: the CTA-wide ring.
 template <int LB, int NORM, bool MAPPED>
 int launch_cross(FastParams& fp, bool with_tail, cudaStream_t stream) {
   static KernelSite site;
@@ -1004,8 +1202,16 @@ int launch_one(QuantizeParams& p, uint64_t seed, cudaStream_t stream) {
     fp.tail = p;
     fp.tail.info = nullptr;
     fp.tail.clear_word = nullptr;
-    if (d >= 1024) return fp.map.src ? launch_cross<LB, NORM, true>(fp, with_tail, stream)
-                                     : launch_cross<LB, NORM, false>(fp, with_tail, stream);
+    if (d >= 1024) {
+      // measured (n = 60 M, s = 15 / 255): with the 2-norm the per-warp pipelines with group barriers
+      // take 83-86 us against the CTA-wide ring's 90-92; with the max-norm (100 against 84) and under a
+      // bucket map (101 against 97) the ring is the faster one
+      if constexpr (NORM == QSGD_NORM_L2) {
+        if (!fp.map.src) return launch_group<LB, NORM, false>(fp, with_tail, stream);
+      }
+      return fp.map.src ? launch_cross<LB, NORM, true>(fp, with_tail, stream)
+                        : launch_cross<LB, NORM, false>(fp, with_tail, stream);
+    }
     if (!fp.map.src) return launch_warp<LB, NORM, kNoMap>(fp, with_tail, stream);
     return d == (uint32_t)kChunk ? launch_warp<LB, NORM, kMapOnePerChunk>(fp, with_tail, stream)
                                  : launch_warp<LB, NORM, kMapSeveralPerChunk>(fp, with_tail, stream);

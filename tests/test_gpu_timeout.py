@@ -24,10 +24,13 @@ def zero_polls():
         Q.qsgd_test_set_wait_polls(Q.qsgd_test_default_wait_polls())
 
 
-# per-warp rings (d <= 512), the CTA ring (d >= 1024) and the CTA ring behind a bucket map
-@pytest.mark.parametrize("d,code_kind", [(512, O.CODE_FIXED), (128, O.CODE_FIXED), (4096, O.CODE_FIXED),
-                                         (512, O.CODE_ELIAS)])
-def test_wait_gives_up_and_kernel_returns(zero_polls, d, code_kind):
+# per-warp rings (d <= 512), per-warp rings with group barriers (d >= 1024, 2-norm: warps of a group
+# must stop together), the CTA ring (d >= 1024, max-norm)
+@pytest.mark.parametrize("d,code_kind,norm_kind", [(512, O.CODE_FIXED, O.NORM_L2), (128, O.CODE_FIXED, O.NORM_L2),
+                                                   (4096, O.CODE_FIXED, O.NORM_L2), (1024, O.CODE_FIXED, O.NORM_L2),
+                                                   (4096, O.CODE_FIXED, O.NORM_MAX), (2048, O.CODE_ELIAS, O.NORM_MAX),
+                                                   (512, O.CODE_ELIAS, O.NORM_L2)])
+def test_wait_gives_up_and_kernel_returns(zero_polls, d, code_kind, norm_kind):
     n, s = 40 * 4096 + 77, 15
     g = torch.from_numpy(I.gaussian(n, 0.01, seed=3)).cuda()
     cap = Q.qsgd_message_capacity(n, d, s, code_kind)
@@ -35,13 +38,13 @@ def test_wait_gives_up_and_kernel_returns(zero_polls, d, code_kind):
     bits = torch.zeros(4, dtype=torch.int64, device="cuda")
     ws = torch.empty(max(Q.qsgd_workspace_bytes(n, d, s, code_kind), 16), dtype=torch.uint8, device="cuda")
     status = Q.new_status()
-    Q.qsgd_encode(g, d, s, O.NORM_L2, code_kind, 7, 0, 0, big[:cap], bits, ws, status)
+    Q.qsgd_encode(g, d, s, norm_kind, code_kind, 7, 0, 0, big[:cap], bits, ws, status)
     torch.cuda.synchronize()                                   # the kernels came back
     assert int(status.item()) & Q.binding.DEV_TIMEOUT
     assert bool((big[cap:] == CANARY).all()), "write past the message buffer"
     # the device still answers, and with the default bound the same call is exact again
     Q.qsgd_test_set_wait_polls(Q.qsgd_test_default_wait_polls())
-    encode_parity(g.cpu().numpy(), d, s, O.NORM_L2, code_kind, seed=7, step=0, worker=0)
+    encode_parity(g.cpu().numpy(), d, s, norm_kind, code_kind, seed=7, step=0, worker=0)
 
 
 @pytest.mark.parametrize("bucket", [512, 128, 4096])
