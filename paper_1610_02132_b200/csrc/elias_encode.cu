@@ -282,10 +282,33 @@ __device__ __forceinline__ LaneSummary summarize_sparse(const uint32_t* tab, con
   return s;
 }
 
+// whole_blocks as above: whole level words are loaded once and their fields taken from the register
+// (fields past the end of the vector are zero in the fixed-width layout but are not coordinates: the
+// count stops at c_hi).
 template <int LB>
 __device__ __forceinline__ uint32_t summarize_dense(const uint32_t* tab, const uint32_t* __restrict__ lwb,
-                                                    uint32_t c_lo, uint32_t c_hi) {
+                                                    uint32_t c_lo, uint32_t c_hi, bool whole_blocks) {
   uint32_t bits = 0;
+  if (whole_blocks) {
+    constexpr uint32_t kFields = 32u / LB, kMask = (1u << LB) - 1u;
+    for (uint32_t c0 = c_lo; c0 < c_hi; c0 += 64u) {
+      const uint32_t* wp = lwb + ((c0 * LB) >> 5);
+#pragma unroll
+      for (uint32_t j = 0; j < 2u * LB; ++j) {
+        const uint32_t cw = c0 + j * kFields;                 // first coordinate of this word
+        if (cw >= c_hi) break;
+        const uint32_t w = __ldg(wp + j);
+        const uint32_t cnt = min(kFields, c_hi - cw);
+        if (cnt == kFields) {
+#pragma unroll
+          for (uint32_t f = 0; f < kFields; ++f) bits += 1u + tab_len(tab, ((w >> (f * LB)) & kMask) + 1u);
+        } else {
+          for (uint32_t f = 0; f < cnt; ++f) bits += 1u + tab_len(tab, ((w >> (f * LB)) & kMask) + 1u);
+        }
+      }
+    }
+    return bits;
+  }
   for (uint32_t c = c_lo; c < c_hi; ++c) bits += 1u + tab_len(tab, level_at<LB>(lwb, c) + 1u);
   return bits;
 }
@@ -329,7 +352,7 @@ __device__ __forceinline__ uint32_t lane_bits(const uint32_t* tab, const uint32_
   uint32_t bits = 0;
   int32_t prev = -1;
   if (DENSE) {
-    if (live) bits = summarize_dense<LB>(tab, lwb, c_lo, c_hi);
+    if (live) bits = summarize_dense<LB>(tab, lwb, c_lo, c_hi, whole_blocks);
   } else {
     LaneSummary s{0u, -1, -1};
     if (live) s = summarize_sparse<LB>(tab, lwb, c_lo, c_hi, whole_blocks);
@@ -564,7 +587,27 @@ __global__ void __launch_bounds__(kThreads) elias_scatter_kernel(const BucketPar
     StageWriter bw;
     bw.begin(stage, lead + bucket_off + (linc - bits));
     if (tl == 0) bw.put(__float_as_uint(__ldg(p.A + b)), 32);
-    if (DENSE) {
+    if (DENSE && (p.seg & 63u) == 0u) {
+      // ranges of whole 64-coordinate blocks: sign and level words are loaded once per block and word
+      constexpr uint32_t kFields = 32u / LB, kMask = (1u << LB) - 1u;
+      for (uint32_t c0 = c_lo; c0 < c_hi; c0 += 64u) {
+        const uint32_t* wp = lwb + ((c0 * LB) >> 5);
+        const uint32_t s0 = __ldg(swb + (c0 >> 5)), s1 = (c0 + 32u < c_hi) ? __ldg(swb + (c0 >> 5) + 1) : 0u;
+        const unsigned long long signs = (unsigned long long)s0 | ((unsigned long long)s1 << 32);
+#pragma unroll
+        for (uint32_t j = 0; j < 2u * LB; ++j) {
+          const uint32_t off = j * kFields;                   // first coordinate of this word in the block
+          if (c0 + off >= c_hi) break;
+          const uint32_t w = __ldg(wp + j);
+          const uint32_t cnt = min(kFields, c_hi - (c0 + off));
+          for (uint32_t f = 0; f < cnt; ++f) {
+            uint32_t ln;
+            const uint32_t code = tab_code(tab, ((w >> (f * LB)) & kMask) + 1u, &ln);
+            bw.put((((uint32_t)(signs >> (off + f)) & 1u) << ln) | code, ln + 1);
+          }
+        }
+      }
+    } else if (DENSE) {
       for (uint32_t c = c_lo; c < c_hi; ++c) {
         const uint32_t sg = (__ldg(swb + (c >> 5)) >> (c & 31)) & 1u;
         uint32_t ln;
