@@ -34,6 +34,8 @@ __device__ __forceinline__ uint32_t parse_to_fields(const PeerSet& peers, uint32
   uint32_t used = 0, err = 0;
   // The row is zero and only this lane writes it, so fields are OR-ed in place.
   if (DENSE) {
+    // every coordinate is coded, in order: level and sign words fill up in registers and are stored whole
+    uint32_t lw = 0u, sg = 0u;
     for (uint32_t c = 0; c < db; ++c) {
       src.refill();
       const uint32_t neg = src.hi >> 31;
@@ -41,12 +43,16 @@ __device__ __forceinline__ uint32_t parse_to_fields(const PeerSet& peers, uint32
       if (!read_int(src, lut, 1u, v, used)) { err = QSGD_DEV_OVERRUN; break; }
       if (used > total) { err = QSGD_DEV_OVERRUN; break; }
       if (v - 1u > s) { err = QSGD_DEV_LEVEL; break; }
-      if (v > 1u) {
-        row[(c * LB) >> 5] |= (v - 1u) << ((c * LB) & 31);
-        if (neg) srow[c >> 5] |= 1u << (c & 31);
-      }
+      lw |= (v - 1u) << ((c * LB) & 31);
+      sg |= (v > 1u ? neg : 0u) << (c & 31);
+      if ((((c + 1u) * LB) & 31u) == 0u) { row[(c * LB) >> 5] = lw; lw = 0u; }
+      if (((c + 1u) & 31u) == 0u) { srow[c >> 5] = sg; sg = 0u; }
     }
-    if (!err && used != total) err = QSGD_DEV_OVERRUN;
+    if (!err) {
+      if ((db * LB) & 31u) row[(db * LB) >> 5] = lw;          // a last word that did not fill up
+      if (db & 31u) srow[db >> 5] = sg;
+      if (used != total) err = QSGD_DEV_OVERRUN;
+    }
   } else {
     uint32_t at = 0xFFFFFFFFu;                        // position of the previous nonzero (-1)
     while (used < total) {
@@ -304,7 +310,11 @@ __global__ void __launch_bounds__(128) decode_elias_ranged_kernel(const __grid_c
       if (readable) {
         uint32_t* srow = row + kLevelWords;
         if (DENSE) {
-          for (uint32_t c = rbeg; c < min(rend, db) && st.err == 0u; ++c) {
+          // every coordinate is coded, in order: level and sign words fill up in registers and are
+          // stored whole (the row is zero, and a range starts on a word boundary)
+          const uint32_t lim = min(rend, db), cnt = lim > rbeg ? lim - rbeg : 0u;
+          uint32_t lw = 0u, sg = 0u;
+          for (uint32_t pos = 0; pos < cnt && st.err == 0u; ++pos) {
             st.src.refill();
             const uint32_t neg = st.src.hi >> 31;
             uint32_t v, len;
@@ -313,11 +323,16 @@ __global__ void __launch_bounds__(128) decode_elias_ranged_kernel(const __grid_c
             st.used += len + 1u;
             if (!ok || st.used > st.total) st.err = QSGD_DEV_OVERRUN;
             else if (v - 1u > p.s) st.err = QSGD_DEV_LEVEL;
-            else if (v > 1u) {
-              const uint32_t pos = c - rbeg;
-              row[(pos * LB) >> 5] |= (v - 1u) << ((pos * LB) & 31);
-              srow[pos >> 5] |= neg << (pos & 31);
+            else {
+              lw |= (v - 1u) << ((pos * LB) & 31);
+              sg |= (v > 1u ? neg : 0u) << (pos & 31);
             }
+            if ((((pos + 1u) * LB) & 31u) == 0u) { row[(pos * LB) >> 5] = lw; lw = 0u; }
+            if (((pos + 1u) & 31u) == 0u) { srow[pos >> 5] = sg; sg = 0u; }
+          }
+          if (st.err == 0u && cnt) {                        // a last word that did not fill up
+            if ((cnt * LB) & 31u) row[(cnt * LB) >> 5] = lw;
+            if (cnt & 31u) srow[cnt >> 5] = sg;
           }
         } else {
           advance(st, rend, 0xFFFFFFFFu, db, p.s, [&](uint32_t, uint32_t en) {
