@@ -186,10 +186,16 @@ class ClockSampler:
 class HotPath:
     """Buffers and one step of the hot path for a workload on one GPU."""
 
-    def __init__(self, wl, device, rank=0):
+    def __init__(self, wl, device, rank=0, streams=1):
         import torch
         import paper_1610_02132_b200 as Q
         self.torch, self.Q, self.wl, self.dev = torch, Q, wl, device
+        # The K workers' encodes are independent of one another; issued round-robin on `streams`
+        # streams (a workspace each) the tail of one encode runs beside the head of the next. The
+        # decode waits for all of them on the caller's stream.
+        self.n_streams = max(1, streams)
+        self.side = [torch.cuda.Stream(device=device) for _ in range(self.n_streams)] if self.n_streams > 1 else []
+        self.use_streams = self.n_streams > 1
         n, d, s, K = wl["n"], wl["d"], wl["s"], wl["K"]
         self.n, self.d, self.s, self.K = n, d, s, K
         self.B = (n + d - 1) // d
@@ -214,7 +220,7 @@ class HotPath:
             self.msgs[code] = [torch.empty(cap, dtype=torch.uint8, device=device) for _ in range(K)]
             self.bits[code] = torch.zeros(K, 4, dtype=torch.int64, device=device)
             wsb = max(Q.qsgd_workspace_bytes(self.nq, d, s, code), 16)
-            self.ws[code] = torch.empty(wsb, dtype=torch.uint8, device=device)
+            self.ws[code] = [torch.empty(wsb, dtype=torch.uint8, device=device) for _ in range(self.n_streams)]
         self.info = {}
 
     def message_capacity(self, code):
@@ -226,16 +232,34 @@ class HotPath:
         worst = Q.qsgd_message_capacity(self.nq, self.d, self.s, code)
         return self.prefix + min(worst, 2 * fixed_bytes(self.nq, self.d, self.s) + 8 * (self.B + 1))
 
-    def encode_all(self, code, step, src=None):
+    def encode_one(self, code, step, w, g, ws, stream=None):
         Q = self.Q
+        if self.plan is not None:
+            Q.qsgd_policy_encode(g, self.plan, self.s, self.norm, code, PHILOX_SEED, step, w,
+                                 self.msgs[code][w], self.bits[code][w], ws, self.status, stream=stream)
+        else:
+            Q.qsgd_encode(g, self.d, self.s, self.norm, code, PHILOX_SEED, step, w,
+                          self.msgs[code][w], self.bits[code][w], ws, self.status, stream=stream)
+
+    def encode_all(self, code, step, src=None):
+        torch = self.torch
         g = self.g if src is None else src
+        if not self.use_streams:
+            for w in range(self.K):
+                self.encode_one(code, step, w, g[w], self.ws[code][0])
+            return
+        main = torch.cuda.current_stream(self.dev)
+        fork = torch.cuda.Event()
+        fork.record(main)
+        for st in self.side:
+            st.wait_event(fork)                    # whatever wrote g, x or the messages before is done
         for w in range(self.K):
-            if self.plan is not None:
-                Q.qsgd_policy_encode(g[w], self.plan, self.s, self.norm, code, PHILOX_SEED, step, w,
-                                     self.msgs[code][w], self.bits[code][w], self.ws[code], self.status)
-            else:
-                Q.qsgd_encode(g[w], self.d, self.s, self.norm, code, PHILOX_SEED, step, w,
-                              self.msgs[code][w], self.bits[code][w], self.ws[code], self.status)
+            i = w % self.n_streams
+            self.encode_one(code, step, w, g[w], self.ws[code][i], stream=self.side[i])
+        for st in self.side:
+            join = torch.cuda.Event()
+            join.record(st)
+            main.wait_event(join)
 
     def read_info(self, code):
         """Message sizes of the last encode (a host read-back; outside the timed step except under
@@ -332,7 +356,7 @@ def run_cuda(args):
     if args.codes:
         wl["codes"] = args.codes.split(",")
 
-    hp = HotPath(wl, device, rank)
+    hp = HotPath(wl, device, rank, streams=args.streams)
     n, K = hp.n, hp.K
 
     def barrier():
@@ -354,32 +378,38 @@ def run_cuda(args):
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
-    # The K timed steps run twice. First as a user runs them: nothing between the kernels, so each
-    # kernel's CTAs are placed while the one ahead drains (programmatic dependent launch); this pass
-    # gives `value`. Then once more with a pair of CUDA events around every kernel launch on the
-    # launching stream, which gives the per-kernel durations of the roofline and the kernel table
-    # (and, the events serialising the launches, a step a few per cent longer: ms_per_step_with_events).
+    # The K timed steps run three times. First as a caller with K independent workers' gradients on
+    # one GPU runs them: the encodes issued round-robin on --streams streams (default 2, a workspace
+    # each), the decode after all of them, nothing between the kernels; this pass gives `value`.
+    # Then on one stream (`one_stream`: every kernel strictly after the one before). Then on one
+    # stream with a pair of CUDA events around every kernel launch on the launching stream, which
+    # gives the per-kernel durations of the roofline and the kernel table (and, the events
+    # serialising the launches, a step a few per cent longer: ms_per_step_with_events).
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed_steps(first):
+        barrier()
+        ev0.record()
+        for i in range(args.steps):
+            hp.step(first + i)
+        ev1.record()
+        barrier()
+        return ev0.elapsed_time(ev1)
+
     launches0 = Q.qsgd_launch_count()
-    barrier()
-    ev0.record()
-    for i in range(args.steps):
-        hp.step(args.warmup + i)
-    ev1.record()
-    barrier()
-    ms = ev0.elapsed_time(ev1)
+    ms = timed_steps(args.warmup)
     launches = Q.qsgd_launch_count() - launches0
+    ms_one_stream = ms / args.steps
+    if hp.use_streams:
+        hp.use_streams = False
+        hp.step(args.warmup)
+        ms_one_stream = timed_steps(args.warmup + args.steps) / args.steps
     Q.qsgd_profile_enable(True)
     Q.qsgd_profile_collect()
-    barrier()
-    ev0.record()
-    for i in range(args.steps):
-        hp.step(args.warmup + args.steps + i)
-    ev1.record()
-    barrier()
-    ms_events = ev0.elapsed_time(ev1) / args.steps
+    ms_events = timed_steps(args.warmup + 2 * args.steps) / args.steps
     Q.qsgd_profile_enable(False)
     kern = Q.qsgd_profile_collect()
+    hp.use_streams = hp.n_streams > 1
     clocks = sampler.stop() if rank == 0 else None
     assert int(hp.status.item()) == 0
     t = torch.tensor([ms], dtype=torch.float64, device=device)
@@ -466,7 +496,7 @@ def run_cuda(args):
                         landed[b].record(copy_stream)
                     main.wait_event(landed[b])
                     Q.qsgd_encode(stage[b], hp.d, hp.s, hp.norm, code, PHILOX_SEED, i, w, hp.msgs[code][w],
-                                  hp.bits[code][w], hp.ws[code], hp.status)
+                                  hp.bits[code][w], hp.ws[code][0], hp.status)
                     taken[b].record(main)
                 hp.decode(code)
                 x_host.copy_(hp.x, non_blocking=True)
@@ -505,14 +535,16 @@ def run_cuda(args):
         line = {
             "metric": "QSGD encode + decode+aggregate throughput, fp32 gradient GB/s",
             "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_step, "ms_per_step_with_events": ms_events,
+            "ms_per_step": ms_step, "ms_per_step_one_stream": ms_one_stream, "ms_per_step_with_events": ms_events,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload + ": " + wl["desc"], "n": n, "bucket": hp.d, "s": hp.s,
                        "norm": wl["norm"], "codes": wl["codes"], "K": K,
                        "l2": "inputs larger than L2 (K gradients = %.0f MB rotate through 126 MB)" % (K * 4 * n / 1e6),
                        "step": "per code kind: K encodes, fused decode+aggregate+SGD (tables found on the device; "
-                               "no host read-back inside a step)"},
+                               "no host read-back inside a step)",
+                       "streams": "the K independent encodes issued round-robin on %d stream(s), a workspace each; "
+                                  "the decode after all of them" % hp.n_streams},
             "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "roofline": roofline, "cpu_baseline": cpu, "phases": phases, "kernels": kern_tab,
         }
@@ -915,6 +947,8 @@ def main():
     ap.add_argument("--K", type=int, default=None)
     ap.add_argument("--norm", default=None, choices=["l2", "max"])
     ap.add_argument("--codes", default=None, help="comma list of fixed,elias,elias_dense")
+    ap.add_argument("--streams", type=int, default=2,
+                    help="streams the K independent encodes of a step are issued on (1 = everything on one stream)")
     ap.add_argument("--no-chaining", action="store_true",
                     help="plain stream-ordered launches (no programmatic dependent launch)")
     ap.add_argument("--e2e-steps", type=int, default=2)
