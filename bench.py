@@ -5,7 +5,10 @@ SGD step, through the C ABI (include/qsgd.h).
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
 
 One step = one pass of the whole hot path over one batch of synthetic gradients: for every code
-kind of the workload, K worker encodes followed by one fused decode + aggregate + SGD step.
+kind of the workload, K worker encodes followed by one fused decode + aggregate + SGD step. The K
+encodes are independent of one another and are issued round-robin on --streams streams (default 2);
+`ms_per_step_one_stream` is the same step with everything on one stream, and the per-kernel figures
+come from a third pass with CUDA events around every launch.
 Prints ONE JSON line (rank 0). Timing is on the device with CUDA events; inputs are resident in
 HBM before the timed region for `value`, and copied from pinned host memory inside it for `e2e`.
 """
