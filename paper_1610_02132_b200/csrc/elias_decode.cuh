@@ -32,7 +32,7 @@ struct SparseShape {
   uint32_t Kpad;      // lanes per bucket: K rounded up to a power of two
   uint32_t G;         // buckets per warp
   uint32_t R;         // positions per range; G * R <= 2048 sums per warp
-  uint32_t C;         // entries per list and range: one per 32 positions, at least 16
+  uint32_t C;         // entries per list and range: one per 32 positions, at least 16, a multiple of 4
 };
 
 inline SparseShape sparse_shape(uint32_t K, uint32_t d, uint64_t B, uint32_t sms) {
@@ -45,6 +45,7 @@ inline SparseShape sparse_shape(uint32_t K, uint32_t d, uint64_t B, uint32_t sms
   if (sh.R > 1024u) sh.R = 1024u;
   if (d <= sh.R) sh.R = d;                 // whole bucket in one range
   sh.C = sh.R / 32u > 16u ? sh.R / 32u : 16u;
+  sh.C = (sh.C + 3u) & ~3u;                // keeps every warp's share of shared memory a multiple of 16 bytes
   return sh;
 }
 

@@ -48,9 +48,10 @@ def make_input(family, n, seed):
 
 
 # QSGD_FUZZ_CASES / QSGD_FUZZ_POLICY_CASES draw more cases from the same seeds (the defaults are a prefix)
+SEED0 = int(os.environ.get("QSGD_FUZZ_SEED", "0"))          # shifts every case's seed: a different campaign
 N_CASES = int(os.environ.get("QSGD_FUZZ_CASES", "72"))
 N_POLICY_CASES = int(os.environ.get("QSGD_FUZZ_POLICY_CASES", "40"))
-CASES = [draw_case(np.random.default_rng(1000 + i)) for i in range(N_CASES)]
+CASES = [draw_case(np.random.default_rng(1000 + SEED0 + i)) for i in range(N_CASES)]
 
 
 @pytest.mark.parametrize("case", CASES, ids=["n%d_d%d_s%d_norm%d_code%d_K%d_%s" % c for c in CASES])
@@ -101,7 +102,7 @@ def draw_policy_case(rng):
     return tuple(sizes), d, s, norm_kind, code_kind, K, tau
 
 
-POLICY_CASES = [draw_policy_case(np.random.default_rng(5000 + i)) for i in range(N_POLICY_CASES)]
+POLICY_CASES = [draw_policy_case(np.random.default_rng(5000 + SEED0 + i)) for i in range(N_POLICY_CASES)]
 
 
 @pytest.mark.parametrize("case", POLICY_CASES,
@@ -124,7 +125,7 @@ def draw_mid_case(rng):
     return n, d, s, norm_kind, code_kind, family
 
 
-MID_CASES = [draw_mid_case(np.random.default_rng(9000 + i)) for i in range(int(os.environ.get("QSGD_FUZZ_MID_CASES", "10")))]
+MID_CASES = [draw_mid_case(np.random.default_rng(9000 + SEED0 + i)) for i in range(int(os.environ.get("QSGD_FUZZ_MID_CASES", "10")))]
 
 
 @pytest.mark.parametrize("case", MID_CASES, ids=["n%d_d%d_s%d_norm%d_code%d_%s" % c for c in MID_CASES])

@@ -223,7 +223,10 @@ def sparse_regime_bits(K, d):
                                            (3 * 4096 + 1, 4096, 1, 1, 0.3), (70 * 64 + 9, 64, 3, 16, 0.98),
                                            # enough buckets that a warp takes its full share of them
                                            (7200 * 64 + 5, 64, 1, 8, 0.98), (14300 * 128 + 3, 128, 1, 3, 0.95),
-                                           (57000 * 32 + 31, 32, 1, 1, 0.98)])
+                                           (57000 * 32 + 31, 32, 1, 1, 0.98),
+                                           # few buckets of a size that is no power of two, one or two peers:
+                                           # one bucket per warp, lists of 928 / 32 = 29 and 608 / 32 = 19 entries
+                                           (46 * 928, 928, 1, 1, 0.3), (30 * 608 - 3, 608, 1, 2, 0.7)])
 @pytest.mark.parametrize("eta", [0.1, -0.25])
 def test_elias_sparse_regime(n, d, s, K, zeros, eta):
     msgs, infos = [], []
