@@ -24,7 +24,7 @@ def draw_case(rng):
     s = int(rng.choice([1, 2, 3, 4, 7, 15, 15, 16, 31, 64, 200, 255]))
     norm_kind = int(rng.choice([O.NORM_L2, O.NORM_MAX]))
     code_kind = int(rng.choice([O.CODE_FIXED, O.CODE_ELIAS, O.CODE_ELIAS, O.CODE_ELIAS_DENSE]))
-    K = int(rng.choice([1, 2, 3, 4, 5, 8, 16, 17, 33]))
+    K = int(rng.choice([1, 2, 3, 4, 5, 8, 16, 17, 33, 64]))
     family = str(rng.choice(["mixture", "gauss", "sparse", "tiny_values", "huge_values", "zeros_inside"]))
     return n, d, s, norm_kind, code_kind, K, family
 
