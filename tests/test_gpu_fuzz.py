@@ -137,3 +137,40 @@ def test_random_mid_size_matches_oracle(case):
         msgs.append(m)
         infos.append(info)
     decode_parity(msgs, infos, n, d, s, code_kind, eta=0.05, x0=I.gaussian(n, 1.0, seed=78))
+
+
+CAP_CASES = [(draw_case(np.random.default_rng(13000 + SEED0 + i)), float(np.random.default_rng(13000 + SEED0 + i).uniform(0.0, 1.15)))
+             for i in range(int(os.environ.get("QSGD_FUZZ_CAPACITY_CASES", "30")))]
+
+
+@pytest.mark.parametrize("case,frac", CAP_CASES, ids=["n%d_d%d_s%d_norm%d_code%d_K%d_%s" % c + "_f%.2f" % f for c, f in CAP_CASES])
+def test_random_message_capacity(case, frac):
+    """An Elias encode into a buffer between the smallest size the host accepts and a little more than
+    the message needs: either the message is there, identical to the unconstrained one, or the
+    capacity flag is up, the size needed is reported and not a byte of the buffer was written."""
+    import paper_1610_02132_b200 as Q
+    from parity_util import CANARY, gpu_encode
+    n, d, s, norm_kind, code_kind, K, family = case
+    if code_kind == O.CODE_FIXED:
+        code_kind = O.CODE_ELIAS
+    g_dev = torch.from_numpy(make_input(family, n, seed=21)).cuda()
+    full, info, st, _ = gpu_encode(g_dev, d, s, norm_kind, code_kind, 4, 2, 1)
+    assert st == 0
+    need = info[2]
+    B = O.n_buckets(n, d)
+    floor = 16 * ((4 * B + 15) // 16) + 8 * (B + 1)             # scales and table: the host's minimum
+    cap = (floor + int(frac * (need - floor))) // 16 * 16
+    cap = max(cap, floor)
+    big, info2, st2, _ = gpu_encode(g_dev, d, s, norm_kind, code_kind, 4, 2, 1, capacity=cap) if cap >= need else (None, None, None, None)
+    if cap >= need:
+        assert st2 == 0 and info2 == info and torch.equal(big[:need], full[:need])
+        return
+    buf = torch.full((cap + 256,), CANARY, dtype=torch.uint8, device="cuda")
+    bits = torch.zeros(4, dtype=torch.int64, device="cuda")
+    ws = torch.empty(max(Q.qsgd_workspace_bytes(n, d, s, code_kind), 16), dtype=torch.uint8, device="cuda")
+    status = Q.new_status("cuda")
+    Q.qsgd_encode(g_dev, d, s, norm_kind, code_kind, 4, 2, 1, buf[:cap], bits, ws, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == Q.binding.DEV_CAPACITY
+    assert bool((buf == CANARY).all()), "bytes written into a buffer that is too small"
+    assert int(bits.cpu().numpy().view(np.uint64)[2]) == need
