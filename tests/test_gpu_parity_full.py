@@ -248,3 +248,31 @@ def test_config5_sweep_quick_whole(d, s, norm, code):
         msgs.append(m)
         infos.append(info)
     decode_parity(msgs, infos, n, d, s, code)
+
+
+# Maximum sizes: index arithmetic past 2^31 coordinates on the whole path, and the largest n the ABI
+# takes (QSGD_MAX_COORDS = 2^32) on Encode. Sampled buckets; about 55 GB on the device at the peak.
+@pytest.mark.parametrize("d,s,norm,code", [(512, 15, O.NORM_L2, O.CODE_FIXED), (512, 15, O.NORM_L2, O.CODE_ELIAS),
+                                           (4096, 1, O.NORM_MAX, O.CODE_ELIAS)])
+def test_beyond_2_31_coordinates_sampled(d, s, norm, code):
+    n = 2 ** 31 + 777
+    gs = [I.gaussian_mixture_device(n, 31 + w, device="cuda") for w in range(2)]
+    run_sampled_config(gs, n, d, s, norm, code, step=2, nsample=40)
+    del gs
+    torch.cuda.empty_cache()
+
+
+def test_largest_n_encode_sampled():
+    n = 2 ** 32 - 4096 * 3 - 5
+    g = I.gaussian_mixture_device(n, 5, device="cuda")
+    for d, s, norm, code in [(512, 15, O.NORM_L2, O.CODE_FIXED), (512, 3, O.NORM_L2, O.CODE_ELIAS)]:
+        B = O.n_buckets(n, d)
+        cap = min(Q.qsgd_message_capacity(n, d, s, code),
+                  2 * Q.qsgd_message_capacity(n, d, s, O.CODE_FIXED) + 8 * (B + 1))
+        big, info, st, _ = gpu_encode(g, d, s, norm, code, SEED, 1, 0, capacity=cap)
+        assert st == 0
+        check_sampled(g, big, info, n, d, s, norm, code, 1, 0, sample_buckets(B, 40, seed=7))
+        del big
+        torch.cuda.empty_cache()
+    del g
+    torch.cuda.empty_cache()
