@@ -261,3 +261,46 @@ def test_elias_sparse_regime_long_lists(d, s, Bn):
         infos.append(info)
     assert sum(i[0] for i in infos) < K * Bn * sparse_regime_bits(K, d), "case is not in the sparse regime"
     decode_parity(msgs, infos, n, d, s, O.CODE_ELIAS, eta=0.5, x0=I.gaussian(n, 1.0, seed=1))
+
+
+@pytest.mark.parametrize("d,s,code_kind", [(512, 15, O.CODE_FIXED), (512, 15, O.CODE_ELIAS), (4096, 1, O.CODE_ELIAS),
+                                           (128, 255, O.CODE_ELIAS_DENSE), (96, 3, O.CODE_FIXED)])
+def test_pointers_with_the_minimum_alignment(d, s, code_kind):
+    """Every pointer the ABI takes needs 16-byte alignment and no more: gradient, message, workspace,
+    accumulator and parameters all sit 16 (or 48) bytes into their allocations here."""
+    n, K = 6 * 4096 + 2 * d + 13, 3
+    dev = "cuda"
+    status = Q.new_status(dev)
+    cap = Q.qsgd_message_capacity(n, d, s, code_kind)
+    wsb = max(Q.qsgd_workspace_bytes(n, d, s, code_kind), 16)
+    ws = torch.empty(wsb + 64, dtype=torch.uint8, device=dev)[48: 48 + wsb]
+    msgs, infos, ref_msgs, ref_tabs = [], [], [], []
+    for w in range(K):
+        g = I.gaussian_mixture(n, seed=60 + w)
+        g_dev = torch.empty(n + 8, dtype=torch.float32, device=dev)[4: 4 + n]
+        g_dev.copy_(torch.from_numpy(g))
+        out = torch.zeros(cap + 64, dtype=torch.uint8, device=dev)[16: 16 + cap]
+        bits = torch.zeros(4, dtype=torch.int64, device=dev)
+        Q.qsgd_encode(g_dev, d, s, O.NORM_MAX, code_kind, 3, 1, w, out, bits, ws, status)
+        torch.cuda.synchronize()
+        info = [int(v) for v in bits.cpu()]
+        m, ref_info = O.encode(g, d, s, O.NORM_MAX, code_kind, 3, 1, w)
+        assert info == ref_info
+        assert np.array_equal(out[: m.size].cpu().numpy(), m)
+        msgs.append(out)
+        infos.append(bits)
+        ref_msgs.append(m)
+        ref_tabs.append(O.message_table(m, ref_info, n, d) if code_kind != O.CODE_FIXED else None)
+    x0 = I.gaussian(n, 1.0, seed=4)
+    x = torch.empty(n + 24, dtype=torch.float32, device=dev)[12: 12 + n]
+    x.copy_(torch.from_numpy(x0))
+    acc = torch.empty(n + 8, dtype=torch.float32, device=dev)[4: 4 + n]
+    elias = code_kind != O.CODE_FIXED
+    Q.qsgd_decode_accumulate_packed(msgs, infos if elias else None, n, d, s, code_kind, acc, status)
+    Q.qsgd_decode_sgd_step_packed(msgs, infos if elias else None, n, d, s, code_kind, x, 0.1, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    st, acc_ref = O.decode_accumulate(ref_msgs, ref_tabs if elias else None, n, d, s, code_kind)
+    assert st == 0
+    assert np.array_equal(acc.cpu().numpy().view(np.uint32), acc_ref.view(np.uint32))
+    assert np.array_equal(x.cpu().numpy().view(np.uint32), O.sgd_step(x0, acc_ref, 0.1, K).view(np.uint32))
