@@ -117,7 +117,7 @@ def draw_mid_case(rng):
     # enough tiles for every persistent warp / CTA of the streaming encoders to go round its ring
     # of stages several times (2.4 M coordinates fill the grid once)
     d = int(rng.choice([32, 128, 512, 1024, 4096]))
-    n = int(rng.integers(5_000_000, 14_000_000))
+    n = int(rng.integers(1_500_000, 14_000_000))      # from less than one tile per CTA of the grid to several
     s = int(rng.choice([1, 3, 15, 255]))
     norm_kind = int(rng.choice([O.NORM_L2, O.NORM_MAX]))
     code_kind = int(rng.choice([O.CODE_FIXED, O.CODE_ELIAS, O.CODE_ELIAS_DENSE]))
