@@ -255,6 +255,26 @@ __global__ void __launch_bounds__(128) decode_elias_ranged_kernel(const __grid_c
   constexpr uint32_t kLevelWords = kR * LB / 32, kRowWords = kLevelWords + kR / 32;
   extern __shared__ __align__(16) uint32_t fsm[];
   __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
+  // Dense code: the next kDenseBits stream bits usually hold two or three whole (sign, Elias(level + 1))
+  // symbols (2, 4, 4, 7 bits for levels 0 .. 3). Entry: symbols held (0 .. 3) | their total length << 2 |
+  // (level | negative << 3) << (6 + 4 j) for symbol j; only levels <= min(s, 7) are listed.
+  constexpr uint32_t kDenseBits = 10;
+  __shared__ uint32_t dense_lut[DENSE ? (1u << kDenseBits) : 1u];
+  if (DENSE) {
+    for (uint32_t i = threadIdx.x; i < (1u << kDenseBits); i += blockDim.x) {
+      uint32_t w = i << (32 - kDenseBits), used = 0, held = 0, entry = 0;
+      while (held < 3u && used + 2u <= kDenseBits) {
+        const uint32_t neg = w >> 31;
+        uint32_t v, len;
+        if (!elias_from_window(w << 1, v, len) || used + 1u + len > kDenseBits || v - 1u > min(p.s, 7u)) break;
+        entry |= ((v - 1u) | (neg << 3)) << (6u + 4u * held);
+        w <<= 1u + len;
+        used += 1u + len;
+        ++held;
+      }
+      dense_lut[i] = held | (used << 2) | entry;
+    }
+  }
   chain_wait();                                   // the messages come from the kernels ahead
   if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -314,8 +334,30 @@ __global__ void __launch_bounds__(128) decode_elias_ranged_kernel(const __grid_c
           // stored whole (the row is zero, and a range starts on a word boundary)
           const uint32_t lim = min(rend, db), cnt = lim > rbeg ? lim - rbeg : 0u;
           uint32_t lw = 0u, sg = 0u;
-          for (uint32_t pos = 0; pos < cnt && st.err == 0u; ++pos) {
+          auto put = [&](uint32_t pos, uint32_t level, uint32_t neg) {
+            lw |= level << ((pos * LB) & 31);
+            sg |= (level ? neg : 0u) << (pos & 31);
+            if ((((pos + 1u) * LB) & 31u) == 0u) { row[(pos * LB) >> 5] = lw; lw = 0u; }
+            if (((pos + 1u) & 31u) == 0u) { srow[pos >> 5] = sg; sg = 0u; }
+          };
+          uint32_t pos = 0;
+          while (pos < cnt && st.err == 0u) {
             st.src.refill();
+            const uint32_t e = dense_lut[st.src.hi >> (32 - kDenseBits)];
+            const uint32_t held = e & 3u;
+            if (held != 0u && pos + held <= cnt) {            // two or three symbols at once (or one)
+              put(pos, (e >> 6) & 7u, (e >> 9) & 1u);
+              if (held > 1u) put(pos + 1u, (e >> 10) & 7u, (e >> 13) & 1u);
+              if (held > 2u) put(pos + 2u, (e >> 14) & 7u, (e >> 17) & 1u);
+              const uint32_t len = (e >> 2) & 15u;
+              st.src.drop(len);
+              st.used += len;
+              pos += held;
+              if (st.used > st.total) st.err = QSGD_DEV_OVERRUN;
+              continue;
+            }
+            // one symbol by the definition's decoder: a level above 7, or fewer coordinates left
+            // in the range than the entry holds
             const uint32_t neg = st.src.hi >> 31;
             uint32_t v, len;
             const bool ok = elias_from_window(st.src.hi << 1, v, len);
@@ -323,12 +365,8 @@ __global__ void __launch_bounds__(128) decode_elias_ranged_kernel(const __grid_c
             st.used += len + 1u;
             if (!ok || st.used > st.total) st.err = QSGD_DEV_OVERRUN;
             else if (v - 1u > p.s) st.err = QSGD_DEV_LEVEL;
-            else {
-              lw |= (v - 1u) << ((pos * LB) & 31);
-              sg |= (v > 1u ? neg : 0u) << (pos & 31);
-            }
-            if ((((pos + 1u) * LB) & 31u) == 0u) { row[(pos * LB) >> 5] = lw; lw = 0u; }
-            if (((pos + 1u) & 31u) == 0u) { srow[pos >> 5] = sg; sg = 0u; }
+            else put(pos, v - 1u, neg);
+            ++pos;
           }
           if (st.err == 0u && cnt) {                        // a last word that did not fill up
             if ((cnt * LB) & 31u) row[(cnt * LB) >> 5] = lw;

@@ -304,3 +304,19 @@ def test_pointers_with_the_minimum_alignment(d, s, code_kind):
     assert st == 0
     assert np.array_equal(acc.cpu().numpy().view(np.uint32), acc_ref.view(np.uint32))
     assert np.array_equal(x.cpu().numpy().view(np.uint32), O.sgd_step(x0, acc_ref, 0.1, K).view(np.uint32))
+
+
+@pytest.mark.parametrize("d", [1024, 4096])
+@pytest.mark.parametrize("s,norm_kind", [(3, O.NORM_L2), (64, O.NORM_L2), (255, O.NORM_MAX), (7, O.NORM_MAX), (8, O.NORM_MAX)])
+def test_dense_code_long_buckets(d, s, norm_kind):
+    """Code'_s with d >= 1024: the decoder takes up to three symbols per table lookup when their levels
+    are at most min(s, 7) and a range has room for them, one symbol by the definition's decoder
+    otherwise (max-norm: every bucket holds level s; ragged last bucket; ranges of 512 positions)."""
+    n, K = 5 * d + d // 2 + 3, 3
+    msgs, infos = [], []
+    for w in range(K):
+        g = I.gaussian(n, 1.0, seed=500 + w)
+        m, info = encode_parity(g, d, s, norm_kind, O.CODE_ELIAS_DENSE, seed=8, step=2, worker=w)
+        msgs.append(m)
+        infos.append(info)
+    decode_parity(msgs, infos, n, d, s, O.CODE_ELIAS_DENSE, eta=0.3, x0=I.gaussian(n, 1.0, seed=2))
