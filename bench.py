@@ -316,13 +316,16 @@ def kernel_algorithmic_bytes(hp, code_name):
     MF = fixed_bytes(hp.nq, d, s)
     out = {"quantize_fixed": 4 * n + MF, "decode_fixed": K * MF + 8 * n, "sgd_step": 12 * n,
            "raw_gather": 8 * hp.n_raw, "raw_decode": (4 * K + 8) * hp.n_raw}
-    if 1 in hp.info:
-        info = hp.info[1]
+    for elias_code in (1, 2):                  # sparse code, else the dense code (a workload has one of them)
+        if elias_code not in hp.info:
+            continue
+        info = hp.info[elias_code]
         msg = float(np.mean(info[:, 2].astype(np.float64))) - hp.prefix
         pay = float(np.mean(info[:, 1].astype(np.float64))) - hp.prefix
         out.update({"decode_elias": K * msg + 8 * n, "decode_elias_sparse": K * msg + 8 * n,
                     "elias_scatter": MF + pay + 8 * (B + 1),
                     "elias_length": MF - 4 * ((n + 31) // 32) + 4 * B})
+        break
     return out
 
 
