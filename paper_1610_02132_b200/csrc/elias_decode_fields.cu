@@ -18,11 +18,32 @@ namespace qsgd {
 
 namespace {
 
+// Dense code: the next kDenseBits stream bits usually hold two or three whole (sign, Elias(level + 1))
+// symbols (2, 4, 4, 7 bits for levels 0 .. 3). Entry: symbols held (0 .. 3) | their total length << 2 |
+// (level | negative << 3) << (6 + 4 j) for symbol j; only levels <= min(s, 7) are listed.
+constexpr uint32_t kDenseBits = 10;
+
+__device__ __forceinline__ void fill_dense_lut(uint32_t* lut, uint32_t s) {
+  for (uint32_t i = threadIdx.x; i < (1u << kDenseBits); i += blockDim.x) {
+    uint32_t w = i << (32 - kDenseBits), used = 0, held = 0, entry = 0;
+    while (held < 3u && used + 2u <= kDenseBits) {
+      const uint32_t neg = w >> 31;
+      uint32_t v, len;
+      if (!elias_from_window(w << 1, v, len) || used + 1u + len > kDenseBits || v - 1u > min(s, 7u)) break;
+      entry |= ((v - 1u) | (neg << 3)) << (6u + 4u * held);
+      w <<= 1u + len;
+      used += 1u + len;
+      ++held;
+    }
+    lut[i] = held | (used << 2) | entry;
+  }
+}
+
 template <int LB, bool DENSE>
 __device__ __forceinline__ uint32_t parse_to_fields(const PeerSet& peers, uint32_t k, uint64_t b,
                                                     uint64_t B, uint32_t db, uint32_t d, uint32_t s,
-                                                    const uint16_t* lut, uint32_t* __restrict__ row,
-                                                    float* A_out) {
+                                                    const uint16_t* lut, const uint32_t* dense_lut,
+                                                    uint32_t* __restrict__ row, float* A_out) {
   *A_out = 0.f;
   const StringRef ref = string_ref(peers, k, b, B, db);
   if (ref.err) return ref.err;
@@ -34,19 +55,40 @@ __device__ __forceinline__ uint32_t parse_to_fields(const PeerSet& peers, uint32
   uint32_t used = 0, err = 0;
   // The row is zero and only this lane writes it, so fields are OR-ed in place.
   if (DENSE) {
-    // every coordinate is coded, in order: level and sign words fill up in registers and are stored whole
+    // every coordinate is coded, in order: level and sign words fill up in registers and are stored
+    // whole; up to three symbols per table lookup, one by the definition's decoder otherwise
     uint32_t lw = 0u, sg = 0u;
-    for (uint32_t c = 0; c < db; ++c) {
-      src.refill();
-      const uint32_t neg = src.hi >> 31;
-      uint32_t v;
-      if (!read_int(src, lut, 1u, v, used)) { err = QSGD_DEV_OVERRUN; break; }
-      if (used > total) { err = QSGD_DEV_OVERRUN; break; }
-      if (v - 1u > s) { err = QSGD_DEV_LEVEL; break; }
-      lw |= (v - 1u) << ((c * LB) & 31);
-      sg |= (v > 1u ? neg : 0u) << (c & 31);
+    auto put = [&](uint32_t c, uint32_t level, uint32_t neg) {
+      lw |= level << ((c * LB) & 31);
+      sg |= (level ? neg : 0u) << (c & 31);
       if ((((c + 1u) * LB) & 31u) == 0u) { row[(c * LB) >> 5] = lw; lw = 0u; }
       if (((c + 1u) & 31u) == 0u) { srow[c >> 5] = sg; sg = 0u; }
+    };
+    uint32_t c = 0;
+    while (c < db) {
+      src.refill();
+      const uint32_t e = dense_lut[src.hi >> (32 - kDenseBits)];
+      const uint32_t held = e & 3u;
+      if (held != 0u && c + held <= db) {
+        put(c, (e >> 6) & 7u, (e >> 9) & 1u);
+        if (held > 1u) put(c + 1u, (e >> 10) & 7u, (e >> 13) & 1u);
+        if (held > 2u) put(c + 2u, (e >> 14) & 7u, (e >> 17) & 1u);
+        const uint32_t len = (e >> 2) & 15u;
+        src.drop(len);
+        used += len;
+        c += held;
+        if (used > total) { err = QSGD_DEV_OVERRUN; break; }
+        continue;
+      }
+      const uint32_t neg = src.hi >> 31;
+      uint32_t v, len;
+      const bool ok = elias_from_window(src.hi << 1, v, len);
+      src.drop(len + 1u);
+      used += len + 1u;
+      if (!ok || used > total) { err = QSGD_DEV_OVERRUN; break; }
+      if (v - 1u > s) { err = QSGD_DEV_LEVEL; break; }
+      put(c, v - 1u, neg);
+      ++c;
     }
     if (!err) {
       if ((db * LB) & 31u) row[(db * LB) >> 5] = lw;          // a last word that did not fill up
@@ -97,13 +139,15 @@ template <int LB, bool DENSE, bool FUSED, bool SINGLE>
 __global__ void __launch_bounds__(320) decode_elias_fields_kernel(const __grid_constant__ FieldParams p) {
   extern __shared__ __align__(16) uint32_t fsm[];
   __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
-  __shared__ uint16_t elias_lut[1u << kLutBits];
+  __shared__ uint16_t elias_lut[DENSE ? 1u : (1u << kLutBits)];
+  __shared__ uint32_t dense_lut[DENSE ? (1u << kDenseBits) : 1u];
   chain_wait();                                   // the messages come from the kernels ahead
   if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
   const float sf = (float)p.s;
   float lut0 = 0.f;
-  fill_elias_lut(elias_lut);
+  if (DENSE) fill_dense_lut(dense_lut, p.s);
+  else fill_elias_lut(elias_lut);
   if (LB == 8) {
     for (uint32_t i = tid; i < 256 * 32; i += blockDim.x) xi_tab[i] = __fdiv_rn((float)(i >> 5), sf);
   }
@@ -136,7 +180,7 @@ __global__ void __launch_bounds__(320) decode_elias_fields_kernel(const __grid_c
         const uint32_t db = (uint32_t)min((uint64_t)p.d, p.n - base);
         float A;
         const uint32_t st = parse_to_fields<LB, DENSE>(p.peers, k, b, p.B, db, p.d,
-                                                       p.s, elias_lut, bucket + k * p.row_words, &A);
+                                                       p.s, elias_lut, dense_lut, bucket + k * p.row_words, &A);
         reinterpret_cast<float*>(bucket + p.K * p.row_words)[k] = A;
         if (st) atomicOr(p.status, st);
       }
@@ -255,26 +299,8 @@ __global__ void __launch_bounds__(128) decode_elias_ranged_kernel(const __grid_c
   constexpr uint32_t kLevelWords = kR * LB / 32, kRowWords = kLevelWords + kR / 32;
   extern __shared__ __align__(16) uint32_t fsm[];
   __shared__ __align__(16) float xi_tab[LB == 8 ? 256 * 32 : 32];
-  // Dense code: the next kDenseBits stream bits usually hold two or three whole (sign, Elias(level + 1))
-  // symbols (2, 4, 4, 7 bits for levels 0 .. 3). Entry: symbols held (0 .. 3) | their total length << 2 |
-  // (level | negative << 3) << (6 + 4 j) for symbol j; only levels <= min(s, 7) are listed.
-  constexpr uint32_t kDenseBits = 10;
   __shared__ uint32_t dense_lut[DENSE ? (1u << kDenseBits) : 1u];
-  if (DENSE) {
-    for (uint32_t i = threadIdx.x; i < (1u << kDenseBits); i += blockDim.x) {
-      uint32_t w = i << (32 - kDenseBits), used = 0, held = 0, entry = 0;
-      while (held < 3u && used + 2u <= kDenseBits) {
-        const uint32_t neg = w >> 31;
-        uint32_t v, len;
-        if (!elias_from_window(w << 1, v, len) || used + 1u + len > kDenseBits || v - 1u > min(p.s, 7u)) break;
-        entry |= ((v - 1u) | (neg << 3)) << (6u + 4u * held);
-        w <<= 1u + len;
-        used += 1u + len;
-        ++held;
-      }
-      dense_lut[i] = held | (used << 2) | entry;
-    }
-  }
+  if (DENSE) fill_dense_lut(dense_lut, p.s);
   chain_wait();                                   // the messages come from the kernels ahead
   if (!DENSE && p.defer_sparse && sparse_regime(p.peers, p.K, p.B, p.d)) return;
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
